@@ -1,0 +1,224 @@
+/*
+ * mixattn.h -- C ABI of the MixAttention inference attention library (sm_100a).
+ *
+ * The library implements the attention + KV-cache path of "Inference-Friendly
+ * Models With MixAttention" (arXiv 2409.15012): every layer is either a
+ * standard attention layer or a sliding-window layer with window s, and either
+ * computes its own KV cache or reuses the cache of an earlier layer
+ * (Section 3).  Grouped-query attention maps query head h to KV head
+ * h / (n_q_heads / n_kv_heads) (Section 3, last paragraph).
+ *
+ * Conventions for every call
+ *   - returns MIXATTN_OK (0) or a negative MIXATTN_ERR_* code; nothing throws,
+ *     aborts or traps.  All validation happens on the host before any launch,
+ *     and a failing call changes no state.
+ *   - "host" pointers are read (or written) before the call returns.
+ *     "device" pointers are borrowed until `stream` has executed the work the
+ *     call enqueued.  `stream` is a cudaStream_t passed as void* (NULL = the
+ *     legacy default stream).  Calls are asynchronous on that stream.
+ *   - a context is not thread-safe; use one stream at a time per context.
+ *   - tensors are dense, row-major, in the context's dtype (float or bf16).
+ */
+#ifndef MIXATTN_H_
+#define MIXATTN_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct mixattn_ctx mixattn_ctx; /* opaque; owned by the library */
+
+enum { MIXATTN_FULL = 0, MIXATTN_SLIDING = 1 };
+enum { MIXATTN_F32 = 0, MIXATTN_BF16 = 1 };
+
+enum {
+  MIXATTN_OK = 0,
+  MIXATTN_ERR_INVALID_ARG = -1,    /* null pointer, size out of range, duplicate sequence id        */
+  MIXATTN_ERR_INVALID_LAYOUT = -2, /* layer layout breaks the rules listed at mixattn_create        */
+  MIXATTN_ERR_NOT_OWNER = -3,      /* K/V offered to a layer that reuses another layer's cache      */
+  MIXATTN_ERR_OUT_OF_PAGES = -4,   /* the paged pool has too few free pages for the call            */
+  MIXATTN_ERR_EMPTY_CONTEXT = -5,  /* decode on a sequence whose cache holds no token               */
+  MIXATTN_ERR_BAD_SEQ = -6,        /* sequence id outside 0 .. max_seqs-1                           */
+  MIXATTN_ERR_UNSUPPORTED = -7,    /* valid request this build does not implement                   */
+  MIXATTN_ERR_CUDA = -8            /* a CUDA call failed, or the context is host-only               */
+};
+
+/* One layer of the layout (Section 3: a mix of sliding-window layers, standard
+ * layers and layers that reuse a KV cache).  `window` is the paper's s and is
+ * ignored for MIXATTN_FULL.  `kv_owner_layer` is the layer whose cache this
+ * layer reads: itself, or an earlier layer. */
+typedef struct {
+  int32_t kind;
+  int32_t window;
+  int32_t kv_owner_layer;
+} mixattn_layer_desc;
+
+typedef struct {
+  int32_t n_layers;
+  const mixattn_layer_desc* layers; /* host, n_layers entries, copied by create                    */
+  int32_t n_q_heads, n_kv_heads;    /* n_q_heads % n_kv_heads == 0                                  */
+  int32_t head_dim;                 /* 64 or 128                                                    */
+  int32_t dtype;                    /* MIXATTN_F32 or MIXATTN_BF16: type of Q, K, V, out and cache  */
+  int32_t max_seqs;                 /* sequence slots 0 .. max_seqs-1                               */
+  int32_t page_size;                /* tokens per page of the full-attention cache; must be 16      */
+  int32_t n_pages;                  /* physical pages per full-attention owner                      */
+  int32_t max_seq_len;              /* longest sequence; 0 = n_pages * page_size                    */
+  const int32_t* free_order;        /* host, optional permutation of 0..n_pages-1: initial FIFO
+                                       order of the free pages; NULL = 0,1,2,...                    */
+  float softmax_scale;              /* 0 = 1/sqrt(head_dim)                                         */
+  int32_t device;                   /* CUDA device ordinal; -1 = host-only context that keeps the
+                                       cache bookkeeping but launches nothing (append_kv then
+                                       ignores k/v; decode and prefill return MIXATTN_ERR_CUDA)     */
+  void* arena;                      /* device memory allocated by the caller, 256-byte aligned      */
+  size_t arena_bytes;               /* >= mixattn_arena_bytes(); the library never frees it         */
+} mixattn_config;
+
+/* Bytes of device memory a context with this config carves out of `arena`:
+ * K/V storage (see mixattn_cache_bytes), the device copy of the block tables
+ * and the split-KV workspace.  Writes *out_bytes.  Errors: INVALID_ARG,
+ * INVALID_LAYOUT. */
+int mixattn_arena_bytes(const mixattn_config* cfg, size_t* out_bytes);
+
+/* Bytes of K/V storage alone: one paged pool of n_pages pages per
+ * full-attention owner and one ring of `window` tokens (rounded up to whole
+ * 16-token pages) per sequence slot per sliding-window owner (Section 3: a
+ * window-s layer only stores the past s tokens).  Layers that reuse a cache
+ * add nothing (Section 3: l layers sharing one cache shrink it by 1/l). */
+int mixattn_cache_bytes(const mixattn_config* cfg, size_t* out_bytes);
+
+/* Builds a context.  Layout rules (Section 3: a layer may reuse the cache
+ * computed by an EARLIER layer), each violation -> MIXATTN_ERR_INVALID_LAYOUT:
+ *   0 <= kv_owner_layer <= layer index;  the owner owns itself (no chains);
+ *   a reader has its owner's kind and, if sliding, its owner's window >= 1.
+ * Other bad fields -> INVALID_ARG.  With device >= 0 the arena is cleared on
+ * that device's legacy default stream and create returns after it finished.
+ * *out receives the context; the caller releases it with mixattn_destroy. */
+int mixattn_create(const mixattn_config* cfg, mixattn_ctx** out);
+
+/* Releases the context's host memory and CUDA events.  The arena is the
+ * caller's.  The caller makes sure no work of the context is still running. */
+int mixattn_destroy(mixattn_ctx* ctx);
+
+/* Empties sequence slot `seq` in every cache: lengths become 0 and its pages
+ * return to the tail of the free FIFO in logical-block order. */
+int mixattn_seq_reset(mixattn_ctx* ctx, int32_t seq);
+
+/* Appends new tokens' K/V to the cache OWNED by `layer` (Section 1: keys and
+ * values of earlier tokens are cached; Section 3: a sliding-window cache keeps
+ * the past s tokens).
+ *   seq_ids  host, n_seqs distinct sequence ids
+ *   n_new    host, tokens per sequence (>= 0), or NULL for one token each
+ *   k, v     device, [sum n_new, n_kv_heads, head_dim], sequences in call order
+ * Full-attention owner: token t of a sequence goes to page
+ * block_table[t / 16], offset t % 16; a free page is taken from the FIFO head
+ * when a sequence first reaches a logical block (sequences in call order,
+ * tokens in position order).  All full-attention owners share one block table
+ * per sequence.  Sliding owner: token t overwrites ring slot t % window.
+ * Errors: NOT_OWNER if the layer reuses another layer's cache, BAD_SEQ,
+ * OUT_OF_PAGES (nothing appended), INVALID_ARG (null, duplicates, length
+ * beyond max_seq_len). */
+int mixattn_append_kv(mixattn_ctx* ctx, int32_t layer, int32_t n_seqs, const int32_t* seq_ids,
+                      const int32_t* n_new, const void* k, const void* v, void* stream);
+
+/* One decode step of `layer` for n_seqs sequences (Section 3).  With n the
+ * number of tokens in the cache the layer reads (its owner's, after this
+ * step's append) the query sits at position n-1 and attends to keys
+ * [0, n) for a standard layer and to the last min(n, window) keys for a
+ * sliding-window layer:  out = softmax(scale * q K^T) V  per query head.
+ *   q, out   device, [n_seqs, n_q_heads, head_dim]
+ * Split-KV flash decoding: partial results go to the context's workspace and a
+ * combine pass writes `out`.  Errors: EMPTY_CONTEXT if a sequence has n == 0
+ * (nothing is written), BAD_SEQ, INVALID_ARG, CUDA. */
+int mixattn_decode(mixattn_ctx* ctx, int32_t layer, int32_t n_seqs, const int32_t* seq_ids,
+                   const void* q, void* out, void* stream);
+
+/* Prompt attention of `layer` for n_seqs sequences that start at position 0
+ * (Section 3; causal as in Section 1).  Query i attends to keys j <= i
+ * (standard) or i - window < j <= i (sliding window); key tiles wholly outside
+ * that band are skipped.
+ *   seq_lens host, prompt length S_b of each sequence (>= 1)
+ *   q, out   device, [sum S_b, n_q_heads, head_dim], sequences back to back
+ *   k, v     device, [sum S_b, n_kv_heads, head_dim]: the K/V computed by the
+ *            layer's owner (a reader is handed its owner's tensors)
+ * If `layer` owns its cache the call also stores K/V as mixattn_append_kv
+ * would (a ring ends up holding the last min(S_b, window) tokens); the
+ * owner's cache for these sequences must be empty, else UNSUPPORTED.  A
+ * reader stores nothing.  Errors: as append_kv and decode. */
+int mixattn_prefill(mixattn_ctx* ctx, int32_t layer, int32_t n_seqs, const int32_t* seq_ids,
+                    const int32_t* seq_lens, const void* q, const void* k, const void* v,
+                    void* out, void* stream);
+
+/* ---- introspection: the surface on which cache indexing is compared bit for bit ---- */
+
+/* Tokens appended so far to the cache `layer` reads, for sequence `seq`. */
+int mixattn_get_len(mixattn_ctx* ctx, int32_t layer, int32_t seq, int32_t* len);
+
+/* Copies the sequence's block table (page id per logical block) to out[0..cap)
+ * (host) and writes the number of blocks in use to *n_blocks (even if > cap). */
+int mixattn_get_block_table(mixattn_ctx* ctx, int32_t seq, int32_t* out, int32_t cap,
+                            int32_t* n_blocks);
+
+/* Number of pages on the free FIFO. */
+int mixattn_get_n_free_pages(mixattn_ctx* ctx, int32_t* n_free);
+
+/* Ring of a sliding-window layer: slot the next token will take (len % window)
+ * and number of valid slots (min(len, window)).  INVALID_ARG for a full layer. */
+int mixattn_get_ring_state(mixattn_ctx* ctx, int32_t layer, int32_t seq, int32_t* next_slot,
+                           int32_t* n_valid);
+
+/* Where token `pos` of `seq` lives in the cache `layer` reads: page id and
+ * offset within the page for a full layer; -1 and ring slot for a sliding
+ * layer.  INVALID_ARG if the token is not stored (any more). */
+int mixattn_locate(mixattn_ctx* ctx, int32_t layer, int32_t seq, int32_t pos, int32_t* page,
+                   int32_t* slot);
+
+/* Copies K and V of token `pos` ([n_kv_heads, head_dim] each, context dtype)
+ * from the device cache to host buffers.  Waits for the whole device first.
+ * The page is looked up in the DEVICE copy of the block table, so the call
+ * also checks that copy.  For tests. */
+int mixattn_debug_read_kv(mixattn_ctx* ctx, int32_t layer, int32_t seq, int32_t pos, void* k_host,
+                          void* v_host);
+
+/* Waits for the device, then reports the status word the kernels share:
+ * 0 = fine, 1 = a bounded wait inside a kernel ran out (results invalid). */
+int mixattn_get_device_status(mixattn_ctx* ctx, int32_t* status);
+
+/* ---- tuning and measurement ---- */
+
+/* Target number of keys per split of the split-KV decode; 0 = automatic.
+ * Results do not depend on it beyond fp32 summation order. */
+int mixattn_set_split_tokens(mixattn_ctx* ctx, int32_t tokens);
+
+/* Kernel classes for mixattn_profile_read. */
+enum {
+  MIXATTN_K_APPEND = 0,
+  MIXATTN_K_DECODE_FULL = 1,    /* split pass of a standard layer        */
+  MIXATTN_K_DECODE_SLIDING = 2, /* split pass of a sliding-window layer  */
+  MIXATTN_K_COMBINE = 3,
+  MIXATTN_K_PREFILL_FULL = 4,
+  MIXATTN_K_PREFILL_SLIDING = 5,
+  MIXATTN_K_COUNT = 6
+};
+
+/* enable != 0: from now on every kernel launch is bracketed by CUDA events on
+ * its stream (costs a little; leave off when timing whole steps) and earlier
+ * records are dropped.  enable == 0: stop recording. */
+int mixattn_profile_enable(mixattn_ctx* ctx, int32_t enable);
+
+/* Waits for the recorded events, then reports launches and summed device
+ * milliseconds of one kernel class since the last enable. */
+int mixattn_profile_read(mixattn_ctx* ctx, int32_t kernel_class, int32_t* launches, float* ms);
+
+/* Kernel launches enqueued by this context since create. */
+int mixattn_get_launch_count(mixattn_ctx* ctx, int64_t* launches);
+
+/* Text for a status code; never NULL. */
+const char* mixattn_strerror(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MIXATTN_H_ */

@@ -1,0 +1,131 @@
+// Shared declarations of the library's translation units (host + device).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "mixattn.h"
+
+namespace mixattn {
+
+constexpr int kPage = 16;          // tokens per page (paged pools and rings alike)
+constexpr int kMaxCallSeqs = 128;  // sequences per kernel launch (metadata travels in kernel params)
+constexpr int kMaxGroupRows = 16;  // query heads of one KV head handled by one work item
+constexpr int kWsExtraChunks = 1024;                        // splits beyond one per sequence
+constexpr int kWsChunks = kMaxCallSeqs + kWsExtraChunks;    // split slots in the workspace
+
+// ---------------------------------------------------------------------------
+// K/V storage format.
+//
+// Paged pools and rings use the same 16-token page.  A page holds, for every KV
+// head g, one contiguous block  [K: 16 tokens x D][V: 16 tokens x D]  so that the
+// decode kernel stages (page, g) with a single bulk copy.  In bf16 mode the 16-byte
+// chunks of a token row are stored XOR-swizzled by (token & 7): the block in HBM is
+// already the bank-conflict-free shared-memory image that ldmatrix wants, and the
+// copy engine needs no tensor map.  fp32 rows are stored unswizzled.
+// ---------------------------------------------------------------------------
+struct KvGeom {
+  int32_t n_kv_heads;
+  int32_t head_dim;
+  int32_t elem_bytes;     // 2 or 4
+  int32_t row_bytes;      // head_dim * elem_bytes
+  int32_t blk_bytes;      // 2 * 16 * row_bytes: K and V of one (page, head)
+  int32_t swizzle;        // 1 in bf16 mode
+  int64_t page_bytes;     // n_kv_heads * blk_bytes
+};
+
+__host__ __device__ inline KvGeom make_geom(int n_kv_heads, int head_dim, int dtype) {
+  KvGeom g;
+  g.n_kv_heads = n_kv_heads;
+  g.head_dim = head_dim;
+  g.elem_bytes = dtype == MIXATTN_BF16 ? 2 : 4;
+  g.row_bytes = head_dim * g.elem_bytes;
+  g.blk_bytes = 2 * kPage * g.row_bytes;
+  g.swizzle = dtype == MIXATTN_BF16 ? 1 : 0;
+  g.page_bytes = (int64_t)n_kv_heads * g.blk_bytes;
+  return g;
+}
+
+// Byte offset, inside a pool, of 16-byte chunk `chunk` of token slot `tok` (0..15) of
+// page `page`, KV head `g`, which = 0 (K) or 1 (V).
+__host__ __device__ inline int64_t kv_chunk_offset(const KvGeom& ge, int64_t page, int g, int which,
+                                                   int tok, int chunk) {
+  int c = ge.swizzle ? (chunk ^ (tok & 7)) : chunk;
+  return page * ge.page_bytes + (int64_t)g * ge.blk_bytes + (int64_t)which * kPage * ge.row_bytes +
+         (int64_t)tok * ge.row_bytes + (int64_t)c * 16;
+}
+
+// ---------------------------------------------------------------------------
+// kernel parameter blocks (passed by value: no per-call metadata copy)
+// ---------------------------------------------------------------------------
+struct AppendEntry {
+  int32_t seq;        // sequence slot
+  int32_t start_pos;  // position of the first new token
+  int32_t n_new;      // tokens appended
+  int32_t src_row0;   // row of the first new token in k / v
+  int32_t page_hint;  // n_new == 1 on a paged pool: page id resolved by the host; else -1
+  int32_t tbl_idx;    // >= 0: device block-table entry this call must set to page_hint
+};
+
+struct AppendParams {
+  const void* k;
+  const void* v;
+  char* pool;            // paged pool or ring storage of the owner
+  int32_t* table;        // device block tables [max_seqs][table_stride]
+  int32_t table_stride;
+  int32_t is_ring;
+  int32_t window;
+  int32_t ring_pages;    // pages per sequence in a ring
+  KvGeom geom;
+  int32_t n_entries;
+  AppendEntry e[kMaxCallSeqs];
+};
+
+struct DecodeParams {
+  const void* q;          // [n_seqs, Hq, D]
+  void* out;              // [n_seqs, Hq, D]
+  const char* pool;       // storage of the cache the layer reads
+  const int32_t* table;   // device block tables, or nullptr for a ring
+  int32_t table_stride;
+  int32_t ring_pages;
+  KvGeom geom;
+  int32_t n_q_heads;
+  int32_t group;          // query heads per KV head
+  int32_t head_chunks;    // ceil(group / 16)
+  float scale_log2e;      // softmax scale * log2(e)
+  float* part_o;          // [chunks, Hq, D] unnormalised partial outputs
+  float2* part_ml;        // [chunks, Hq] running max (log2 units) and sum
+  int32_t* status;        // device error word (0 = fine)
+  int32_t n_seqs;
+  int32_t total_items;    // chunks * Hkv * head_chunks
+  int32_t seq_id[kMaxCallSeqs];
+  int32_t n_eff[kMaxCallSeqs];           // keys attended: min(len, window) or len
+  int32_t chunk_len[kMaxCallSeqs];       // keys per split of this sequence (multiple of 16)
+  int32_t chunk_base[kMaxCallSeqs + 1];  // first split index of each sequence
+};
+
+struct PrefillParams {
+  const void* q;
+  const void* k;
+  const void* v;
+  void* out;
+  int32_t n_q_heads, n_kv_heads, head_dim;
+  int32_t window;        // 0 = standard layer
+  float scale_log2e;
+  int32_t n_seqs;
+  int32_t* status;
+  int32_t row0[kMaxCallSeqs + 1];  // first row of each sequence in the packed tensors
+};
+
+// device status codes written to the status word
+enum { kDevOk = 0, kDevWaitTimeout = 1 };
+
+// launchers (each returns the cudaError_t of its launch)
+cudaError_t launch_append(const AppendParams& p, int max_n_new, cudaStream_t st);
+cudaError_t prepare_decode_bf16();
+cudaError_t launch_decode_split_bf16(const DecodeParams& p, int sm_count, cudaStream_t st);
+cudaError_t launch_decode_split_f32(const DecodeParams& p, cudaStream_t st);
+cudaError_t launch_decode_combine(const DecodeParams& p, int dtype, cudaStream_t st);
+cudaError_t launch_prefill_simple(const PrefillParams& p, int dtype, int max_len, cudaStream_t st);
+
+}  // namespace mixattn
