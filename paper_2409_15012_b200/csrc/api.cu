@@ -1,0 +1,637 @@
+// The C ABI (include/mixattn.h): argument validation, host bookkeeping, arena carving and
+// kernel launches.  Everything that can fail is checked on the host before any launch.
+#include <math.h>
+#include <string.h>
+
+#include <new>
+#include <vector>
+
+#include "cache_manager.hpp"
+#include "internal.h"
+
+using namespace mixattn;
+
+namespace {
+
+constexpr size_t kAlign = 256;
+constexpr int kItemsPerSm = 4;       // automatic split: work items per SM aimed for
+constexpr int kMinSplitTokens = 256;
+
+inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
+
+struct ArenaPlan {
+  std::vector<size_t> owner_off;  // per owner slot
+  std::vector<size_t> owner_bytes;
+  size_t table_off = 0, table_bytes = 0;
+  size_t part_o_off = 0, part_ml_off = 0, status_off = 0;
+  size_t cache_bytes = 0, total = 0;
+};
+
+int ring_pages_of(int window) { return (window + kPage - 1) / kPage; }
+
+ArenaPlan plan_arena(const CacheManager& cm, const mixattn_config& cfg) {
+  ArenaPlan pl;
+  KvGeom ge = make_geom(cfg.n_kv_heads, cfg.head_dim, cfg.dtype);
+  size_t off = 0;
+  for (int o : cm.owners()) {
+    const LayerInfo& li = cm.layer(o);
+    size_t bytes = li.kind == MIXATTN_FULL
+                       ? (size_t)cfg.n_pages * ge.page_bytes
+                       : (size_t)cfg.max_seqs * ring_pages_of(li.window) * ge.page_bytes;
+    pl.owner_off.push_back(off);
+    pl.owner_bytes.push_back(bytes);
+    pl.cache_bytes += bytes;
+    off += align_up(bytes);
+  }
+  pl.table_off = off;
+  pl.table_bytes = (size_t)cm.max_seqs() * cm.max_blocks() * sizeof(int32_t);
+  off += align_up(pl.table_bytes);
+  pl.part_o_off = off;
+  off += align_up((size_t)kWsChunks * cfg.n_q_heads * cfg.head_dim * sizeof(float));
+  pl.part_ml_off = off;
+  off += align_up((size_t)kWsChunks * cfg.n_q_heads * sizeof(float2));
+  pl.status_off = off;
+  off += kAlign;
+  pl.total = off;
+  return pl;
+}
+
+struct ProfileRecord {
+  int cls;
+  cudaEvent_t start, stop;
+};
+
+}  // namespace
+
+struct mixattn_ctx {
+  CacheManager cm;
+  mixattn_config cfg;  // layers / free_order pointers are not kept
+  KvGeom geom;
+  ArenaPlan plan;
+  char* arena = nullptr;
+  bool host_only = true;
+  int device = -1;
+  int sm_count = 148;
+  float scale = 0.f;
+  int32_t split_tokens = 0;
+  int64_t launches = 0;
+  bool profiling = false;
+  std::vector<ProfileRecord> records;
+  std::vector<cudaEvent_t> event_pool;
+  bool sticky_cuda_error = false;
+
+  char* owner_storage(int layer) const { return arena + plan.owner_off[cm.layer(layer).owner_slot]; }
+  int32_t* dev_table() const { return reinterpret_cast<int32_t*>(arena + plan.table_off); }
+  int32_t* dev_status() const { return reinterpret_cast<int32_t*>(arena + plan.status_off); }
+};
+
+namespace {
+
+struct DeviceGuard {
+  int prev = -1;
+  bool ok = true;
+  explicit DeviceGuard(int dev) {
+    if (cudaGetDevice(&prev) != cudaSuccess) { ok = false; return; }
+    if (prev != dev && cudaSetDevice(dev) != cudaSuccess) ok = false;
+    target = dev;
+  }
+  ~DeviceGuard() {
+    if (ok && prev >= 0 && prev != target) cudaSetDevice(prev);
+  }
+  int target = -1;
+};
+
+cudaEvent_t take_event(mixattn_ctx* c) {
+  if (!c->event_pool.empty()) {
+    cudaEvent_t e = c->event_pool.back();
+    c->event_pool.pop_back();
+    return e;
+  }
+  cudaEvent_t e = nullptr;
+  cudaEventCreate(&e);
+  return e;
+}
+
+// Brackets one launch with events when profiling is on.
+template <typename F>
+cudaError_t launch_recorded(mixattn_ctx* c, int cls, cudaStream_t st, F&& f) {
+  ProfileRecord rec{cls, nullptr, nullptr};
+  if (c->profiling) {
+    rec.start = take_event(c);
+    rec.stop = take_event(c);
+    if (rec.start) cudaEventRecord(rec.start, st);
+  }
+  cudaError_t e = f();
+  if (c->profiling) {
+    if (rec.stop) cudaEventRecord(rec.stop, st);
+    c->records.push_back(rec);
+  }
+  if (e == cudaSuccess) ++c->launches;
+  else c->sticky_cuda_error = true;
+  return e;
+}
+
+int validate_config(const mixattn_config* cfg, CacheManager* cm) {
+  if (cfg == nullptr) return MIXATTN_ERR_INVALID_ARG;
+  int rc = cm->init(*cfg);
+  if (rc != MIXATTN_OK) return rc;
+  if (cfg->softmax_scale < 0.f || !isfinite(cfg->softmax_scale)) return MIXATTN_ERR_INVALID_ARG;
+  if (cm->n_full_owners() > 0 && cfg->n_pages < 1) return MIXATTN_ERR_INVALID_ARG;
+  return MIXATTN_OK;
+}
+
+// Enqueues the device side of an append the host bookkeeping has already applied.
+int enqueue_append(mixattn_ctx* c, int layer, int n_seqs, const int32_t* seq_ids,
+                   const int32_t* n_new, const std::vector<int32_t>& start_pos,
+                   const std::vector<PageGrant>& grants, const void* k, const void* v,
+                   cudaStream_t st) {
+  const LayerInfo& li = c->cm.layer(layer);
+  const bool ring = li.kind == MIXATTN_SLIDING;
+  bool single = true;
+  for (int i = 0; i < n_seqs; ++i) single = single && (n_new == nullptr || n_new[i] == 1);
+  const int stride = c->cm.max_blocks();
+  if (!ring && !single && !grants.empty()) {
+    // bulk append: push each sequence's new table entries, then let the kernel read the table
+    size_t a = 0;
+    while (a < grants.size()) {
+      size_t b = a;
+      while (b + 1 < grants.size() && grants[b + 1].seq == grants[a].seq) ++b;
+      const int32_t* src = c->cm.table_row(grants[a].seq) + grants[a].block;
+      int32_t* dst = c->dev_table() + (size_t)grants[a].seq * stride + grants[a].block;
+      if (cudaMemcpyAsync(dst, src, (b - a + 1) * sizeof(int32_t), cudaMemcpyHostToDevice, st) !=
+          cudaSuccess) {
+        c->sticky_cuda_error = true;
+        return MIXATTN_ERR_CUDA;
+      }
+      a = b + 1;
+    }
+  }
+  AppendParams p;
+  p.k = k;
+  p.v = v;
+  p.pool = c->owner_storage(layer);
+  p.table = c->dev_table();
+  p.table_stride = stride;
+  p.is_ring = ring;
+  p.window = ring ? li.window : 0;
+  p.ring_pages = ring ? ring_pages_of(li.window) : 0;
+  p.geom = c->geom;
+  int row = 0;
+  size_t gi = 0;
+  for (int i0 = 0; i0 < n_seqs; i0 += kMaxCallSeqs) {
+    const int nb = n_seqs - i0 < kMaxCallSeqs ? n_seqs - i0 : kMaxCallSeqs;
+    int max_new = 0;
+    for (int j = 0; j < nb; ++j) {
+      const int i = i0 + j;
+      AppendEntry& e = p.e[j];
+      e.seq = seq_ids[i];
+      e.start_pos = start_pos[i];
+      e.n_new = n_new ? n_new[i] : 1;
+      e.src_row0 = row;
+      e.page_hint = -1;
+      e.tbl_idx = -1;
+      if (!ring && single) {
+        e.page_hint = c->cm.table_row(e.seq)[e.start_pos / kPage];
+        // grants are in call order: at most one per sequence in single-token mode
+        if (gi < grants.size() && grants[gi].seq == e.seq) {
+          e.tbl_idx = e.seq * stride + grants[gi].block;
+          ++gi;
+        }
+      }
+      row += e.n_new;
+      if (e.n_new > max_new) max_new = e.n_new;
+    }
+    p.n_entries = nb;
+    if (max_new == 0) {
+      bool any_tbl = false;
+      for (int j = 0; j < nb; ++j) any_tbl = any_tbl || p.e[j].tbl_idx >= 0;
+      if (!any_tbl) continue;
+    }
+    cudaError_t e = launch_recorded(c, MIXATTN_K_APPEND, st, [&] { return launch_append(p, max_new, st); });
+    if (e != cudaSuccess) return MIXATTN_ERR_CUDA;
+  }
+  return MIXATTN_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int mixattn_arena_bytes(const mixattn_config* cfg, size_t* out_bytes) {
+  if (out_bytes == nullptr) return MIXATTN_ERR_INVALID_ARG;
+  CacheManager cm;
+  int rc = validate_config(cfg, &cm);
+  if (rc != MIXATTN_OK) return rc;
+  *out_bytes = plan_arena(cm, *cfg).total;
+  return MIXATTN_OK;
+}
+
+int mixattn_cache_bytes(const mixattn_config* cfg, size_t* out_bytes) {
+  if (out_bytes == nullptr) return MIXATTN_ERR_INVALID_ARG;
+  CacheManager cm;
+  int rc = validate_config(cfg, &cm);
+  if (rc != MIXATTN_OK) return rc;
+  *out_bytes = plan_arena(cm, *cfg).cache_bytes;
+  return MIXATTN_OK;
+}
+
+int mixattn_create(const mixattn_config* cfg, mixattn_ctx** out) {
+  if (out == nullptr) return MIXATTN_ERR_INVALID_ARG;
+  *out = nullptr;
+  mixattn_ctx* c = new (std::nothrow) mixattn_ctx();
+  if (c == nullptr) return MIXATTN_ERR_INVALID_ARG;
+  int rc = validate_config(cfg, &c->cm);
+  if (rc != MIXATTN_OK) { delete c; return rc; }
+  c->cfg = *cfg;
+  c->cfg.layers = nullptr;
+  c->cfg.free_order = nullptr;
+  c->geom = make_geom(cfg->n_kv_heads, cfg->head_dim, cfg->dtype);
+  c->plan = plan_arena(c->cm, *cfg);
+  c->scale = cfg->softmax_scale > 0.f ? cfg->softmax_scale : 1.0f / sqrtf((float)cfg->head_dim);
+  c->host_only = cfg->device < 0;
+  c->device = cfg->device;
+  if (!c->host_only) {
+    if (cfg->arena == nullptr || cfg->arena_bytes < c->plan.total ||
+        (reinterpret_cast<uintptr_t>(cfg->arena) % kAlign) != 0) {
+      delete c;
+      return MIXATTN_ERR_INVALID_ARG;
+    }
+    c->arena = static_cast<char*>(cfg->arena);
+    DeviceGuard g(c->device);
+    cudaDeviceProp prop;
+    if (!g.ok || cudaGetDeviceProperties(&prop, c->device) != cudaSuccess) { delete c; return MIXATTN_ERR_CUDA; }
+    c->sm_count = prop.multiProcessorCount;
+    if (prepare_decode_bf16() != cudaSuccess) { delete c; return MIXATTN_ERR_CUDA; }
+    if (cudaMemsetAsync(c->arena, 0, c->plan.total, 0) != cudaSuccess ||
+        cudaStreamSynchronize(0) != cudaSuccess) {
+      delete c;
+      return MIXATTN_ERR_CUDA;
+    }
+  }
+  *out = c;
+  return MIXATTN_OK;
+}
+
+int mixattn_destroy(mixattn_ctx* c) {
+  if (c == nullptr) return MIXATTN_ERR_INVALID_ARG;
+  if (!c->host_only) {
+    DeviceGuard g(c->device);
+    for (auto& r : c->records) {
+      if (r.start) cudaEventDestroy(r.start);
+      if (r.stop) cudaEventDestroy(r.stop);
+    }
+    for (auto e : c->event_pool) cudaEventDestroy(e);
+  }
+  delete c;
+  return MIXATTN_OK;
+}
+
+int mixattn_seq_reset(mixattn_ctx* c, int32_t seq) {
+  if (c == nullptr) return MIXATTN_ERR_INVALID_ARG;
+  if (!c->cm.valid_seq(seq)) return MIXATTN_ERR_BAD_SEQ;
+  c->cm.seq_reset(seq);
+  return MIXATTN_OK;
+}
+
+int mixattn_append_kv(mixattn_ctx* c, int32_t layer, int32_t n_seqs, const int32_t* seq_ids,
+                      const int32_t* n_new, const void* k, const void* v, void* stream) {
+  if (c == nullptr) return MIXATTN_ERR_INVALID_ARG;
+  int rc = c->cm.check_append(layer, n_seqs, seq_ids, n_new);
+  if (rc != MIXATTN_OK) return rc;
+  int64_t total = 0;
+  for (int i = 0; i < n_seqs; ++i) total += n_new ? n_new[i] : 1;
+  if (total > INT32_MAX) return MIXATTN_ERR_INVALID_ARG;
+  if (!c->host_only) {
+    if (total > 0 && (k == nullptr || v == nullptr)) return MIXATTN_ERR_INVALID_ARG;
+    if (c->sticky_cuda_error) return MIXATTN_ERR_CUDA;
+  }
+  std::vector<int32_t> start(n_seqs);
+  for (int i = 0; i < n_seqs; ++i) start[i] = c->cm.len(layer, seq_ids[i]);
+  std::vector<PageGrant> grants;
+  c->cm.apply_append(layer, n_seqs, seq_ids, n_new, &grants);
+  if (c->host_only) return MIXATTN_OK;
+  DeviceGuard g(c->device);
+  if (!g.ok) return MIXATTN_ERR_CUDA;
+  return enqueue_append(c, layer, n_seqs, seq_ids, n_new, start, grants, k, v,
+                        static_cast<cudaStream_t>(stream));
+}
+
+int mixattn_decode(mixattn_ctx* c, int32_t layer, int32_t n_seqs, const int32_t* seq_ids,
+                   const void* q, void* out, void* stream) {
+  if (c == nullptr || !c->cm.valid_layer(layer) || n_seqs < 0) return MIXATTN_ERR_INVALID_ARG;
+  if (n_seqs > 0 && (seq_ids == nullptr || q == nullptr || out == nullptr)) return MIXATTN_ERR_INVALID_ARG;
+  for (int i = 0; i < n_seqs; ++i) {
+    if (!c->cm.valid_seq(seq_ids[i])) return MIXATTN_ERR_BAD_SEQ;
+  }
+  for (int i = 0; i < n_seqs; ++i) {
+    if (c->cm.len(layer, seq_ids[i]) < 1) return MIXATTN_ERR_EMPTY_CONTEXT;
+  }
+  if (c->host_only || c->sticky_cuda_error) return MIXATTN_ERR_CUDA;
+  if (n_seqs == 0) return MIXATTN_OK;
+  DeviceGuard g(c->device);
+  if (!g.ok) return MIXATTN_ERR_CUDA;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+
+  const LayerInfo& li = c->cm.layer(layer);
+  const bool ring = li.kind == MIXATTN_SLIDING;
+  const int Hq = c->cfg.n_q_heads, Hkv = c->cfg.n_kv_heads, D = c->cfg.head_dim;
+  const size_t esz = c->geom.elem_bytes;
+
+  DecodeParams p;
+  p.pool = c->owner_storage(layer);
+  p.table = ring ? nullptr : c->dev_table();
+  p.table_stride = c->cm.max_blocks();
+  p.ring_pages = ring ? ring_pages_of(li.window) : 0;
+  p.geom = c->geom;
+  p.n_q_heads = Hq;
+  p.group = Hq / Hkv;
+  p.head_chunks = (p.group + kMaxGroupRows - 1) / kMaxGroupRows;
+  p.scale_log2e = c->scale * 1.4426950408889634f;
+  p.part_o = reinterpret_cast<float*>(c->arena + c->plan.part_o_off);
+  p.part_ml = reinterpret_cast<float2*>(c->arena + c->plan.part_ml_off);
+  p.status = c->dev_status();
+
+  for (int i0 = 0; i0 < n_seqs; i0 += kMaxCallSeqs) {
+    const int nb = n_seqs - i0 < kMaxCallSeqs ? n_seqs - i0 : kMaxCallSeqs;
+    int64_t total = 0;
+    for (int j = 0; j < nb; ++j) {
+      p.seq_id[j] = seq_ids[i0 + j];
+      p.n_eff[j] = c->cm.n_attended(layer, p.seq_id[j]);
+      total += p.n_eff[j];
+    }
+    // split length: aim at kItemsPerSm work items per SM, never more splits than the workspace holds
+    int64_t T;
+    if (c->split_tokens > 0) {
+      T = (c->split_tokens + kPage - 1) / kPage * kPage;
+    } else {
+      int64_t chunks_target = (int64_t)c->sm_count * kItemsPerSm / ((int64_t)Hkv * p.head_chunks);
+      if (chunks_target < 1) chunks_target = 1;
+      T = (total + chunks_target - 1) / chunks_target;
+      T = (T + 63) / 64 * 64;
+      if (T < kMinSplitTokens) T = kMinSplitTokens;
+    }
+    int64_t t_min = (total + kWsExtraChunks - 1) / kWsExtraChunks;
+    t_min = (t_min + kPage - 1) / kPage * kPage;
+    if (T < t_min) T = t_min;
+    int base = 0;
+    bool any_split = false;
+    for (int j = 0; j < nb; ++j) {
+      const int64_t n = p.n_eff[j];
+      const int64_t nc = (n + T - 1) / T;
+      int64_t len = (n + nc - 1) / nc;
+      len = (len + kPage - 1) / kPage * kPage;
+      p.chunk_base[j] = base;
+      p.chunk_len[j] = (int32_t)len;
+      base += (int)nc;
+      any_split = any_split || nc > 1;
+    }
+    p.chunk_base[nb] = base;
+    p.n_seqs = nb;
+    p.total_items = base * Hkv * p.head_chunks;
+    p.q = static_cast<const char*>(q) + (size_t)i0 * Hq * D * esz;
+    p.out = static_cast<char*>(out) + (size_t)i0 * Hq * D * esz;
+    const int cls = ring ? MIXATTN_K_DECODE_SLIDING : MIXATTN_K_DECODE_FULL;
+    cudaError_t e = launch_recorded(c, cls, st, [&] {
+      return c->cfg.dtype == MIXATTN_BF16 ? launch_decode_split_bf16(p, c->sm_count, st)
+                                          : launch_decode_split_f32(p, st);
+    });
+    if (e != cudaSuccess) return MIXATTN_ERR_CUDA;
+    if (any_split) {
+      e = launch_recorded(c, MIXATTN_K_COMBINE, st,
+                          [&] { return launch_decode_combine(p, c->cfg.dtype, st); });
+      if (e != cudaSuccess) return MIXATTN_ERR_CUDA;
+    }
+  }
+  return MIXATTN_OK;
+}
+
+int mixattn_prefill(mixattn_ctx* c, int32_t layer, int32_t n_seqs, const int32_t* seq_ids,
+                    const int32_t* seq_lens, const void* q, const void* k, const void* v,
+                    void* out, void* stream) {
+  if (c == nullptr || !c->cm.valid_layer(layer) || n_seqs < 0) return MIXATTN_ERR_INVALID_ARG;
+  if (n_seqs > 0 && (seq_ids == nullptr || seq_lens == nullptr)) return MIXATTN_ERR_INVALID_ARG;
+  const LayerInfo& li = c->cm.layer(layer);
+  const bool owner = li.owner == layer;
+  int64_t total = 0;
+  int max_len = 0;
+  {
+    std::vector<char> seen(c->cm.max_seqs(), 0);
+    for (int i = 0; i < n_seqs; ++i) {
+      if (!c->cm.valid_seq(seq_ids[i])) return MIXATTN_ERR_BAD_SEQ;
+      if (seen[seq_ids[i]]) return MIXATTN_ERR_INVALID_ARG;
+      seen[seq_ids[i]] = 1;
+      if (seq_lens[i] < 1) return MIXATTN_ERR_INVALID_ARG;
+      total += seq_lens[i];
+      if (seq_lens[i] > max_len) max_len = seq_lens[i];
+    }
+  }
+  if (total > INT32_MAX) return MIXATTN_ERR_INVALID_ARG;
+  if (owner) {
+    for (int i = 0; i < n_seqs; ++i)
+      if (c->cm.len(layer, seq_ids[i]) != 0) return MIXATTN_ERR_UNSUPPORTED;
+    int rc = c->cm.check_append(layer, n_seqs, seq_ids, seq_lens);
+    if (rc != MIXATTN_OK) return rc;
+  }
+  if (c->host_only || c->sticky_cuda_error) return MIXATTN_ERR_CUDA;
+  if (n_seqs == 0) return MIXATTN_OK;
+  if (q == nullptr || k == nullptr || v == nullptr || out == nullptr) return MIXATTN_ERR_INVALID_ARG;
+  DeviceGuard g(c->device);
+  if (!g.ok) return MIXATTN_ERR_CUDA;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (owner) {
+    std::vector<int32_t> start(n_seqs, 0);
+    std::vector<PageGrant> grants;
+    c->cm.apply_append(layer, n_seqs, seq_ids, seq_lens, &grants);
+    int rc = enqueue_append(c, layer, n_seqs, seq_ids, seq_lens, start, grants, k, v, st);
+    if (rc != MIXATTN_OK) return rc;
+  }
+  const int Hq = c->cfg.n_q_heads, Hkv = c->cfg.n_kv_heads, D = c->cfg.head_dim;
+  const size_t esz = c->geom.elem_bytes;
+  PrefillParams p;
+  p.n_q_heads = Hq;
+  p.n_kv_heads = Hkv;
+  p.head_dim = D;
+  p.window = li.kind == MIXATTN_SLIDING ? li.window : 0;
+  p.scale_log2e = c->scale * 1.4426950408889634f;
+  p.status = c->dev_status();
+  int64_t row = 0;
+  for (int i0 = 0; i0 < n_seqs; i0 += kMaxCallSeqs) {
+    const int nb = n_seqs - i0 < kMaxCallSeqs ? n_seqs - i0 : kMaxCallSeqs;
+    int r = 0, mlen = 0;
+    for (int j = 0; j < nb; ++j) {
+      p.row0[j] = r;
+      r += seq_lens[i0 + j];
+      if (seq_lens[i0 + j] > mlen) mlen = seq_lens[i0 + j];
+    }
+    p.row0[nb] = r;
+    p.n_seqs = nb;
+    p.q = static_cast<const char*>(q) + (size_t)row * Hq * D * esz;
+    p.out = static_cast<char*>(out) + (size_t)row * Hq * D * esz;
+    p.k = static_cast<const char*>(k) + (size_t)row * Hkv * D * esz;
+    p.v = static_cast<const char*>(v) + (size_t)row * Hkv * D * esz;
+    row += r;
+    const int cls = p.window ? MIXATTN_K_PREFILL_SLIDING : MIXATTN_K_PREFILL_FULL;
+    cudaError_t e = launch_recorded(c, cls, st, [&] {
+      return launch_prefill_simple(p, c->cfg.dtype, mlen, st);
+    });
+    if (e != cudaSuccess) return MIXATTN_ERR_CUDA;
+  }
+  return MIXATTN_OK;
+}
+
+int mixattn_get_len(mixattn_ctx* c, int32_t layer, int32_t seq, int32_t* len) {
+  if (c == nullptr || len == nullptr || !c->cm.valid_layer(layer)) return MIXATTN_ERR_INVALID_ARG;
+  if (!c->cm.valid_seq(seq)) return MIXATTN_ERR_BAD_SEQ;
+  *len = c->cm.len(layer, seq);
+  return MIXATTN_OK;
+}
+
+int mixattn_get_block_table(mixattn_ctx* c, int32_t seq, int32_t* out, int32_t cap, int32_t* n_blocks) {
+  if (c == nullptr || n_blocks == nullptr || cap < 0 || (cap > 0 && out == nullptr))
+    return MIXATTN_ERR_INVALID_ARG;
+  if (!c->cm.valid_seq(seq)) return MIXATTN_ERR_BAD_SEQ;
+  const int n = c->cm.n_blocks(seq);
+  *n_blocks = n;
+  const int m = n < cap ? n : cap;
+  if (m > 0) memcpy(out, c->cm.table_row(seq), (size_t)m * sizeof(int32_t));
+  return MIXATTN_OK;
+}
+
+int mixattn_get_n_free_pages(mixattn_ctx* c, int32_t* n_free) {
+  if (c == nullptr || n_free == nullptr) return MIXATTN_ERR_INVALID_ARG;
+  *n_free = c->cm.n_free();
+  return MIXATTN_OK;
+}
+
+int mixattn_get_ring_state(mixattn_ctx* c, int32_t layer, int32_t seq, int32_t* next_slot, int32_t* n_valid) {
+  if (c == nullptr || next_slot == nullptr || n_valid == nullptr || !c->cm.valid_layer(layer))
+    return MIXATTN_ERR_INVALID_ARG;
+  if (!c->cm.valid_seq(seq)) return MIXATTN_ERR_BAD_SEQ;
+  const LayerInfo& li = c->cm.layer(layer);
+  if (li.kind != MIXATTN_SLIDING) return MIXATTN_ERR_INVALID_ARG;
+  const int32_t n = c->cm.len(layer, seq);
+  *next_slot = n % li.window;
+  *n_valid = n < li.window ? n : li.window;
+  return MIXATTN_OK;
+}
+
+int mixattn_locate(mixattn_ctx* c, int32_t layer, int32_t seq, int32_t pos, int32_t* page, int32_t* slot) {
+  if (c == nullptr || page == nullptr || slot == nullptr || !c->cm.valid_layer(layer))
+    return MIXATTN_ERR_INVALID_ARG;
+  if (!c->cm.valid_seq(seq)) return MIXATTN_ERR_BAD_SEQ;
+  return c->cm.locate(layer, seq, pos, page, slot) ? MIXATTN_OK : MIXATTN_ERR_INVALID_ARG;
+}
+
+int mixattn_debug_read_kv(mixattn_ctx* c, int32_t layer, int32_t seq, int32_t pos, void* k_host, void* v_host) {
+  if (c == nullptr || k_host == nullptr || v_host == nullptr || !c->cm.valid_layer(layer))
+    return MIXATTN_ERR_INVALID_ARG;
+  if (!c->cm.valid_seq(seq)) return MIXATTN_ERR_BAD_SEQ;
+  int32_t page, slot;
+  if (!c->cm.locate(layer, seq, pos, &page, &slot)) return MIXATTN_ERR_INVALID_ARG;
+  if (c->host_only) return MIXATTN_ERR_CUDA;
+  DeviceGuard g(c->device);
+  if (!g.ok || cudaDeviceSynchronize() != cudaSuccess) return MIXATTN_ERR_CUDA;
+  const LayerInfo& li = c->cm.layer(layer);
+  const KvGeom& ge = c->geom;
+  int64_t phys;
+  if (li.kind == MIXATTN_FULL) {
+    int32_t dev_page = -1;
+    if (cudaMemcpy(&dev_page, c->dev_table() + (size_t)seq * c->cm.max_blocks() + pos / kPage,
+                   sizeof(int32_t), cudaMemcpyDeviceToHost) != cudaSuccess)
+      return MIXATTN_ERR_CUDA;
+    phys = dev_page;
+  } else {
+    phys = (int64_t)seq * ring_pages_of(li.window) + slot / kPage;
+    slot = slot % kPage;
+  }
+  const char* pool = c->owner_storage(layer);
+  std::vector<char> row(ge.row_bytes);
+  const int chunks = ge.row_bytes / 16;
+  for (int which = 0; which < 2; ++which) {
+    char* dst = static_cast<char*>(which ? v_host : k_host);
+    for (int gh = 0; gh < ge.n_kv_heads; ++gh) {
+      // start of the token row; its 16-byte chunks are permuted in bf16 mode
+      const char* src = pool + phys * ge.page_bytes + (int64_t)gh * ge.blk_bytes +
+                        (int64_t)which * kPage * ge.row_bytes + (int64_t)slot * ge.row_bytes;
+      if (cudaMemcpy(row.data(), src, ge.row_bytes, cudaMemcpyDeviceToHost) != cudaSuccess)
+        return MIXATTN_ERR_CUDA;
+      for (int ch = 0; ch < chunks; ++ch) {
+        const int phys_ch = ge.swizzle ? (ch ^ (slot & 7)) : ch;
+        memcpy(dst + (size_t)gh * ge.row_bytes + ch * 16, row.data() + phys_ch * 16, 16);
+      }
+    }
+  }
+  return MIXATTN_OK;
+}
+
+int mixattn_get_device_status(mixattn_ctx* c, int32_t* status) {
+  if (c == nullptr || status == nullptr) return MIXATTN_ERR_INVALID_ARG;
+  if (c->host_only) return MIXATTN_ERR_CUDA;
+  DeviceGuard g(c->device);
+  if (!g.ok || cudaDeviceSynchronize() != cudaSuccess) return MIXATTN_ERR_CUDA;
+  if (cudaMemcpy(status, c->dev_status(), sizeof(int32_t), cudaMemcpyDeviceToHost) != cudaSuccess)
+    return MIXATTN_ERR_CUDA;
+  return MIXATTN_OK;
+}
+
+int mixattn_set_split_tokens(mixattn_ctx* c, int32_t tokens) {
+  if (c == nullptr || tokens < 0) return MIXATTN_ERR_INVALID_ARG;
+  c->split_tokens = tokens;
+  return MIXATTN_OK;
+}
+
+int mixattn_profile_enable(mixattn_ctx* c, int32_t enable) {
+  if (c == nullptr) return MIXATTN_ERR_INVALID_ARG;
+  if (c->host_only) return MIXATTN_ERR_CUDA;
+  for (auto& r : c->records) {
+    if (r.start) c->event_pool.push_back(r.start);
+    if (r.stop) c->event_pool.push_back(r.stop);
+  }
+  c->records.clear();
+  c->profiling = enable != 0;
+  return MIXATTN_OK;
+}
+
+int mixattn_profile_read(mixattn_ctx* c, int32_t cls, int32_t* launches, float* ms) {
+  if (c == nullptr || launches == nullptr || ms == nullptr || cls < 0 || cls >= MIXATTN_K_COUNT)
+    return MIXATTN_ERR_INVALID_ARG;
+  if (c->host_only) return MIXATTN_ERR_CUDA;
+  DeviceGuard g(c->device);
+  if (!g.ok) return MIXATTN_ERR_CUDA;
+  int n = 0;
+  float total = 0.f;
+  for (auto& r : c->records) {
+    if (r.cls != cls || !r.start || !r.stop) continue;
+    if (cudaEventSynchronize(r.stop) != cudaSuccess) return MIXATTN_ERR_CUDA;
+    float t = 0.f;
+    if (cudaEventElapsedTime(&t, r.start, r.stop) != cudaSuccess) return MIXATTN_ERR_CUDA;
+    total += t;
+    ++n;
+  }
+  *launches = n;
+  *ms = total;
+  return MIXATTN_OK;
+}
+
+int mixattn_get_launch_count(mixattn_ctx* c, int64_t* launches) {
+  if (c == nullptr || launches == nullptr) return MIXATTN_ERR_INVALID_ARG;
+  *launches = c->launches;
+  return MIXATTN_OK;
+}
+
+const char* mixattn_strerror(int code) {
+  switch (code) {
+    case MIXATTN_OK: return "ok";
+    case MIXATTN_ERR_INVALID_ARG: return "invalid argument";
+    case MIXATTN_ERR_INVALID_LAYOUT: return "invalid layer layout";
+    case MIXATTN_ERR_NOT_OWNER: return "layer reuses another layer's KV cache and takes no K/V";
+    case MIXATTN_ERR_OUT_OF_PAGES: return "not enough free pages";
+    case MIXATTN_ERR_EMPTY_CONTEXT: return "sequence has no cached token";
+    case MIXATTN_ERR_BAD_SEQ: return "sequence id out of range";
+    case MIXATTN_ERR_UNSUPPORTED: return "unsupported request";
+    case MIXATTN_ERR_CUDA: return "CUDA error or host-only context";
+    default: return "unknown status";
+  }
+}
+
+}  // extern "C"
