@@ -1,0 +1,445 @@
+"""Benchmark of the MixAttention decode path (and a prompt-pass figure beside it).
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--workload NAME]
+
+A step is one decode step of the whole model: for each of the 24 layers, append
+the new token's K/V if the layer owns a cache, then attend (split pass +
+combine).  Workload: the mid-decode configuration (batch 32, context 32768,
+window 1024, 32/8 heads of 128, bf16) with seeded synthetic inputs.
+
+Prints ONE JSON line (rank 0).  `value` is decode-attention GB/s: KV bytes each
+layer reads (a shared cache counted once per reading layer) / device time, with
+all inputs resident in HBM.  `e2e` is the same metric with each step's inputs
+copied from pinned host memory and the step's outputs read back, inside the
+timed region.  With --gpus N > 1 every rank runs an independent replica (the
+path has no exchange step); the value is the sum over ranks / max time.
+
+--impl reference times the CPU checker (oracle/) on the host cores on a
+bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+
+from synth import configs as cf
+from synth import inputs as si
+
+METRIC = "decode attention HBM GB/s (% of peak) & tokens/s; prefill TFLOP/s (% bf16 peak)"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel from an
+# ncu capture (profiles/); None until captured for the current kernel
+DECODE_FULL_TRAFFIC_BYTES = None
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        d["_source"] = "measured"
+        return d
+    d = dict(FALLBACK_PEAKS)
+    d["_source"] = "fallback"
+    return d
+
+
+def get_workload(name: str) -> cf.Workload:
+    if name == "long_decode_pairs":
+        return cf.long_decode(pairs=True)
+    return cf.ALL[name]()
+
+
+# ---------------------------------------------------------------------------
+# clocks
+# ---------------------------------------------------------------------------
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-i", str(self.index), "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], None, set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            parts = [p.strip() for p in ln.split(",")]
+            if len(parts) < 6:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                mx = float(parts[1])
+            except ValueError:
+                continue
+            for nm, val in zip(names, parts[2:6]):
+                if val.lower().startswith("active"):
+                    reasons.add(nm)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": mx,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# ---------------------------------------------------------------------------
+# CPU checker timing (cpu_baseline leg and --impl reference)
+# ---------------------------------------------------------------------------
+def oracle_sample_prepare(wl: cf.Workload, n_seqs: int, heads_per_layer: int):
+    """Inputs of the CPU checker's timed sample: layer 0 (standard) and layer 1
+    (sliding window), the first `n_seqs` sequences, `heads_per_layer` query heads."""
+    dt = torch.bfloat16 if wl.dtype == cf.BF16 else torch.float32
+    e = 2 if wl.dtype == cf.BF16 else 4
+    G = wl.n_q_heads // wl.n_kv_heads
+    n = wl.context + 1
+    heads = list(range(heads_per_layer))
+    jobs = []
+    for layer in (0, 1):
+        kind, W, owner = wl.layout[layer]
+        lo = 0 if kind == cf.FULL else max(0, n - W)
+        for b in range(n_seqs):
+            q = si.q_tokens(wl.seed, layer, b, n - 1, 1, wl.n_q_heads, wl.head_dim, dt)[0].double().numpy()
+            kv = {}
+            for g in sorted({h // G for h in heads}):
+                K, V = si.kv_tokens_head(wl.seed, owner, b, lo, n - lo, wl.n_kv_heads, wl.head_dim, g, dt)
+                kv[g] = (K.double().numpy(), V.double().numpy())
+            # bytes the job stands for: the KV heads touched, counted once per group of heads
+            jobs.append((q, kv, heads, G, (n - lo) * 2 * wl.head_dim * e * (len(heads) / G)))
+    return jobs, 1.0 / np.sqrt(wl.head_dim)
+
+
+def oracle_sample_run(jobs, scale):
+    """One pass of the CPU checker over the prepared sample: (seconds, KV bytes)."""
+    from oracle import mixattn_oracle as mo
+    t0 = time.perf_counter()
+    nbytes = 0.0
+    for q, kv, heads, G, b in jobs:
+        for h in heads:
+            K, V = kv[h // G]
+            mo.softmax_attend(q[h], K, V, scale)
+        nbytes += b
+    return time.perf_counter() - t0, nbytes
+
+
+def blas_threads() -> int:
+    try:
+        from threadpoolctl import threadpool_info
+        return max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
+    except Exception:
+        return 1
+
+
+def run_reference_arm(args, wl):
+    """The CPU checker as the reference arm: K steps, each one pass over a bounded sample."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    n_seqs, heads = 2, wl.n_q_heads
+    jobs, scale = oracle_sample_prepare(wl, n_seqs, heads)
+    for _ in range(args.warmup):
+        oracle_sample_run(jobs, scale)
+    secs, nbytes = 0.0, 0.0
+    for _ in range(args.steps):
+        s, b = oracle_sample_run(jobs, scale)
+        secs += s
+        nbytes += b
+    threads = blas_threads()
+    value = nbytes / secs / 1e9
+    sample = (f"layers 0 (standard) and 1 (sliding window) of sequences 0..{n_seqs - 1}, all {heads} query "
+              f"heads, context {wl.context}+1, per step")
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": secs / args.steps * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+        "data": "synthetic", "config": {"workload": wl.name, "sample": sample},
+        "cpu_baseline": {"value": value, "unit": "GB/s", "cores": threads, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line), flush=True)
+
+
+# ---------------------------------------------------------------------------
+# GPU arm
+# ---------------------------------------------------------------------------
+def prefill_figures(mx, runner, peaks, device):
+    """Prompt pass on the prefill configuration: one standard and one sliding layer."""
+    wl = cf.prefill_chunk()
+    sess = runner.Session(wl, [0] * wl.batch, device=device)
+    res = {}
+    try:
+        S, W, D, Hq, B = wl.seq_len, 1024, wl.head_dim, wl.n_q_heads, wl.batch
+        pairs_full = S * (S + 1) // 2
+        pairs_slide = sum(min(i + 1, W) for i in range(S))
+        for name, layer, pairs, cls in (("full", 12, pairs_full, mx.K_PREFILL_FULL),
+                                        ("sliding", 2, pairs_slide, mx.K_PREFILL_SLIDING)):
+            q, k, v = sess.prefill_inputs(layer)      # readers: no cache writes, repeatable
+            out = torch.empty_like(q)
+            reps = 3
+            sess.prefill_layer(layer, q, k, v, out)
+            torch.cuda.synchronize()
+            sess.ctx.profile_enable(True)
+            for _ in range(reps):
+                sess.prefill_layer(layer, q, k, v, out)
+            n, ms = sess.ctx.profile_read(cls)
+            sess.ctx.profile_enable(False)
+            flops = 4.0 * D * pairs * Hq * B
+            tf = flops / (ms / n * 1e-3) / 1e12
+            res[name] = {"ms_per_layer": ms / n, "tflops": tf, "frac_of_bf16_peak": tf / peaks["bf16_tflops"],
+                         "useful_flop": flops}
+        res["config"] = {"workload": wl.name, "batch": B, "seq_len": S, "window": W}
+        res["peak_tflops"] = peaks["bf16_tflops"]
+        res["peak_source"] = peaks["_source"]
+    finally:
+        sess.close()
+    return res
+
+
+def run_gpu_arm(args, wl):
+    from paper_2409_15012_b200 import build as mbuild
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU path")
+    if rank == 0:
+        mbuild.build()
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local}"))
+        dist.barrier()
+    from paper_2409_15012_b200 import binding as mx, runner
+    peaks = load_peaks()
+    K, Wm = args.steps, args.warmup
+    total_steps = 2 * (K + Wm) + K + 2       # device-timed pass, e2e pass, profiled pass
+
+    if wl.context_range != (0, 0):
+        lengths = si.draw_lengths(wl.seed, wl.batch, *wl.context_range).tolist()
+    else:
+        lengths = [wl.context] * wl.batch
+    free_order = None
+    if wl.permute_pages:
+        n_pages = sum(-(-(n + total_steps) // wl.page_size) for n in lengths)
+        free_order = si.page_permutation(wl.seed, n_pages)
+    sess = runner.Session(wl, lengths, device=local, headroom_tokens=total_steps, free_order=free_order)
+    sess.fill(1024)
+    stream = torch.cuda.current_stream()
+    outs = sess.alloc_outputs()
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def bytes_next_step():
+        return runner.kv_bytes_per_step(wl, [int(p) + 1 for p in sess.pos])
+
+    # ---- device-resident pass: `value` ----
+    step_inputs = []
+    pos_save = sess.pos.copy()
+    for s in range(Wm + K):
+        step_inputs.append(sess.step_inputs())
+        sess.pos += 1
+    sess.pos[:] = pos_save
+    for s in range(Wm):
+        sess.decode_step(step_inputs[s], outs, stream)
+    launches0 = sess.ctx.get_launch_count()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    barrier()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    kv_bytes = 0
+    ev0.record(stream)
+    for s in range(K):
+        kv_bytes += bytes_next_step()
+        sess.decode_step(step_inputs[Wm + s], outs, stream)
+    ev1.record(stream)
+    barrier()
+    ms = ev0.elapsed_time(ev1)
+    clocks = sampler.stop() if rank == 0 else None
+    launches = sess.ctx.get_launch_count() - launches0
+    assert sess.ctx.get_device_status() == 0, "a kernel reported a wait time-out"
+
+    # ---- end-to-end pass: host inputs, host outputs ----
+    host_inputs = []
+    pos_save = sess.pos.copy()
+    for s in range(Wm + K):
+        ent = sess.step_inputs()
+        host_inputs.append({l: {k: t.cpu().pin_memory() for k, t in d.items()} for l, d in ent.items()})
+        sess.pos += 1
+    sess.pos[:] = pos_save
+    dev_buf = {l: {k: torch.empty_like(t, device=sess.dev) for k, t in d.items()} for l, d in host_inputs[0].items()}
+    host_out = torch.empty(outs.shape, dtype=outs.dtype).pin_memory()
+    h2d = sum(t.numel() * t.element_size() for d in host_inputs[0].values() for t in d.values())
+    d2h = outs.numel() * outs.element_size()
+
+    def e2e_step(s):
+        for l, d in host_inputs[s].items():
+            for k, t in d.items():
+                dev_buf[l][k].copy_(t, non_blocking=True)
+        sess.decode_step(dev_buf, outs, stream)
+        host_out.copy_(outs, non_blocking=True)
+        stream.synchronize()
+
+    for s in range(Wm):
+        e2e_step(s)
+    barrier()
+    e2e_bytes = 0
+    t0 = time.perf_counter()
+    ev0.record(stream)
+    for s in range(K):
+        e2e_bytes += bytes_next_step()
+        e2e_step(Wm + s)
+    ev1.record(stream)
+    barrier()
+    e2e_ms = max(ev0.elapsed_time(ev1), (time.perf_counter() - t0) * 1e3 if world == 1 else 0.0)
+
+    # ---- per-kernel pass: roofline of the dominant kernel (split pass of a standard layer) ----
+    full_layers = [l for l, (kind, _, _) in enumerate(wl.layout) if kind == cf.FULL]
+    slide_layers = [l for l, (kind, _, _) in enumerate(wl.layout) if kind == cf.SLIDING]
+    e = 2 if wl.dtype == cf.BF16 else 4
+    per_tok = 2 * wl.n_kv_heads * wl.head_dim * e
+    sess.ctx.profile_enable(True)
+    full_bytes = 0
+    for s in range(K):
+        ent = sess.step_inputs()
+        full_bytes += sum(int(p) + 1 for p in sess.pos) * per_tok
+        sess.decode_step(ent, outs, stream)
+    n_full, ms_full = sess.ctx.profile_read(mx.K_DECODE_FULL)
+    n_slide, ms_slide = sess.ctx.profile_read(mx.K_DECODE_SLIDING)
+    n_comb, ms_comb = sess.ctx.profile_read(mx.K_COMBINE)
+    n_app, ms_app = sess.ctx.profile_read(mx.K_APPEND)
+    sess.ctx.profile_enable(False)
+
+    # ---- max over ranks, sum of work ----
+    if dist is not None:
+        t = torch.tensor([ms, e2e_ms], device=sess.dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms, e2e_ms = t.tolist()
+        w = torch.tensor([float(kv_bytes), float(e2e_bytes), float(launches)], device=sess.dev, dtype=torch.float64)
+        dist.all_reduce(w, op=dist.ReduceOp.SUM)
+        kv_bytes, e2e_bytes, launches = w.tolist()
+    if rank != 0:
+        sess.close()
+        dist.destroy_process_group()
+        return
+
+    value = kv_bytes / (ms * 1e-3) / 1e9
+    # achieved = bytes per launch / seconds per launch
+    bytes_per_launch = full_bytes / K if K else 0
+    sec_per_launch = ms_full / max(n_full, 1) * 1e-3
+    achieved = bytes_per_launch / sec_per_launch / 1e9
+    roofline = {
+        "kernel": "decode_split_bf16_kernel (standard layer)" if wl.dtype == cf.BF16 else "decode_split_f32_kernel",
+        "bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+        "frac": achieved / peaks["hbm_gbs"], "traffic": DECODE_FULL_TRAFFIC_BYTES,
+        "peak_source": f"of {peaks['_source']}", "bytes_per_launch": bytes_per_launch,
+        "us_per_launch": sec_per_launch * 1e6, "frac_of_nominal_8TBs": achieved / 8000.0,
+    }
+
+    # ---- CPU checker beside it (bounded sample) ----
+    cpu = None
+    if not args.no_cpu_baseline:
+        jobs, scale = oracle_sample_prepare(wl.scaled(context=int(lengths[0])), 2, wl.n_q_heads)
+        secs, nbytes, reps = 0.0, 0.0, 0
+        while secs < 10.0:
+            s_, b_ = oracle_sample_run(jobs, scale)
+            secs += s_
+            nbytes += b_
+            reps += 1
+        cpu = {"value": nbytes / secs / 1e9, "unit": "GB/s", "cores": blas_threads(), "kind": "oracle",
+               "sample": f"layers 0 (standard) and 1 (sliding window), sequences 0-1, all {wl.n_q_heads} query "
+                         f"heads, context {int(lengths[0])}+1; {reps} passes, {secs:.1f} s",
+               "host_cores": os.cpu_count()}
+
+    prefill = None
+    if not args.no_prefill:
+        sess.close()
+        prefill = prefill_figures(mx, runner, peaks, local)
+
+    line = {
+        "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": K, "warmup": Wm,
+        "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16" if wl.dtype == cf.BF16 else "f32", "data": "synthetic",
+        "config": {"workload": wl.name, "batch": wl.batch, "context": wl.context or list(wl.context_range),
+                   "window": 1024, "layers": len(wl.layout), "heads": f"{wl.n_q_heads}/{wl.n_kv_heads}x{wl.head_dim}",
+                   "l2": "inputs larger than L2 (KV read per step >> 126 MB)", "parallelism": "replicas only"},
+        "tokens_per_s": wl.batch * world / (ms / K * 1e-3),
+        "frac_of_measured_hbm": value / world / peaks["hbm_gbs"],
+        "frac_of_nominal_8TBs": value / world / 8000.0,
+        "us_per_layer": {"full_split": ms_full / max(n_full, 1) * 1e3, "sliding_split": ms_slide / max(n_slide, 1) * 1e3,
+                         "combine": ms_comb / max(n_comb, 1) * 1e3, "append": ms_app / max(n_app, 1) * 1e3},
+        "e2e": {"value": e2e_bytes / (e2e_ms * 1e-3) / 1e9, "unit": "GB/s", "h2d_bytes_per_step": h2d,
+                "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms / K},
+        "gpu_launches": int(launches),
+        "clocks": clocks,
+        "roofline": roofline,
+        "cpu_baseline": cpu,
+        "prefill": prefill,
+    }
+    print(json.dumps(line), flush=True)
+    if prefill is None:
+        sess.close()
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="mid_decode",
+                    choices=["mid_decode", "long_decode", "long_decode_pairs", "mixed_serving", "tiny_decode"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-prefill", action="store_true")
+    args = ap.parse_args()
+    if args.warmup < 3:
+        args.warmup = 3
+    wl = get_workload(args.workload)
+    if args.impl == "reference":
+        run_reference_arm(args, wl)
+    else:
+        run_gpu_arm(args, wl)
+
+
+if __name__ == "__main__":
+    main()

@@ -50,8 +50,9 @@ def stream_key(seed: int, stream: int, a: int, b: int) -> int:
     return k
 
 
-def unit_normal(key: int, idx: torch.Tensor) -> torch.Tensor:
-    """fp32 tensor, one ~N(0,1) value per int64 counter in `idx` (any device)."""
+def unit_normal(key, idx: torch.Tensor) -> torch.Tensor:
+    """fp32 tensor, one ~N(0,1) value per int64 counter in `idx` (any device).
+    `key` is a 32-bit int or an int64 tensor of such keys that broadcasts with idx."""
     x = _mix32((idx & _M32) ^ key)
     x = _mix32(x ^ ((idx >> 32) & _M32))
     acc = torch.zeros_like(idx)
@@ -76,6 +77,31 @@ def kv_tokens(seed, owner, seq, pos0, n, n_kv_heads, head_dim, dtype, device="cp
     key = stream_key(seed, _STREAM_KV, owner, seq)
     per_tok = 2 * n_kv_heads * head_dim
     kv = _block(key, pos0 * per_tok, (n, 2, n_kv_heads, head_dim), dtype, device)
+    return kv[:, 0].contiguous(), kv[:, 1].contiguous()
+
+
+def kv_tokens_multi(seed, owner, seqs, pos0s, n, n_kv_heads, head_dim, dtype, device="cpu"):
+    """Same values as kv_tokens for several sequences at once: tokens
+    pos0s[i] .. pos0s[i]+n-1 of seqs[i].  Returns (K, V), each
+    [len(seqs), n, n_kv_heads, head_dim]."""
+    per_tok = 2 * n_kv_heads * head_dim
+    keys = torch.tensor([stream_key(seed, _STREAM_KV, owner, int(s)) for s in seqs],
+                        dtype=torch.int64, device=device).view(-1, 1)
+    first = torch.tensor([int(p) * per_tok for p in pos0s], dtype=torch.int64, device=device).view(-1, 1)
+    idx = first + torch.arange(n * per_tok, dtype=torch.int64, device=device).view(1, -1)
+    kv = unit_normal(keys, idx).to(dtype).reshape(len(seqs), n, 2, n_kv_heads, head_dim)
+    return kv[:, :, 0].contiguous(), kv[:, :, 1].contiguous()
+
+
+def kv_tokens_head(seed, owner, seq, pos0, n, n_kv_heads, head_dim, g, dtype, device="cpu"):
+    """K and V of one KV head `g` only: (K, V), each [n, head_dim]; same values
+    as kv_tokens(...)[..][:, g]."""
+    key = stream_key(seed, _STREAM_KV, owner, seq)
+    pos = torch.arange(pos0, pos0 + n, dtype=torch.int64, device=device).view(n, 1, 1)
+    which = torch.arange(2, dtype=torch.int64, device=device).view(1, 2, 1)
+    d = torch.arange(head_dim, dtype=torch.int64, device=device).view(1, 1, head_dim)
+    idx = ((pos * 2 + which) * n_kv_heads + g) * head_dim + d
+    kv = unit_normal(key, idx).to(dtype)
     return kv[:, 0].contiguous(), kv[:, 1].contiguous()
 
 

@@ -45,3 +45,12 @@ def test_layouts():
     pairs = cf.layout_pairs(1024)
     assert pairs[2][2] == 1 and pairs[11][2] == 11 and pairs[13][2] == 13 and pairs[14][2] == 13
     assert pairs[23][2] == 23 and pairs[12] == (cf.FULL, 0, 0)
+
+
+def test_multi_and_head_variants_agree():
+    K, V = si.kv_tokens(3, 1, 4, 10, 6, 2, 16, torch.bfloat16)
+    Km, Vm = si.kv_tokens_multi(3, 1, [2, 4], [0, 10], 6, 2, 16, torch.bfloat16)
+    assert torch.equal(Km[1], K) and torch.equal(Vm[1], V)
+    assert torch.equal(Km[0], si.kv_tokens(3, 1, 2, 0, 6, 2, 16, torch.bfloat16)[0])
+    Kh, Vh = si.kv_tokens_head(3, 1, 4, 10, 6, 2, 16, 1, torch.bfloat16)
+    assert torch.equal(Kh, K[:, 1]) and torch.equal(Vh, V[:, 1])
