@@ -109,6 +109,12 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   __nv_bfloat162 t = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<uint32_t*>(&t);
 }
+// (x, y) -> packed bf16 pair `hi` and packed bf16 pair `lo` of the rounding residuals
+__device__ __forceinline__ void split_bf16(float x, float y, uint32_t& hi, uint32_t& lo) {
+  __nv_bfloat162 h = __floats2bfloat162_rn(x, y);
+  hi = *reinterpret_cast<uint32_t*>(&h);
+  lo = pack_bf16(x - __low2float(h), y - __high2float(h));
+}
 __device__ __forceinline__ void consumer_bar() {  // the 256 consumer threads only
   asm volatile("bar.sync 1, %0;" ::"n"(kConsumerWarps * 32) : "memory");
 }
@@ -297,11 +303,13 @@ decode_split_bf16_kernel(const __grid_constant__ DecodeParams p, const int n_sta
         s1[2] = exp2f(s1[2] - mn1); s1[3] = exp2f(s1[3] - mn1);
         l[0] = l[0] * a0 + (s0[0] + s0[1] + s1[0] + s1[1]);
         l[1] = l[1] * a1 + (s0[2] + s0[3] + s1[2] + s1[3]);
-        uint32_t pa[4];
-        pa[0] = pack_bf16(s0[0], s0[1]);
-        pa[1] = pack_bf16(s0[2], s0[3]);
-        pa[2] = pack_bf16(s1[0], s1[1]);
-        pa[3] = pack_bf16(s1[2], s1[3]);
+        // P as two bf16 terms (hi + residual): the HBM stream leaves tensor-core time
+        // to spare, so P keeps ~16 significant bits instead of 8
+        uint32_t pa[4], pr[4];
+        split_bf16(s0[0], s0[1], pa[0], pr[0]);
+        split_bf16(s0[2], s0[3], pa[1], pr[1]);
+        split_bf16(s1[0], s1[1], pa[2], pr[2]);
+        split_bf16(s1[2], s1[3], pa[3], pr[3]);
 #pragma unroll
         for (int j = 0; j < D / 8; ++j) {
           o[j][0] *= a0; o[j][1] *= a0;
@@ -313,6 +321,8 @@ decode_split_bf16_kernel(const __grid_constant__ DecodeParams p, const int n_sta
           ldsm_x4_t(vb + v_tok * kRowBytes + (((2 * jj + v_chk) ^ (v_tok & 7)) << 4), b0, b1, b2, b3);
           mma_bf16(o[2 * jj], pa, b0, b1);
           mma_bf16(o[2 * jj + 1], pa, b2, b3);
+          mma_bf16(o[2 * jj], pr, b0, b1);
+          mma_bf16(o[2 * jj + 1], pr, b2, b3);
         }
       }
       __syncwarp();
