@@ -14,8 +14,8 @@ using namespace mixattn;
 namespace {
 
 constexpr size_t kAlign = 256;
-constexpr int kItemsPerSm = 4;       // automatic split: work items per SM aimed for
-constexpr int kMinSplitTokens = 256;
+constexpr int kSplitTokens = 4096;    // automatic split length of long caches (keys)
+constexpr int kMinSplitTokens = 1024; // single-wave splitting never makes splits shorter than this
 
 inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
@@ -359,27 +359,29 @@ int mixattn_decode(mixattn_ctx* c, int32_t layer, int32_t n_seqs, const int32_t*
       p.n_eff[j] = c->cm.n_attended(layer, p.seq_id[j]);
       total += p.n_eff[j];
     }
-    // split length: aim at kItemsPerSm work items per SM, never more splits than the workspace holds
-    int64_t T;
-    if (c->split_tokens > 0) {
-      T = (c->split_tokens + kPage - 1) / kPage * kPage;
-    } else {
-      int64_t chunks_target = (int64_t)c->sm_count * kItemsPerSm / ((int64_t)Hkv * p.head_chunks);
-      if (chunks_target < 1) chunks_target = 1;
-      T = (total + chunks_target - 1) / chunks_target;
-      T = (T + 63) / 64 * 64;
-      if (T < kMinSplitTokens) T = kMinSplitTokens;
-    }
+    // Split choice.  Long caches are cut into splits of kSplitTokens keys (large splits
+    // keep the per-item epilogue negligible; thousands of items balance over the SMs).
+    // When there are fewer (sequence, KV head) pairs than SMs, short caches are cut
+    // further, but only up to one item per SM, so the launch stays a single wave.
+    int64_t T = c->split_tokens > 0 ? (c->split_tokens + kPage - 1) / kPage * kPage : kSplitTokens;
     int64_t t_min = (total + kWsExtraChunks - 1) / kWsExtraChunks;
     t_min = (t_min + kPage - 1) / kPage * kPage;
     if (T < t_min) T = t_min;
+    const int64_t pairs = (int64_t)nb * Hkv * p.head_chunks;
+    const int64_t nc_wave = c->split_tokens > 0 ? 1 : c->sm_count / pairs;
     int base = 0;
     bool any_split = false;
     for (int j = 0; j < nb; ++j) {
       const int64_t n = p.n_eff[j];
-      const int64_t nc = (n + T - 1) / T;
+      int64_t nc = (n + T - 1) / T;
+      if (nc < nc_wave) {
+        int64_t by_len = n / kMinSplitTokens;
+        nc = by_len < nc_wave ? by_len : nc_wave;
+        if (nc < 1) nc = 1;
+      }
       int64_t len = (n + nc - 1) / nc;
       len = (len + kPage - 1) / kPage * kPage;
+      nc = (n + len - 1) / len;
       p.chunk_base[j] = base;
       p.chunk_len[j] = (int32_t)len;
       base += (int)nc;

@@ -13,10 +13,13 @@
 //     running across work items, so the next item's keys arrive during this item's
 //     epilogue;
 //   * eight consumer warps, two groups alternating stages, one 16-key page per warp:
-//     S = Q K^T and O += P V on mma.sync m16n8k16 (bf16 in, fp32 out), online softmax in
-//     base 2 with quad shuffles, private running (max, sum, O) per warp;
+//     S^T = K Q^T and O^T += V^T P^T on mma.sync m16n8k16 (bf16 in, fp32 out) with the
+//     keys as the M dimension and the heads as N = 8, online softmax in base 2, private
+//     running (max, sum, O) per warp;
 //   * per item the warps merge through shared memory and write either the final output
 //     (sequence not split) or an unnormalised partial + (max, sum) for the combine pass.
+//     (Combining inside this kernel -- last split to finish, ticket counter -- was
+//     measured slower: the fence before the ticket stalls the consumers per item.)
 //
 // Every mbarrier wait is bounded: on time-out the kernel raises a status word and all
 // roles leave.
@@ -115,6 +118,11 @@ __device__ __forceinline__ void split_bf16(float x, float y, uint32_t& hi, uint3
   hi = *reinterpret_cast<uint32_t*>(&h);
   lo = pack_bf16(x - __low2float(h), y - __high2float(h));
 }
+__device__ __forceinline__ uint32_t movmatrix_t(uint32_t a) {  // transpose an 8x8 b16 fragment
+  uint32_t d;
+  asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(d) : "r"(a));
+  return d;
+}
 __device__ __forceinline__ void consumer_bar() {  // the 256 consumer threads only
   asm volatile("bar.sync 1, %0;" ::"n"(kConsumerWarps * 32) : "memory");
 }
@@ -192,16 +200,28 @@ decode_split_bf16_kernel(const __grid_constant__ DecodeParams p, const int n_sta
       const int64_t ring_page0 = (int64_t)seq * p.ring_pages;
       const int page_lo = x.t0 / kPage;
       const int page_hi = (x.t1 + kPage - 1) / kPage;
+      // page ids are fetched 32 at a time (one per lane), one batch ahead of their use,
+      // so the table lookup is off the issue path of the copies
+      int ids_next = 0;
+      if (tbl && page_lo + lane < page_hi) ids_next = tbl[page_lo + lane];
+      int ids = 0;
       for (int pg = page_lo; pg < page_hi; pg += kGroupWarps, ++K) {
+        const int rel = pg - page_lo;
+        if ((rel & 31) == 0) {
+          ids = ids_next;
+          if (tbl && pg + 32 + lane < page_hi) ids_next = tbl[pg + 32 + lane];
+        }
         const int s = K % n_stages;
-        if (K >= n_stages) {
-          if (!mbar_wait(empty0 + 8 * s, ((K / n_stages) - 1) & 1, abort_flag)) { ok = false; break; }
+        if (K >= n_stages) {  // lane 0 waits; the verdict is made warp-uniform
+          int w = 1;
+          if (lane == 0) w = mbar_wait(empty0 + 8 * s, ((K / n_stages) - 1) & 1, abort_flag);
+          if (!__shfl_sync(0xffffffffu, w, 0)) { ok = false; break; }
         }
         const int n_pg = min(kGroupWarps, page_hi - pg);
         if (lane == 0) mbar_arrive_expect_tx(full0 + 8 * s, n_pg * kBlkBytes);
-        __syncwarp();
+        const int my_id = __shfl_sync(0xffffffffu, ids, (rel & 31) + (lane & (kGroupWarps - 1)));
         if (lane < n_pg) {
-          const int64_t phys = tbl ? (int64_t)tbl[pg + lane] : ring_page0 + pg + lane;
+          const int64_t phys = tbl ? (int64_t)my_id : ring_page0 + pg + lane;
           const char* src = p.pool + phys * ge.page_bytes + (int64_t)x.g * kBlkBytes;
           bulk_g2s(smem_u32(stages + (size_t)s * kStageBytes + lane * kBlkBytes), src, kBlkBytes,
                    full0 + 8 * s);
@@ -220,14 +240,19 @@ decode_split_bf16_kernel(const __grid_constant__ DecodeParams p, const int n_sta
   }
 
   // -------------------------------- consumers --------------------------------
+  // Transposed formulation: keys are the M dimension, the (up to 8) query heads of the
+  // group the N dimension.  S^T = K Q^T (one m16n8 tile per 16 keys), P^T is transposed
+  // in registers (movmatrix) into the B operand of O^T += V^T P^T.  Each thread owns two
+  // heads (columns 2*(lane&3), +1) of every accumulator, so the online-softmax state is
+  // thread-local apart from the column max / sum over the eight row groups.
   const int grp = warp / kGroupWarps;   // which stages this warp consumes
   const int wig = warp % kGroupWarps;   // page of the stage
-  const int qrow = lane >> 2;           // fragment row (and row + 8)
-  const int qcol = (lane & 3) * 2;
+  const int frow = lane >> 2;           // fragment row (and row + 8)
+  const int fcol = (lane & 3) * 2;      // fragment column pair = the two heads of this thread
   // ldmatrix.x4 lane addressing inside a (page, head) block: lane -> (matrix lm, row lr)
   const int lm = lane >> 3, lr = lane & 7;
-  const int k_tok = (lm >> 1) * 8 + lr, k_chk = lm & 1;   // K: (keys 0-7 | 8-15) x (chunk 2ks | 2ks+1)
-  const int v_tok = (lm & 1) * 8 + lr, v_chk = lm >> 1;   // V: (keys 0-7 | 8-15) x (chunk 2jj | 2jj+1)
+  const int k_tok = (lm & 1) * 8 + lr, k_chk = lm >> 1;   // K as A: (keys 0-7|8-15) x (chunk 2ks|2ks+1)
+  const int v_tok = (lm >> 1) * 8 + lr, v_chk = lm & 1;   // V^T as A (.trans): (chunk 2jt|2jt+1) x (keys 0-7|8-15)
 
   int K = 0;
   for (int it = blockIdx.x; it < p.total_items; it += gridDim.x) {
@@ -235,95 +260,85 @@ decode_split_bf16_kernel(const __grid_constant__ DecodeParams p, const int n_sta
     const int rows = min(kMaxGroupRows, p.group - x.hc * kMaxGroupRows);
     const int h0 = x.g * p.group + x.hc * kMaxGroupRows;
 
-    // Q fragments (A operand), rows = query heads of the group
-    uint32_t qa[kKSteps][4];
+    // Q^T fragments (B operand): thread holds head (lane >> 2), channels 16 ks + fcol (+8)
+    uint32_t qb[kKSteps][2];
     {
-      const __nv_bfloat16* qb = reinterpret_cast<const __nv_bfloat16*>(p.q) +
-                                ((int64_t)x.i * p.n_q_heads + h0) * D;
+      const __nv_bfloat16* qp = reinterpret_cast<const __nv_bfloat16*>(p.q) +
+                                ((int64_t)x.i * p.n_q_heads + h0 + frow) * D + fcol;
 #pragma unroll
       for (int ks = 0; ks < kKSteps; ++ks) {
-        const int d = ks * 16 + qcol;
-        qa[ks][0] = qrow < rows ? *reinterpret_cast<const uint32_t*>(qb + qrow * D + d) : 0u;
-        qa[ks][1] = qrow + 8 < rows ? *reinterpret_cast<const uint32_t*>(qb + (qrow + 8) * D + d) : 0u;
-        qa[ks][2] = qrow < rows ? *reinterpret_cast<const uint32_t*>(qb + qrow * D + d + 8) : 0u;
-        qa[ks][3] = qrow + 8 < rows ? *reinterpret_cast<const uint32_t*>(qb + (qrow + 8) * D + d + 8) : 0u;
+        qb[ks][0] = frow < rows ? *reinterpret_cast<const uint32_t*>(qp + ks * 16) : 0u;
+        qb[ks][1] = frow < rows ? *reinterpret_cast<const uint32_t*>(qp + ks * 16 + 8) : 0u;
       }
     }
     float m[2] = {-INFINITY, -INFINITY};
     float l[2] = {0.f, 0.f};
-    float o[D / 8][4];
+    float o[D / 16][4];   // O^T: rows = channels 16 jt + frow (+8), cols = the thread's two heads
 #pragma unroll
-    for (int j = 0; j < D / 8; ++j) o[j][0] = o[j][1] = o[j][2] = o[j][3] = 0.f;
+    for (int j = 0; j < D / 16; ++j) o[j][0] = o[j][1] = o[j][2] = o[j][3] = 0.f;
 
     const int n_tiles = ((x.t1 + kPage - 1) / kPage - x.t0 / kPage + kGroupWarps - 1) / kGroupWarps;
     for (int k = 0; k < n_tiles; ++k) {
       const int Kg = K + k;
       if ((Kg & 1) != grp) continue;
       const int s = Kg % n_stages;
-      if (!mbar_wait(full0 + 8 * s, (Kg / n_stages) & 1, abort_flag)) break;  // abort_flag is set
+      // every lane waits (each needs to observe the copy), the verdict is warp-uniform
+      if (!__all_sync(0xffffffffu, mbar_wait(full0 + 8 * s, (Kg / n_stages) & 1, abort_flag))) break;
       const int tok_base = x.t0 + k * kTileKeys + wig * kPage;
       if (tok_base < x.t1) {
         const uint32_t kb = smem_u32(stages + (size_t)s * kStageBytes + wig * kBlkBytes);
         const uint32_t vb = kb + kPage * kRowBytes;
-        float s0[4] = {0.f, 0.f, 0.f, 0.f}, s1[4] = {0.f, 0.f, 0.f, 0.f};
+        float st[4] = {0.f, 0.f, 0.f, 0.f}, st2[4] = {0.f, 0.f, 0.f, 0.f};  // two chains: shorter latency
 #pragma unroll
-        for (int ks = 0; ks < kKSteps; ++ks) {
-          uint32_t b0, b1, b2, b3;
-          ldsm_x4(kb + k_tok * kRowBytes + (((2 * ks + k_chk) ^ (k_tok & 7)) << 4), b0, b1, b2, b3);
-          mma_bf16(s0, qa[ks], b0, b1);
-          mma_bf16(s1, qa[ks], b2, b3);
+        for (int ks = 0; ks < kKSteps; ks += 2) {
+          uint32_t a[4], b[4];
+          ldsm_x4(kb + k_tok * kRowBytes + (((2 * ks + k_chk) ^ (k_tok & 7)) << 4), a[0], a[1], a[2], a[3]);
+          ldsm_x4(kb + k_tok * kRowBytes + (((2 * ks + 2 + k_chk) ^ (k_tok & 7)) << 4), b[0], b[1], b[2], b[3]);
+          mma_bf16(st, a, qb[ks][0], qb[ks][1]);
+          mma_bf16(st2, b, qb[ks + 1][0], qb[ks + 1][1]);
         }
 #pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          s0[e] *= p.scale_log2e;
-          s1[e] *= p.scale_log2e;
-        }
-        if (tok_base + kPage > x.t1) {  // ragged end of the split
+        for (int e = 0; e < 4; ++e) st[e] = (st[e] + st2[e]) * p.scale_log2e;
+        if (tok_base + kPage > x.t1) {  // ragged end of the split: keys are rows frow, frow + 8
           const int lim = x.t1 - tok_base;
-#pragma unroll
-          for (int e = 0; e < 4; ++e) {
-            if (qcol + (e & 1) >= lim) s0[e] = -INFINITY;
-            if (8 + qcol + (e & 1) >= lim) s1[e] = -INFINITY;
-          }
+          if (frow >= lim) st[0] = st[1] = -INFINITY;
+          if (frow + 8 >= lim) st[2] = st[3] = -INFINITY;
         }
-        // online softmax: rows qrow (elements 0,1) and qrow + 8 (elements 2,3)
-        float mx0 = fmaxf(fmaxf(s0[0], s0[1]), fmaxf(s1[0], s1[1]));
-        float mx1 = fmaxf(fmaxf(s0[2], s0[3]), fmaxf(s1[2], s1[3]));
-        mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 1));
-        mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 2));
-        mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 1));
-        mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 2));
+        // column (head) max over the 16 keys: two rows here, eight row groups across lanes
+        float mx0 = fmaxf(st[0], st[2]), mx1 = fmaxf(st[1], st[3]);
+#pragma unroll
+        for (int sh = 4; sh < 32; sh <<= 1) {
+          mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, sh));
+          mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, sh));
+        }
         const float mn0 = fmaxf(m[0], mx0), mn1 = fmaxf(m[1], mx1);
         const float a0 = exp2f(m[0] - mn0), a1 = exp2f(m[1] - mn1);
         m[0] = mn0;
         m[1] = mn1;
-        s0[0] = exp2f(s0[0] - mn0); s0[1] = exp2f(s0[1] - mn0);
-        s1[0] = exp2f(s1[0] - mn0); s1[1] = exp2f(s1[1] - mn0);
-        s0[2] = exp2f(s0[2] - mn1); s0[3] = exp2f(s0[3] - mn1);
-        s1[2] = exp2f(s1[2] - mn1); s1[3] = exp2f(s1[3] - mn1);
-        l[0] = l[0] * a0 + (s0[0] + s0[1] + s1[0] + s1[1]);
-        l[1] = l[1] * a1 + (s0[2] + s0[3] + s1[2] + s1[3]);
-        // P as two bf16 terms (hi + residual): the HBM stream leaves tensor-core time
-        // to spare, so P keeps ~16 significant bits instead of 8
-        uint32_t pa[4], pr[4];
-        split_bf16(s0[0], s0[1], pa[0], pr[0]);
-        split_bf16(s0[2], s0[3], pa[1], pr[1]);
-        split_bf16(s1[0], s1[1], pa[2], pr[2]);
-        split_bf16(s1[2], s1[3], pa[3], pr[3]);
+        st[0] = exp2f(st[0] - mn0); st[1] = exp2f(st[1] - mn1);
+        st[2] = exp2f(st[2] - mn0); st[3] = exp2f(st[3] - mn1);
+        l[0] = l[0] * a0 + (st[0] + st[2]);
+        l[1] = l[1] * a1 + (st[1] + st[3]);
+        // P^T as two bf16 terms (value + rounding residual): the stream leaves tensor
+        // time to spare, so P keeps ~16 significant bits; then transpose 8x8 blocks so
+        // that keys become the k index of the B operand
+        uint32_t ph0, pl0, ph1, pl1;
+        split_bf16(st[0], st[1], ph0, pl0);   // keys 0-7
+        split_bf16(st[2], st[3], ph1, pl1);   // keys 8-15
+        ph0 = movmatrix_t(ph0); ph1 = movmatrix_t(ph1);
+        pl0 = movmatrix_t(pl0); pl1 = movmatrix_t(pl1);
+        uint32_t va[D / 16][4];
 #pragma unroll
-        for (int j = 0; j < D / 8; ++j) {
-          o[j][0] *= a0; o[j][1] *= a0;
-          o[j][2] *= a1; o[j][3] *= a1;
+        for (int jt = 0; jt < D / 16; ++jt) {
+          ldsm_x4_t(vb + v_tok * kRowBytes + (((2 * jt + v_chk) ^ (v_tok & 7)) << 4), va[jt][0], va[jt][1],
+                    va[jt][2], va[jt][3]);
+          o[jt][0] *= a0; o[jt][1] *= a1;
+          o[jt][2] *= a0; o[jt][3] *= a1;
         }
 #pragma unroll
-        for (int jj = 0; jj < D / 16; ++jj) {
-          uint32_t b0, b1, b2, b3;
-          ldsm_x4_t(vb + v_tok * kRowBytes + (((2 * jj + v_chk) ^ (v_tok & 7)) << 4), b0, b1, b2, b3);
-          mma_bf16(o[2 * jj], pa, b0, b1);
-          mma_bf16(o[2 * jj + 1], pa, b2, b3);
-          mma_bf16(o[2 * jj], pr, b0, b1);
-          mma_bf16(o[2 * jj + 1], pr, b2, b3);
-        }
+        for (int jt = 0; jt < D / 16; ++jt) mma_bf16(o[jt], va[jt], ph0, ph1);
+#pragma unroll
+        for (int jt = 0; jt < D / 16; ++jt) mma_bf16(o[jt], va[jt], pl0, pl1);
       }
       __syncwarp();
       if (lane == 0) mbar_arrive(empty0 + 8 * s);
@@ -331,23 +346,24 @@ decode_split_bf16_kernel(const __grid_constant__ DecodeParams p, const int n_sta
     K += n_tiles;
 
     // ---- merge the eight warps' (max, sum, O) and write the item's result ----
-    l[0] += __shfl_xor_sync(0xffffffffu, l[0], 1);
-    l[0] += __shfl_xor_sync(0xffffffffu, l[0], 2);
-    l[1] += __shfl_xor_sync(0xffffffffu, l[1], 1);
-    l[1] += __shfl_xor_sync(0xffffffffu, l[1], 2);
+#pragma unroll
+    for (int sh = 4; sh < 32; sh <<= 1) {
+      l[0] += __shfl_xor_sync(0xffffffffu, l[0], sh);
+      l[1] += __shfl_xor_sync(0xffffffffu, l[1], sh);
+    }
     float* mo = merge + (size_t)warp * rows_cap * D;
     float* mml = merge_ml + (size_t)warp * rows_cap * 2;
-    if (qrow < rows) {
 #pragma unroll
-      for (int j = 0; j < D / 8; ++j)
-        *reinterpret_cast<float2*>(mo + qrow * D + j * 8 + qcol) = make_float2(o[j][0], o[j][1]);
-      if ((lane & 3) == 0) { mml[qrow * 2] = m[0]; mml[qrow * 2 + 1] = l[0]; }
-    }
-    if (qrow + 8 < rows) {
+    for (int e = 0; e < 2; ++e) {
+      const int r = fcol + e;
+      if (r < rows) {
 #pragma unroll
-      for (int j = 0; j < D / 8; ++j)
-        *reinterpret_cast<float2*>(mo + (qrow + 8) * D + j * 8 + qcol) = make_float2(o[j][2], o[j][3]);
-      if ((lane & 3) == 0) { mml[(qrow + 8) * 2] = m[1]; mml[(qrow + 8) * 2 + 1] = l[1]; }
+        for (int jt = 0; jt < D / 16; ++jt) {
+          mo[r * D + jt * 16 + frow] = o[jt][e];
+          mo[r * D + jt * 16 + frow + 8] = o[jt][2 + e];
+        }
+        if (frow == 0) { mml[r * 2] = m[e]; mml[r * 2 + 1] = l[e]; }
+      }
     }
     consumer_bar();
     if (*abort_flag) {  // uniform: set before the barrier by whichever role gave up
@@ -383,7 +399,7 @@ decode_split_bf16_kernel(const __grid_constant__ DecodeParams p, const int n_sta
 size_t smem_bytes(int D, int group, int n_stages) {
   const int rows_cap = group < kMaxGroupRows ? group : kMaxGroupRows;
   size_t stage = (size_t)kGroupWarps * 2 * kPage * D * 2;
-  return n_stages * stage + (size_t)kConsumerWarps * rows_cap * (D + 2) * 4 + 2 * kMaxStages * 8 + 16;
+  return n_stages * stage + (size_t)kConsumerWarps * rows_cap * (D + 2) * 4 + 2 * kMaxStages * 8 + 32;
 }
 
 }  // namespace

@@ -10,9 +10,9 @@ namespace mixattn {
 
 constexpr int kPage = 16;          // tokens per page (paged pools and rings alike)
 constexpr int kMaxCallSeqs = 128;  // sequences per kernel launch (metadata travels in kernel params)
-constexpr int kMaxGroupRows = 16;  // query heads of one KV head handled by one work item
+constexpr int kMaxGroupRows = 8;   // query heads of one KV head handled by one work item
 constexpr int kWsExtraChunks = 1024;                        // splits beyond one per sequence
-constexpr int kWsChunks = kMaxCallSeqs + kWsExtraChunks;    // split slots in the workspace
+constexpr int kWsChunks = kMaxCallSeqs + kWsExtraChunks + 256;  // split slots in the workspace (256: single-wave splits)
 
 // ---------------------------------------------------------------------------
 // K/V storage format.
@@ -91,7 +91,7 @@ struct DecodeParams {
   KvGeom geom;
   int32_t n_q_heads;
   int32_t group;          // query heads per KV head
-  int32_t head_chunks;    // ceil(group / 16)
+  int32_t head_chunks;    // ceil(group / 8)
   float scale_log2e;      // softmax scale * log2(e)
   float* part_o;          // [chunks, Hq, D] unnormalised partial outputs
   float2* part_ml;        // [chunks, Hq] running max (log2 units) and sum
