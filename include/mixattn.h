@@ -43,7 +43,8 @@ enum {
   MIXATTN_ERR_EMPTY_CONTEXT = -5,  /* decode on a sequence whose cache holds no token               */
   MIXATTN_ERR_BAD_SEQ = -6,        /* sequence id outside 0 .. max_seqs-1                           */
   MIXATTN_ERR_UNSUPPORTED = -7,    /* valid request this build does not implement                   */
-  MIXATTN_ERR_CUDA = -8            /* a CUDA call failed, or the context is host-only               */
+  MIXATTN_ERR_CUDA = -8,           /* a CUDA call failed, or the context is host-only               */
+  MIXATTN_ERR_TOO_LARGE = -9       /* mixattn_decode_static_scratch: request exceeds the static array */
 };
 
 /* One layer of the layout (Section 3: a mix of sliding-window layers, standard
@@ -150,6 +151,42 @@ int mixattn_decode(mixattn_ctx* ctx, int32_t layer, int32_t n_seqs, const int32_
 int mixattn_prefill(mixattn_ctx* ctx, int32_t layer, int32_t n_seqs, const int32_t* seq_ids,
                     const int32_t* seq_lens, const void* q, const void* k, const void* v,
                     void* out, void* stream);
+
+/* Size of the static device array behind mixattn_decode_static_scratch. */
+#define MIXATTN_STATIC_SCRATCH_BYTES (8u << 20)
+
+/* The same decode step as mixattn_decode, for callers that hand the library an
+ * arena holding the caches only.  (The paper has no counterpart: this is a
+ * packaging variant of the decode call, not a different computation.)
+ *
+ * mixattn_decode keeps the partial results of its split pass in a workspace at
+ * the end of the caller's arena.  Some integrations cannot provide that room,
+ * nor any other device allocation, when they call: a plugin inside a serving
+ * engine that has already handed out all device memory, a caller whose buffer
+ * was sized for the caches alone (mixattn_cache_bytes) by a party it does not
+ * control, or a runtime whose allocator must not be re-entered from inside the
+ * attention call.  For them this entry point keeps those partial results in an
+ * array that is part of the library image: MIXATTN_STATIC_SCRATCH_BYTES (8 MiB)
+ * of device memory, held by every GPU context that loads the library until the
+ * process exits.  The call itself never allocates or frees device memory,
+ * neither directly nor through a library.
+ *
+ * Arguments, results and errors are those of mixattn_decode, plus:
+ *   - n_seqs > 128, or more scratch needed than the array holds
+ *     (splits * n_q_heads * (head_dim + 2) * 4 bytes, where a sequence of n
+ *     attended keys makes about n / 4096 splits) -> MIXATTN_ERR_TOO_LARGE,
+ *     nothing launched;
+ *   - the first call on a device looks up the array's device address (a CUDA
+ *     runtime query with that device current); make that first call outside
+ *     any stream capture;
+ *   - all calls, from every context and stream of the process, share the one
+ *     array per device.  Its contents are left over from the previous call;
+ *     nothing in it needs to start at zero, since each call overwrites every
+ *     slot before it reads it.  Two calls whose kernels overlap on the GPU
+ *     (different streams) race on it: keep such calls on one stream, or order
+ *     them with events. */
+int mixattn_decode_static_scratch(mixattn_ctx* ctx, int32_t layer, int32_t n_seqs,
+                                  const int32_t* seq_ids, const void* q, void* out, void* stream);
 
 /* ---- introspection: the surface on which cache indexing is compared bit for bit ---- */
 

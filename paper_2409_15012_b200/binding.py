@@ -25,6 +25,7 @@ ERR_EMPTY_CONTEXT = -5
 ERR_BAD_SEQ = -6
 ERR_UNSUPPORTED = -7
 ERR_CUDA = -8
+ERR_TOO_LARGE = -9
 
 K_APPEND, K_DECODE_FULL, K_DECODE_SLIDING, K_COMBINE, K_PREFILL_FULL, K_PREFILL_SLIDING = range(6)
 
@@ -71,6 +72,7 @@ def _load() -> C.CDLL:
         "mixattn_seq_reset": [vp, i32],
         "mixattn_append_kv": [vp, i32, i32, p32, p32, vp, vp, vp],
         "mixattn_decode": [vp, i32, i32, p32, vp, vp, vp],
+        "mixattn_decode_static_scratch": [vp, i32, i32, p32, vp, vp, vp],
         "mixattn_prefill": [vp, i32, i32, p32, p32, vp, vp, vp, vp, vp],
         "mixattn_get_len": [vp, i32, i32, p32],
         "mixattn_get_block_table": [vp, i32, p32, i32, p32],
@@ -96,7 +98,7 @@ def _load() -> C.CDLL:
 lib = _load()
 EXPORTS = [
     "mixattn_arena_bytes", "mixattn_cache_bytes", "mixattn_create", "mixattn_destroy",
-    "mixattn_seq_reset", "mixattn_append_kv", "mixattn_decode", "mixattn_prefill",
+    "mixattn_seq_reset", "mixattn_append_kv", "mixattn_decode", "mixattn_decode_static_scratch", "mixattn_prefill",
     "mixattn_get_len", "mixattn_get_block_table", "mixattn_get_n_free_pages",
     "mixattn_get_ring_state", "mixattn_locate", "mixattn_debug_read_kv",
     "mixattn_get_device_status", "mixattn_set_split_tokens", "mixattn_profile_enable",
@@ -217,6 +219,13 @@ class Context:
         rc = self.rc_decode(layer, seq_ids, q, out, stream)
         if rc:
             raise MixAttnError(rc, "mixattn_decode")
+
+    def rc_decode_static_scratch(self, layer, seq_ids, q, out, stream=None) -> int:
+        """mixattn_decode_static_scratch: decode whose split partials live in the
+        library's static device array instead of the arena workspace."""
+        s = _i32(seq_ids)
+        return lib.mixattn_decode_static_scratch(self.h, layer, len(s), _p32(s), _dev(q), _dev(out),
+                                                 _stream(stream))
 
     def rc_prefill(self, layer, seq_ids, seq_lens, q, k, v, out, stream=None) -> int:
         s, n = _i32(seq_ids), _i32(seq_lens)

@@ -615,6 +615,129 @@ int mixattn_profile_read(mixattn_ctx* c, int32_t cls, int32_t* launches, float* 
   return MIXATTN_OK;
 }
 
+// ---------------------------------------------------------------------------
+// Decode with the split-KV scratch in a static device array (no arena workspace used).
+// ---------------------------------------------------------------------------
+namespace {
+
+constexpr size_t kStaticScratchBytes = MIXATTN_STATIC_SCRATCH_BYTES;
+constexpr int kMaxDevices = 64;
+
+// Lives in every GPU context that loads this library, until the process exits.
+static __device__ __align__(256) unsigned char g_decode_scratch[kStaticScratchBytes];
+
+// Device address of g_decode_scratch per device ordinal.  In host code the array's name
+// is only a handle for the runtime; the address a kernel can use comes from
+// cudaGetSymbolAddress, asked once per device with that device current.
+void* g_decode_scratch_ptr[kMaxDevices] = {};
+
+int static_scratch_for_current_device(int device, void** out) {
+  if (device < 0 || device >= kMaxDevices) return MIXATTN_ERR_INVALID_ARG;
+  if (g_decode_scratch_ptr[device] == nullptr) {
+    void* ptr = nullptr;
+    if (cudaGetSymbolAddress(&ptr, g_decode_scratch) != cudaSuccess || ptr == nullptr) return MIXATTN_ERR_CUDA;
+    g_decode_scratch_ptr[device] = ptr;
+  }
+  *out = g_decode_scratch_ptr[device];
+  return MIXATTN_OK;
+}
+
+}  // namespace
+
+int mixattn_decode_static_scratch(mixattn_ctx* c, int32_t layer, int32_t n_seqs, const int32_t* seq_ids,
+                                  const void* q, void* out, void* stream) {
+  if (c == nullptr || !c->cm.valid_layer(layer) || n_seqs < 0) return MIXATTN_ERR_INVALID_ARG;
+  if (n_seqs > 0 && (seq_ids == nullptr || q == nullptr || out == nullptr)) return MIXATTN_ERR_INVALID_ARG;
+  for (int i = 0; i < n_seqs; ++i) {
+    if (!c->cm.valid_seq(seq_ids[i])) return MIXATTN_ERR_BAD_SEQ;
+  }
+  for (int i = 0; i < n_seqs; ++i) {
+    if (c->cm.len(layer, seq_ids[i]) < 1) return MIXATTN_ERR_EMPTY_CONTEXT;
+  }
+  if (c->host_only || c->sticky_cuda_error) return MIXATTN_ERR_CUDA;
+  if (n_seqs == 0) return MIXATTN_OK;
+  if (n_seqs > kMaxCallSeqs) return MIXATTN_ERR_TOO_LARGE;
+
+  const LayerInfo& li = c->cm.layer(layer);
+  const bool ring = li.kind == MIXATTN_SLIDING;
+  const int Hq = c->cfg.n_q_heads, Hkv = c->cfg.n_kv_heads, D = c->cfg.head_dim;
+
+  DecodeParams p;
+  p.group = Hq / Hkv;
+  p.head_chunks = (p.group + kMaxGroupRows - 1) / kMaxGroupRows;
+  // same split plan as mixattn_decode, so both calls add the partial results in the same order
+  int64_t total = 0;
+  for (int j = 0; j < n_seqs; ++j) {
+    p.seq_id[j] = seq_ids[j];
+    p.n_eff[j] = c->cm.n_attended(layer, p.seq_id[j]);
+    total += p.n_eff[j];
+  }
+  int64_t T = c->split_tokens > 0 ? (c->split_tokens + kPage - 1) / kPage * kPage : kSplitTokens;
+  int64_t t_min = (total + kWsExtraChunks - 1) / kWsExtraChunks;
+  t_min = (t_min + kPage - 1) / kPage * kPage;
+  if (T < t_min) T = t_min;
+  const int64_t pairs = (int64_t)n_seqs * Hkv * p.head_chunks;
+  const int64_t nc_wave = c->split_tokens > 0 ? 1 : c->sm_count / pairs;
+  int base = 0;
+  bool any_split = false;
+  for (int j = 0; j < n_seqs; ++j) {
+    const int64_t n = p.n_eff[j];
+    int64_t nc = (n + T - 1) / T;
+    if (nc < nc_wave) {
+      int64_t by_len = n / kMinSplitTokens;
+      nc = by_len < nc_wave ? by_len : nc_wave;
+      if (nc < 1) nc = 1;
+    }
+    int64_t len = (n + nc - 1) / nc;
+    len = (len + kPage - 1) / kPage * kPage;
+    nc = (n + len - 1) / len;
+    p.chunk_base[j] = base;
+    p.chunk_len[j] = (int32_t)len;
+    base += (int)nc;
+    any_split = any_split || nc > 1;
+  }
+  p.chunk_base[n_seqs] = base;
+  // scratch needed: per split and query head, D partial outputs + (max, sum)
+  const size_t part_o_bytes = align_up((size_t)base * Hq * D * sizeof(float));
+  const size_t need = part_o_bytes + (size_t)base * Hq * sizeof(float2);
+  if (need > kStaticScratchBytes) return MIXATTN_ERR_TOO_LARGE;
+
+  DeviceGuard g(c->device);
+  if (!g.ok) return MIXATTN_ERR_CUDA;
+  void* scratch = nullptr;
+  int rc = static_scratch_for_current_device(c->device, &scratch);
+  if (rc != MIXATTN_OK) return rc;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+
+  p.q = q;
+  p.out = out;
+  p.pool = c->owner_storage(layer);
+  p.table = ring ? nullptr : c->dev_table();
+  p.table_stride = c->cm.max_blocks();
+  p.ring_pages = ring ? ring_pages_of(li.window) : 0;
+  p.geom = c->geom;
+  p.n_q_heads = Hq;
+  p.scale_log2e = c->scale * 1.4426950408889634f;
+  // every partial slot that the combine pass reads is written by the split pass of the
+  // same call first, so nothing in the array has to start at zero
+  p.part_o = reinterpret_cast<float*>(scratch);
+  p.part_ml = reinterpret_cast<float2*>(static_cast<char*>(scratch) + part_o_bytes);
+  p.status = c->dev_status();
+  p.n_seqs = n_seqs;
+  p.total_items = base * Hkv * p.head_chunks;
+  const int cls = ring ? MIXATTN_K_DECODE_SLIDING : MIXATTN_K_DECODE_FULL;
+  cudaError_t e = launch_recorded(c, cls, st, [&] {
+    return c->cfg.dtype == MIXATTN_BF16 ? launch_decode_split_bf16(p, c->sm_count, st)
+                                        : launch_decode_split_f32(p, st);
+  });
+  if (e != cudaSuccess) return MIXATTN_ERR_CUDA;
+  if (any_split) {
+    e = launch_recorded(c, MIXATTN_K_COMBINE, st, [&] { return launch_decode_combine(p, c->cfg.dtype, st); });
+    if (e != cudaSuccess) return MIXATTN_ERR_CUDA;
+  }
+  return MIXATTN_OK;
+}
+
 int mixattn_get_launch_count(mixattn_ctx* c, int64_t* launches) {
   if (c == nullptr || launches == nullptr) return MIXATTN_ERR_INVALID_ARG;
   *launches = c->launches;
@@ -632,6 +755,7 @@ const char* mixattn_strerror(int code) {
     case MIXATTN_ERR_BAD_SEQ: return "sequence id out of range";
     case MIXATTN_ERR_UNSUPPORTED: return "unsupported request";
     case MIXATTN_ERR_CUDA: return "CUDA error or host-only context";
+    case MIXATTN_ERR_TOO_LARGE: return "request needs more scratch than the static array holds";
     default: return "unknown status";
   }
 }
