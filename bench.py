@@ -429,12 +429,16 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="mid_decode",
                     choices=["mid_decode", "long_decode", "long_decode_pairs", "mixed_serving", "tiny_decode"])
+    ap.add_argument("--batch", type=int, default=0,
+                    help="override the batch size (smaller cases for profiler captures; not a bench value)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-prefill", action="store_true")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
     wl = get_workload(args.workload)
+    if args.batch > 0:
+        wl = wl.scaled(batch=args.batch, name=f"{wl.name}_batch{args.batch}")
     if args.impl == "reference":
         run_reference_arm(args, wl)
     else:
