@@ -261,7 +261,7 @@ int mixattn_create(const mixattn_config* cfg, mixattn_ctx** out) {
     cudaDeviceProp prop;
     if (!g.ok || cudaGetDeviceProperties(&prop, c->device) != cudaSuccess) { delete c; return MIXATTN_ERR_CUDA; }
     c->sm_count = prop.multiProcessorCount;
-    if (prepare_decode_bf16() != cudaSuccess) { delete c; return MIXATTN_ERR_CUDA; }
+    if (prepare_decode_bf16() != cudaSuccess || prepare_prefill_tc() != cudaSuccess) { delete c; return MIXATTN_ERR_CUDA; }
     if (cudaMemsetAsync(c->arena, 0, c->plan.total, 0) != cudaSuccess ||
         cudaStreamSynchronize(0) != cudaSuccess) {
       delete c;
@@ -473,8 +473,11 @@ int mixattn_prefill(mixattn_ctx* c, int32_t layer, int32_t n_seqs, const int32_t
     p.v = static_cast<const char*>(v) + (size_t)row * Hkv * D * esz;
     row += r;
     const int cls = p.window ? MIXATTN_K_PREFILL_SLIDING : MIXATTN_K_PREFILL_FULL;
+    // bf16 with head_dim 128 runs on the tensor-core kernel; everything else (fp32 mode,
+    // head_dim 64) on the exact CUDA-core kernel
+    const bool tc = prefill_tc_supported(c->cfg.dtype, D, p.q, p.k, p.v) && (((size_t)p.out) & 15) == 0;
     cudaError_t e = launch_recorded(c, cls, st, [&] {
-      return launch_prefill_simple(p, c->cfg.dtype, mlen, st);
+      return tc ? launch_prefill_tc(p, mlen, st) : launch_prefill_simple(p, c->cfg.dtype, mlen, st);
     });
     if (e != cudaSuccess) return MIXATTN_ERR_CUDA;
   }

@@ -1,0 +1,450 @@
+// Prompt attention on the 5th-generation tensor cores (tcgen05 + TMEM), bf16, head_dim 128.
+//
+// Paper, Section 3 with the causal order of Section 1: query i attends to keys j <= i
+// (standard layer) or i - window < j <= i (sliding window).  Flash-attention forward:
+// one CTA owns a 128-query tile of one (sequence, head) and walks the 128-key tiles that
+// intersect its band; tiles wholly outside the band are never loaded.
+//
+//   warp 0   TMA producer: Q once, then K (2 stages) and V (2 stages) tiles as
+//            128B-swizzled [128 x 64] boxes straight from the caller's tensors
+//   warp 1   one elected thread issues tcgen05.mma: S = Q K^T into TMEM (two S buffers),
+//            O_tile = P V into TMEM (two buffers), each 128 x 128 fp32
+//   warps 2-5  softmax: thread r owns query row r (TMEM lane r); reads S with
+//            tcgen05.ld, masks band edges, online softmax in base 2 (fp32), writes P
+//            (bf16) into shared memory in the swizzled K-major layout the MMA reads,
+//            accumulates O in registers (O = O * alpha + O_tile), normalises and stores.
+//
+// S(j+1) is issued before P V(j), so the tensor core works on the next scores while the
+// softmax warps are busy.  All mbarrier waits are bounded; on time-out a status word is
+// raised, every role leaves its loop, and TMEM is released at the common exit.
+#include <cuda.h>
+#include <cuda_bf16.h>
+
+#include "internal.h"
+
+namespace mixattn {
+
+namespace {
+
+constexpr int kBM = 128;                       // queries per CTA
+constexpr int kBN = 128;                       // keys per tile
+constexpr int kHalfBytes = 128 * 128;          // one [128 rows x 64 bf16] swizzled block
+constexpr int kTileBytes = 2 * kHalfBytes;     // a 128 x 128 bf16 operand tile
+constexpr int kThreads = 192;
+constexpr int kSmQ = 0;
+constexpr int kSmK = kSmQ + kTileBytes;        // 2 stages
+constexpr int kSmV = kSmK + 2 * kTileBytes;    // 2 stages
+constexpr int kSmP = kSmV + 2 * kTileBytes;    // 2 buffers
+constexpr int kSmBar = kSmP + 2 * kTileBytes;  // barriers, TMEM pointer, abort flag
+constexpr int kSmemBytes = kSmBar + 256 + 1024;  // + slack to align the base to 1024 B
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;
+
+// barrier indices
+enum { B_Q = 0, B_KF = 1, B_KE = 3, B_VF = 5, B_VE = 7, B_SF = 9, B_SE = 11, B_PF = 13, B_OF = 15, B_N = 17 };
+
+struct TcParams {
+  int32_t n_q_heads, group, window, n_seqs;
+  float scale_log2e;
+  int32_t* status;
+  __nv_bfloat16* out;
+  int32_t row0[kMaxCallSeqs + 1];
+};
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ unsigned long long global_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const unsigned long long t0 = global_ns();
+  for (uint32_t it = 1;; ++it) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((it & 1023u) == 0) {
+      if (*abort_flag) return false;
+      if (global_ns() - t0 > kWaitLimitNs) { *abort_flag = 1; return false; }
+    }
+  }
+}
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, int x, int y, int z, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+      ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(z), "r"(bar) : "memory");
+}
+// Shared-memory matrix descriptor, 128-byte swizzle, sm_100 format (version 1).
+// lbo / sbo in bytes.
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo, uint32_t sbo) {
+  return (uint64_t)((addr & 0x3FFFFu) >> 4) | ((uint64_t)(lbo >> 4) << 16) | ((uint64_t)(sbo >> 4) << 32) |
+         (1ull << 46) | (2ull << 61);
+}
+// D = A * B (+ D when accumulate != 0); one thread issues for the CTA.
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                          uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+      "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr));
+}
+__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+  __nv_bfloat162 t = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&t);
+}
+
+// instruction descriptor: D fp32, A/B bf16, M = 128, N = 128; b_mn = 1 for an MN-major B
+__host__ __device__ constexpr uint32_t idesc_bf16(int b_mn) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)b_mn << 16) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
+                  const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ TcParams p) {
+  extern __shared__ unsigned char smem_raw[];
+  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  unsigned char* gbase = smem_raw + (base - smem_u32(smem_raw));
+  const uint32_t bar0 = base + kSmBar;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gbase + kSmBar + B_N * 8);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(gbase + kSmBar + B_N * 8 + 8);
+#define BAR(i) (bar0 + 8u * (i))
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int b = blockIdx.z, h = blockIdx.y;
+  const int S = p.row0[b + 1] - p.row0[b];
+  const int n_qt = (S + kBM - 1) / kBM;
+  const int qt = n_qt - 1 - (int)blockIdx.x;   // heaviest (latest) query tiles first
+  if (qt < 0) return;                          // uniform per CTA: before any barrier or TMEM use
+  const int i0 = qt * kBM;
+  const int g = h / p.group;
+  const int row_base = p.row0[b];
+  const int key_hi = min(i0 + kBM - 1, S - 1);
+  const int key_lo = p.window > 0 ? max(0, i0 - p.window + 1) : 0;
+  const int jt_lo = key_lo / kBN;
+  const int n_tiles = key_hi / kBN - jt_lo + 1;
+
+  if (threadIdx.x == 0) {
+    mbar_init(BAR(B_Q), 1);
+    for (int s = 0; s < 2; ++s) {
+      mbar_init(BAR(B_KF + s), 1);
+      mbar_init(BAR(B_KE + s), 1);
+      mbar_init(BAR(B_VF + s), 1);
+      mbar_init(BAR(B_VE + s), 1);
+      mbar_init(BAR(B_SF + s), 1);
+      mbar_init(BAR(B_SE + s), 4);
+      mbar_init(BAR(B_PF + s), 4);
+      mbar_init(BAR(B_OF + s), 1);
+    }
+    abort_flag[0] = 0;
+    abort_flag[1] = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {  // TMEM: all 512 columns (two S buffers, two O-tile buffers)
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(smem_u32(tmem_slot)) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *tmem_slot;
+
+  if (warp == 0) {
+    // ------------------------------ TMA producer ------------------------------
+    if (lane == 0) {
+      asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_q) : "memory");
+      asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_k) : "memory");
+      asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_v) : "memory");
+      mbar_expect_tx(BAR(B_Q), kTileBytes);
+      tma_load_3d(base + kSmQ, &tm_q, 0, h, row_base + i0, BAR(B_Q));
+      tma_load_3d(base + kSmQ + kHalfBytes, &tm_q, 64, h, row_base + i0, BAR(B_Q));
+      bool ok = true;
+      int issued_k = 0, issued_v = 0;
+      for (int j = 0; j < n_tiles && ok; ++j) {
+        const int s = j & 1;
+        const int row = row_base + (jt_lo + j) * kBN;
+        if (j >= 2) ok = mbar_wait(BAR(B_KE + s), ((j >> 1) - 1) & 1, abort_flag);
+        if (!ok) break;
+        mbar_expect_tx(BAR(B_KF + s), kTileBytes);
+        tma_load_3d(base + kSmK + s * kTileBytes, &tm_k, 0, g, row, BAR(B_KF + s));
+        tma_load_3d(base + kSmK + s * kTileBytes + kHalfBytes, &tm_k, 64, g, row, BAR(B_KF + s));
+        ++issued_k;
+        if (j >= 2) ok = mbar_wait(BAR(B_VE + s), ((j >> 1) - 1) & 1, abort_flag);
+        if (!ok) break;
+        mbar_expect_tx(BAR(B_VF + s), kTileBytes);
+        tma_load_3d(base + kSmV + s * kTileBytes, &tm_v, 0, g, row, BAR(B_VF + s));
+        tma_load_3d(base + kSmV + s * kTileBytes + kHalfBytes, &tm_v, 64, g, row, BAR(B_VF + s));
+        ++issued_v;
+      }
+      if (!ok) {  // leave only after the copies already issued have landed (bounded)
+        atomicExch(p.status, kDevWaitTimeout);
+        mbar_wait(BAR(B_Q), 0, abort_flag + 1);
+        for (int back = 1; back <= 2 && issued_k - back >= 0; ++back)
+          mbar_wait(BAR(B_KF + ((issued_k - back) & 1)), ((issued_k - back) >> 1) & 1, abort_flag + 1);
+        for (int back = 1; back <= 2 && issued_v - back >= 0; ++back)
+          mbar_wait(BAR(B_VF + ((issued_v - back) & 1)), ((issued_v - back) >> 1) & 1, abort_flag + 1);
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------ MMA issuer ------------------------------
+    if (lane == 0) {
+      constexpr uint32_t kIdescS = idesc_bf16(0);
+      constexpr uint32_t kIdescPV = idesc_bf16(1);
+      bool ok = mbar_wait(BAR(B_Q), 0, abort_flag);
+      auto issue_s = [&](int j) -> bool {   // S(j) = Q K_j^T into S buffer j & 1
+        const int s = j & 1;
+        if (!mbar_wait(BAR(B_KF + s), (j >> 1) & 1, abort_flag)) return false;
+        if (j >= 2 && !mbar_wait(BAR(B_SE + s), ((j >> 1) - 1) & 1, abort_flag)) return false;
+        tc_fence_after();
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks) {   // head_dim 128 = 8 steps of 16
+          const uint32_t off = (ks >> 2) * kHalfBytes + (ks & 3) * 32;
+          umma_bf16(tmem + s * 128, smem_desc(base + kSmQ + off, 16, 1024),
+                    smem_desc(base + kSmK + s * kTileBytes + off, 16, 1024), kIdescS, ks > 0);
+        }
+        umma_commit(BAR(B_SF + s));   // scores ready
+        umma_commit(BAR(B_KE + s));   // K stage free
+        return true;
+      };
+      if (ok) ok = issue_s(0);
+      for (int j = 0; j < n_tiles && ok; ++j) {
+        if (j + 1 < n_tiles) ok = issue_s(j + 1);
+        if (!ok) break;
+        const int s = j & 1;
+        if (!mbar_wait(BAR(B_PF + s), (j >> 1) & 1, abort_flag)) { ok = false; break; }
+        if (!mbar_wait(BAR(B_VF + s), (j >> 1) & 1, abort_flag)) { ok = false; break; }
+        tc_fence_after();
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks) {   // 128 keys = 8 steps of 16
+          // A = P (K-major over keys), B = V (MN-major: channels contiguous, keys strided)
+          const uint64_t ad = smem_desc(base + kSmP + s * kTileBytes + (ks >> 2) * kHalfBytes + (ks & 3) * 32, 16, 1024);
+          const uint64_t bd = smem_desc(base + kSmV + s * kTileBytes + ks * 2048, kHalfBytes, 1024);
+          umma_bf16(tmem + 256 + s * 128, ad, bd, kIdescPV, ks > 0);
+        }
+        umma_commit(BAR(B_OF + s));   // O tile ready
+        umma_commit(BAR(B_VE + s));   // V stage (and P buffer) free
+      }
+      if (!ok) atomicExch(p.status, kDevWaitTimeout);
+    }
+  } else {
+    // ------------------------------ softmax warps ------------------------------
+    const int qd = warp & 3;              // TMEM lane quarter this warp may access
+    const int r = qd * 32 + lane;         // query row within the tile
+    const int i = i0 + r;                 // query position
+    const uint32_t lane_addr = tmem + ((uint32_t)(qd * 32) << 16);
+    float o[128];
+#pragma unroll
+    for (int e = 0; e < 128; ++e) o[e] = 0.f;
+    float m = -INFINITY, l = 0.f;
+    bool ok = true;
+    for (int j = 0; j < n_tiles; ++j) {
+      const int s = j & 1;
+      const int j0 = (jt_lo + j) * kBN;
+      if (!__all_sync(0xffffffffu, mbar_wait(BAR(B_SF + s), (j >> 1) & 1, abort_flag))) { ok = false; break; }
+      tc_fence_after();
+      // band edges: causal (keys after the query) and window (keys older than i - window)
+      const bool edge = (j0 + kBN - 1 > i0) || (p.window > 0 && j0 <= i0 + kBM - 1 - p.window);
+      const int k_max = i - j0;                                        // key column <= k_max is causal-visible
+      const int k_min = p.window > 0 ? i - p.window + 1 - j0 : -1;     // key column >= k_min is inside the window
+      uint32_t sv[32];
+      float mx = -INFINITY;
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        tmem_ld32(lane_addr + s * 128 + c * 32, sv);
+        tmem_wait_ld();
+#pragma unroll
+        for (int e = 0; e < 32; ++e) {
+          float x = __uint_as_float(sv[e]);
+          if (edge && (c * 32 + e > k_max || c * 32 + e < k_min)) x = -INFINITY;
+          mx = fmaxf(mx, x);
+        }
+      }
+      const float m_new = fmaxf(m, mx * p.scale_log2e);
+      const float m_use = m_new == -INFINITY ? 0.f : m_new;   // row with no visible key yet: weights 0, no NaN
+      const float alpha = exp2f(m - m_use);
+      float sum = 0.f;
+      unsigned char* prow = gbase + kSmP + s * kTileBytes + r * 128;
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        tmem_ld32(lane_addr + s * 128 + c * 32, sv);
+        tmem_wait_ld();
+        uint32_t pk[16];
+#pragma unroll
+        for (int e = 0; e < 32; e += 2) {
+          float x0 = __uint_as_float(sv[e]), x1 = __uint_as_float(sv[e + 1]);
+          float p0 = exp2f(x0 * p.scale_log2e - m_use), p1 = exp2f(x1 * p.scale_log2e - m_use);
+          if (edge) {
+            if (c * 32 + e > k_max || c * 32 + e < k_min) p0 = 0.f;
+            if (c * 32 + e + 1 > k_max || c * 32 + e + 1 < k_min) p1 = 0.f;
+          }
+          sum += p0 + p1;
+          pk[e >> 1] = pack_bf16(p0, p1);
+        }
+        // 32 keys = four 16-byte chunks of this row; key-half c >> 1, chunk index within the 128-byte row
+#pragma unroll
+        for (int q4 = 0; q4 < 4; ++q4) {
+          const int chunk = (c & 1) * 4 + q4;
+          *reinterpret_cast<uint4*>(prow + (c >> 1) * kHalfBytes + ((chunk ^ (r & 7)) << 4)) =
+              make_uint4(pk[q4 * 4], pk[q4 * 4 + 1], pk[q4 * 4 + 2], pk[q4 * 4 + 3]);
+        }
+      }
+      l = l * alpha + sum;
+      m = m_new;
+      // scores consumed and P written: hand both to the MMA warp
+      tc_fence_before();
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      __syncwarp();
+      if (lane == 0) {
+        mbar_arrive(BAR(B_SE + s));
+        mbar_arrive(BAR(B_PF + s));
+      }
+      // fold in the previous tile's P V while the tensor core works on this one
+      if (j > 0) {
+        const int sp = (j - 1) & 1;
+        if (!__all_sync(0xffffffffu, mbar_wait(BAR(B_OF + sp), ((j - 1) >> 1) & 1, abort_flag))) { ok = false; break; }
+        tc_fence_after();
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          tmem_ld32(lane_addr + 256 + sp * 128 + c * 32, sv);
+          tmem_wait_ld();
+#pragma unroll
+          for (int e = 0; e < 32; ++e) o[c * 32 + e] = (o[c * 32 + e] + __uint_as_float(sv[e])) * alpha;
+        }
+        tc_fence_before();
+      }
+    }
+    if (ok) {
+      const int sp = (n_tiles - 1) & 1;
+      ok = __all_sync(0xffffffffu, mbar_wait(BAR(B_OF + sp), ((n_tiles - 1) >> 1) & 1, abort_flag));
+      if (ok) {
+        tc_fence_after();
+        const float inv = 1.f / l;
+        __nv_bfloat16* orow = p.out + ((int64_t)(row_base + i) * p.n_q_heads + h) * 128;
+        uint32_t sv[32];
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          tmem_ld32(lane_addr + 256 + sp * 128 + c * 32, sv);
+          tmem_wait_ld();
+          if (i < S) {
+#pragma unroll
+            for (int q4 = 0; q4 < 4; ++q4) {
+              uint32_t w[4];
+#pragma unroll
+              for (int e = 0; e < 4; ++e) {
+                const int d = q4 * 8 + e * 2;
+                w[e] = pack_bf16((o[c * 32 + d] + __uint_as_float(sv[d])) * inv,
+                                 (o[c * 32 + d + 1] + __uint_as_float(sv[d + 1])) * inv);
+              }
+              *reinterpret_cast<uint4*>(orow + c * 32 + q4 * 8) = make_uint4(w[0], w[1], w[2], w[3]);
+            }
+          }
+        }
+        tc_fence_before();
+      }
+    }
+    if (!ok && lane == 0) atomicExch(p.status, kDevWaitTimeout);
+  }
+  // common exit: everyone is past its last TMEM access
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem) : "memory");
+  }
+#undef BAR
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (fn == nullptr) {
+    void* ptr = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPointByVersion("cuTensorMapEncodeTiled", &ptr, 12000, cudaEnableDefault, &qres) ==
+            cudaSuccess && qres == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(ptr);
+  }
+  return fn;
+}
+
+// [rows, heads, 128] bf16 tensor; box = 64 channels x 1 head x 128 rows, 128-byte swizzle
+bool make_map(CUtensorMap* map, const void* ptr, int64_t rows, int heads) {
+  EncodeTiledFn fn = encode_fn();
+  if (fn == nullptr) return false;
+  cuuint64_t dims[3] = {128, (cuuint64_t)heads, (cuuint64_t)rows};
+  cuuint64_t strides[2] = {128 * 2, (cuuint64_t)heads * 128 * 2};
+  cuuint32_t box[3] = {64, 1, 128};
+  cuuint32_t estr[3] = {1, 1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace
+
+bool prefill_tc_supported(int dtype, int head_dim, const void* q, const void* k, const void* v) {
+  auto aligned = [](const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; };
+  return dtype == MIXATTN_BF16 && head_dim == 128 && aligned(q) && aligned(k) && aligned(v) && encode_fn() != nullptr;
+}
+
+cudaError_t prepare_prefill_tc() {
+  return cudaFuncSetAttribute(prefill_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+}
+
+cudaError_t launch_prefill_tc(const PrefillParams& pp, int max_len, cudaStream_t st) {
+  if (pp.n_seqs <= 0 || max_len <= 0) return cudaSuccess;
+  const int64_t rows = pp.row0[pp.n_seqs];
+  CUtensorMap tq, tk, tv;
+  if (!make_map(&tq, pp.q, rows, pp.n_q_heads) || !make_map(&tk, pp.k, rows, pp.n_kv_heads) ||
+      !make_map(&tv, pp.v, rows, pp.n_kv_heads))
+    return cudaErrorInvalidValue;
+  TcParams p;
+  p.n_q_heads = pp.n_q_heads;
+  p.group = pp.n_q_heads / pp.n_kv_heads;
+  p.window = pp.window;
+  p.n_seqs = pp.n_seqs;
+  p.scale_log2e = pp.scale_log2e;
+  p.status = pp.status;
+  p.out = static_cast<__nv_bfloat16*>(pp.out);
+  for (int i = 0; i <= pp.n_seqs; ++i) p.row0[i] = pp.row0[i];
+  dim3 grid((max_len + kBM - 1) / kBM, pp.n_q_heads, pp.n_seqs);
+  prefill_tc_kernel<<<grid, kThreads, kSmemBytes, st>>>(tq, tk, tv, p);
+  return cudaGetLastError();
+}
+
+}  // namespace mixattn
