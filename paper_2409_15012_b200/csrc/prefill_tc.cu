@@ -8,11 +8,12 @@
 //   warp 0   TMA producer: Q once, then K (2 stages) and V (2 stages) tiles as
 //            128B-swizzled [128 x 64] boxes straight from the caller's tensors
 //   warp 1   one elected thread issues tcgen05.mma: S = Q K^T into TMEM (two S buffers),
-//            O_tile = P V into TMEM (two buffers), each 128 x 128 fp32
+//            O += P V into TMEM (128 x 128 fp32 each)
 //   warps 2-5  softmax: thread r owns query row r (TMEM lane r); reads S with
 //            tcgen05.ld, masks band edges, online softmax in base 2 (fp32), writes P
-//            (bf16) into shared memory in the swizzled K-major layout the MMA reads,
-//            accumulates O in registers (O = O * alpha + O_tile), normalises and stores.
+//            (bf16) into shared memory in the swizzled K-major layout the MMA reads.
+//            O stays in TMEM; its rows are rescaled lazily (only when the running max
+//            grew by more than 2^8), then normalised and stored at the end.
 //
 // S(j+1) is issued before P V(j), so the tensor core works on the next scores while the
 // softmax warps are busy.  All mbarrier waits are bounded; on time-out a status word is
@@ -117,6 +118,22 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
         "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
         "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
       : "r"(taddr));
+}
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,"
+      "%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};"
+      ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+        "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]),
+        "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]),
+        "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+      : "memory");
+}
+__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ float ex2_approx(float x) {   // 2^x, single MUFU op; 2^-inf = 0
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
 }
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
@@ -251,7 +268,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
           // A = P (K-major over keys), B = V (MN-major: channels contiguous, keys strided)
           const uint64_t ad = smem_desc(base + kSmP + s * kTileBytes + (ks >> 2) * kHalfBytes + (ks & 3) * 32, 16, 1024);
           const uint64_t bd = smem_desc(base + kSmV + s * kTileBytes + ks * 2048, kHalfBytes, 1024);
-          umma_bf16(tmem + 256 + s * 128, ad, bd, kIdescPV, ks > 0);
+          umma_bf16(tmem + 256, ad, bd, kIdescPV, (j > 0 || ks > 0) ? 1u : 0u);
         }
         umma_commit(BAR(B_OF + s));   // O tile ready
         umma_commit(BAR(B_VE + s));   // V stage (and P buffer) free
@@ -264,86 +281,89 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     const int r = qd * 32 + lane;         // query row within the tile
     const int i = i0 + r;                 // query position
     const uint32_t lane_addr = tmem + ((uint32_t)(qd * 32) << 16);
-    float o[128];
-#pragma unroll
-    for (int e = 0; e < 128; ++e) o[e] = 0.f;
-    float m = -INFINITY, l = 0.f;
+    // O stays in TMEM and P V accumulates into it.  m_ref is the exponent reference of the
+    // row: it follows the running max lazily (only when the max grew by more than
+    // kRescaleGap, in log2 units), so the read-scale-write of the O row is rare.
+    constexpr float kRescaleGap = 8.f;
+    float m_ref = -INFINITY, l = 0.f;
     bool ok = true;
     for (int j = 0; j < n_tiles; ++j) {
       const int s = j & 1;
       const int j0 = (jt_lo + j) * kBN;
       if (!__all_sync(0xffffffffu, mbar_wait(BAR(B_SF + s), (j >> 1) & 1, abort_flag))) { ok = false; break; }
       tc_fence_after();
+      uint32_t sv[128];
+      tmem_ld32(lane_addr + s * 128, *reinterpret_cast<uint32_t(*)[32]>(&sv[0]));
+      tmem_ld32(lane_addr + s * 128 + 32, *reinterpret_cast<uint32_t(*)[32]>(&sv[32]));
+      tmem_ld32(lane_addr + s * 128 + 64, *reinterpret_cast<uint32_t(*)[32]>(&sv[64]));
+      tmem_ld32(lane_addr + s * 128 + 96, *reinterpret_cast<uint32_t(*)[32]>(&sv[96]));
+      tmem_wait_ld();
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(BAR(B_SE + s));   // scores are in registers: the S buffer is free
       // band edges: causal (keys after the query) and window (keys older than i - window)
       const bool edge = (j0 + kBN - 1 > i0) || (p.window > 0 && j0 <= i0 + kBM - 1 - p.window);
-      const int k_max = i - j0;                                        // key column <= k_max is causal-visible
-      const int k_min = p.window > 0 ? i - p.window + 1 - j0 : -1;     // key column >= k_min is inside the window
-      uint32_t sv[32];
-      float mx = -INFINITY;
+      if (edge) {
+        const int k_max = i - j0;                                      // columns <= k_max are causal-visible
+        const int k_min = p.window > 0 ? i - p.window + 1 - j0 : 0;    // columns >= k_min are inside the window
 #pragma unroll
-      for (int c = 0; c < 4; ++c) {
-        tmem_ld32(lane_addr + s * 128 + c * 32, sv);
-        tmem_wait_ld();
-#pragma unroll
-        for (int e = 0; e < 32; ++e) {
-          float x = __uint_as_float(sv[e]);
-          if (edge && (c * 32 + e > k_max || c * 32 + e < k_min)) x = -INFINITY;
-          mx = fmaxf(mx, x);
-        }
+        for (int e = 0; e < 128; ++e)
+          if (e > k_max || e < k_min) sv[e] = 0xff800000u;             // -inf
       }
-      const float m_new = fmaxf(m, mx * p.scale_log2e);
-      const float m_use = m_new == -INFINITY ? 0.f : m_new;   // row with no visible key yet: weights 0, no NaN
-      const float alpha = exp2f(m - m_use);
-      float sum = 0.f;
+      float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
+#pragma unroll
+      for (int e = 0; e < 128; e += 4) {
+        mx0 = fmaxf(mx0, __uint_as_float(sv[e]));
+        mx1 = fmaxf(mx1, __uint_as_float(sv[e + 1]));
+        mx2 = fmaxf(mx2, __uint_as_float(sv[e + 2]));
+        mx3 = fmaxf(mx3, __uint_as_float(sv[e + 3]));
+      }
+      const float mt = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * p.scale_log2e;
+      const bool grow = mt > m_ref + kRescaleGap;    // also true for the first visible key (m_ref = -inf)
+      if (__any_sync(0xffffffffu, grow)) {
+        const float alpha = grow ? ex2_approx(m_ref - mt) : 1.f;   // m_ref = -inf gives 0
+        if (j > 0) {   // the O row holds earlier tiles: rescale it once P V(j-1) has landed
+          const int sp = (j - 1) & 1;
+          if (!__all_sync(0xffffffffu, mbar_wait(BAR(B_OF + sp), ((j - 1) >> 1) & 1, abort_flag))) { ok = false; break; }
+          tc_fence_after();
+#pragma unroll
+          for (int c = 0; c < 4; ++c) {
+            uint32_t ov[32];
+            tmem_ld32(lane_addr + 256 + c * 32, ov);
+            tmem_wait_ld();
+#pragma unroll
+            for (int e = 0; e < 32; ++e) ov[e] = __float_as_uint(__uint_as_float(ov[e]) * alpha);
+            tmem_st32(lane_addr + 256 + c * 32, ov);
+          }
+          tmem_wait_st();
+        }
+        l *= alpha;
+        if (grow) m_ref = mt;
+      }
+      const float neg_m = m_ref == -INFINITY ? 0.f : -m_ref;   // row with no visible key yet: weights 0, no NaN
+      float sum0 = 0.f, sum1 = 0.f;
+      uint32_t pk[64];
+#pragma unroll
+      for (int e = 0; e < 128; e += 2) {
+        const float p0 = ex2_approx(fmaf(__uint_as_float(sv[e]), p.scale_log2e, neg_m));
+        const float p1 = ex2_approx(fmaf(__uint_as_float(sv[e + 1]), p.scale_log2e, neg_m));
+        sum0 += p0;
+        sum1 += p1;
+        pk[e >> 1] = pack_bf16(p0, p1);
+      }
+      l += sum0 + sum1;
+      // the P buffer was last read by P V(j-2)
+      if (j >= 2 && !__all_sync(0xffffffffu, mbar_wait(BAR(B_OF + s), ((j >> 1) - 1) & 1, abort_flag))) { ok = false; break; }
       unsigned char* prow = gbase + kSmP + s * kTileBytes + r * 128;
 #pragma unroll
-      for (int c = 0; c < 4; ++c) {
-        tmem_ld32(lane_addr + s * 128 + c * 32, sv);
-        tmem_wait_ld();
-        uint32_t pk[16];
-#pragma unroll
-        for (int e = 0; e < 32; e += 2) {
-          float x0 = __uint_as_float(sv[e]), x1 = __uint_as_float(sv[e + 1]);
-          float p0 = exp2f(x0 * p.scale_log2e - m_use), p1 = exp2f(x1 * p.scale_log2e - m_use);
-          if (edge) {
-            if (c * 32 + e > k_max || c * 32 + e < k_min) p0 = 0.f;
-            if (c * 32 + e + 1 > k_max || c * 32 + e + 1 < k_min) p1 = 0.f;
-          }
-          sum += p0 + p1;
-          pk[e >> 1] = pack_bf16(p0, p1);
-        }
-        // 32 keys = four 16-byte chunks of this row; key-half c >> 1, chunk index within the 128-byte row
-#pragma unroll
-        for (int q4 = 0; q4 < 4; ++q4) {
-          const int chunk = (c & 1) * 4 + q4;
-          *reinterpret_cast<uint4*>(prow + (c >> 1) * kHalfBytes + ((chunk ^ (r & 7)) << 4)) =
-              make_uint4(pk[q4 * 4], pk[q4 * 4 + 1], pk[q4 * 4 + 2], pk[q4 * 4 + 3]);
-        }
+      for (int c16 = 0; c16 < 16; ++c16) {   // 16-byte chunks of 8 keys; key-half c16 >> 3
+        *reinterpret_cast<uint4*>(prow + (c16 >> 3) * kHalfBytes + (((c16 & 7) ^ (r & 7)) << 4)) =
+            make_uint4(pk[c16 * 4], pk[c16 * 4 + 1], pk[c16 * 4 + 2], pk[c16 * 4 + 3]);
       }
-      l = l * alpha + sum;
-      m = m_new;
-      // scores consumed and P written: hand both to the MMA warp
       tc_fence_before();
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
       __syncwarp();
-      if (lane == 0) {
-        mbar_arrive(BAR(B_SE + s));
-        mbar_arrive(BAR(B_PF + s));
-      }
-      // fold in the previous tile's P V while the tensor core works on this one
-      if (j > 0) {
-        const int sp = (j - 1) & 1;
-        if (!__all_sync(0xffffffffu, mbar_wait(BAR(B_OF + sp), ((j - 1) >> 1) & 1, abort_flag))) { ok = false; break; }
-        tc_fence_after();
-#pragma unroll
-        for (int c = 0; c < 4; ++c) {
-          tmem_ld32(lane_addr + 256 + sp * 128 + c * 32, sv);
-          tmem_wait_ld();
-#pragma unroll
-          for (int e = 0; e < 32; ++e) o[c * 32 + e] = (o[c * 32 + e] + __uint_as_float(sv[e])) * alpha;
-        }
-        tc_fence_before();
-      }
+      if (lane == 0) mbar_arrive(BAR(B_PF + s));
     }
     if (ok) {
       const int sp = (n_tiles - 1) & 1;
@@ -352,21 +372,18 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         tc_fence_after();
         const float inv = 1.f / l;
         __nv_bfloat16* orow = p.out + ((int64_t)(row_base + i) * p.n_q_heads + h) * 128;
-        uint32_t sv[32];
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
-          tmem_ld32(lane_addr + 256 + sp * 128 + c * 32, sv);
+          uint32_t ov[32];
+          tmem_ld32(lane_addr + 256 + c * 32, ov);
           tmem_wait_ld();
           if (i < S) {
 #pragma unroll
             for (int q4 = 0; q4 < 4; ++q4) {
               uint32_t w[4];
 #pragma unroll
-              for (int e = 0; e < 4; ++e) {
-                const int d = q4 * 8 + e * 2;
-                w[e] = pack_bf16((o[c * 32 + d] + __uint_as_float(sv[d])) * inv,
-                                 (o[c * 32 + d + 1] + __uint_as_float(sv[d + 1])) * inv);
-              }
+              for (int e = 0; e < 4; ++e)
+                w[e] = pack_bf16(__uint_as_float(ov[q4 * 8 + e * 2]) * inv, __uint_as_float(ov[q4 * 8 + e * 2 + 1]) * inv);
               *reinterpret_cast<uint4*>(orow + c * 32 + q4 * 8) = make_uint4(w[0], w[1], w[2], w[3]);
             }
           }
