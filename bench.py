@@ -80,7 +80,7 @@ class ClockSampler:
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
-                 "-i", str(self.index), "-lms", "100"],
+                 "-i", str(self.index), "-lms", "20"],
                 stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
@@ -247,7 +247,7 @@ def run_gpu_arm(args, wl):
     from paper_2409_15012_b200 import binding as mx, runner
     peaks = load_peaks()
     K, Wm = args.steps, args.warmup
-    total_steps = 2 * (K + Wm) + K + 2       # device-timed pass, e2e pass, profiled pass
+    total_steps = 2 * (K + Wm) + min(K, 20) + 2       # device-timed pass, e2e pass, profiled pass
 
     if wl.context_range != (0, 0):
         lengths = si.draw_lengths(wl.seed, wl.batch, *wl.context_range).tolist()
@@ -271,14 +271,17 @@ def run_gpu_arm(args, wl):
         return runner.kv_bytes_per_step(wl, [int(p) + 1 for p in sess.pos])
 
     # ---- device-resident pass: `value` ----
+    # step inputs: a ring of kRing distinct seeded steps reused cyclically (the values do not
+    # change the work; positions, appends and lengths advance every step as in serving)
+    kRing = min(8, Wm + K)
     step_inputs = []
     pos_save = sess.pos.copy()
-    for s in range(Wm + K):
+    for s in range(kRing):
         step_inputs.append(sess.step_inputs())
         sess.pos += 1
     sess.pos[:] = pos_save
     for s in range(Wm):
-        sess.decode_step(step_inputs[s], outs, stream)
+        sess.decode_step(step_inputs[s % kRing], outs, stream)
     launches0 = sess.ctx.get_launch_count()
     sampler = ClockSampler(local)
     if rank == 0:
@@ -289,7 +292,7 @@ def run_gpu_arm(args, wl):
     ev0.record(stream)
     for s in range(K):
         kv_bytes += bytes_next_step()
-        sess.decode_step(step_inputs[Wm + s], outs, stream)
+        sess.decode_step(step_inputs[(Wm + s) % kRing], outs, stream)
     ev1.record(stream)
     barrier()
     ms = ev0.elapsed_time(ev1)
@@ -300,18 +303,15 @@ def run_gpu_arm(args, wl):
     # ---- end-to-end pass: host inputs, host outputs ----
     host_inputs = []
     pos_save = sess.pos.copy()
-    for s in range(Wm + K):
-        ent = sess.step_inputs()
-        host_inputs.append({l: {k: t.cpu().pin_memory() for k, t in d.items()} for l, d in ent.items()})
-        sess.pos += 1
-    sess.pos[:] = pos_save
+    for s in range(kRing):
+        host_inputs.append({l: {k: t.cpu().pin_memory() for k, t in d.items()} for l, d in step_inputs[s].items()})
     dev_buf = {l: {k: torch.empty_like(t, device=sess.dev) for k, t in d.items()} for l, d in host_inputs[0].items()}
     host_out = torch.empty(outs.shape, dtype=outs.dtype).pin_memory()
     h2d = sum(t.numel() * t.element_size() for d in host_inputs[0].values() for t in d.values())
     d2h = outs.numel() * outs.element_size()
 
     def e2e_step(s):
-        for l, d in host_inputs[s].items():
+        for l, d in host_inputs[s % kRing].items():
             for k, t in d.items():
                 dev_buf[l][k].copy_(t, non_blocking=True)
         sess.decode_step(dev_buf, outs, stream)
@@ -338,10 +338,10 @@ def run_gpu_arm(args, wl):
     per_tok = 2 * wl.n_kv_heads * wl.head_dim * e
     sess.ctx.profile_enable(True)
     full_bytes = 0
-    for s in range(K):
-        ent = sess.step_inputs()
+    Kp = min(K, 20)
+    for s in range(Kp):
         full_bytes += sum(int(p) + 1 for p in sess.pos) * per_tok
-        sess.decode_step(ent, outs, stream)
+        sess.decode_step(step_inputs[s % kRing], outs, stream)
     n_full, ms_full = sess.ctx.profile_read(mx.K_DECODE_FULL)
     n_slide, ms_slide = sess.ctx.profile_read(mx.K_DECODE_SLIDING)
     n_comb, ms_comb = sess.ctx.profile_read(mx.K_COMBINE)
@@ -363,7 +363,7 @@ def run_gpu_arm(args, wl):
 
     value = kv_bytes / (ms * 1e-3) / 1e9
     # achieved = bytes per launch / seconds per launch
-    bytes_per_launch = full_bytes / K if K else 0
+    bytes_per_launch = full_bytes / Kp if Kp else 0
     sec_per_launch = ms_full / max(n_full, 1) * 1e-3
     achieved = bytes_per_launch / sec_per_launch / 1e9
     roofline = {
@@ -424,7 +424,7 @@ def run_gpu_arm(args, wl):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="mid_decode",

@@ -93,8 +93,8 @@ class Session:
         out: Dict[int, Dict[str, torch.Tensor]] = {}
         B = wl.batch
         for l in range(len(wl.layout)):
-            q = torch.stack([si.q_tokens(wl.seed, l, b, int(self.pos[b]), 1, wl.n_q_heads, wl.head_dim,
-                                         self.dt, device)[0] for b in range(B)])
+            q = si.q_tokens_multi(wl.seed, l, list(range(B)), [int(p) for p in self.pos], 1, wl.n_q_heads,
+                                  wl.head_dim, self.dt, device)[:, 0].contiguous()
             ent = {"q": q}
             if l in self.owners:
                 K, V = si.kv_tokens_multi(wl.seed, l, list(range(B)), [int(p) for p in self.pos], 1,
@@ -128,8 +128,8 @@ class Session:
         device = self.dev if device is None else device
         owner = wl.layout[layer][2]
         S = wl.seq_len
-        q = torch.cat([si.q_tokens(wl.seed, layer, b, 0, S, wl.n_q_heads, wl.head_dim, self.dt, device)
-                       for b in range(wl.batch)])
+        q = si.q_tokens_multi(wl.seed, layer, list(range(wl.batch)), [0] * wl.batch, S, wl.n_q_heads,
+                              wl.head_dim, self.dt, device).reshape(-1, wl.n_q_heads, wl.head_dim)
         K, V = si.kv_tokens_multi(wl.seed, owner, list(range(wl.batch)), [0] * wl.batch, S,
                                   wl.n_kv_heads, wl.head_dim, self.dt, device)
         return q, K.reshape(-1, wl.n_kv_heads, wl.head_dim), V.reshape(-1, wl.n_kv_heads, wl.head_dim)

@@ -112,6 +112,17 @@ def q_tokens(seed, layer, seq, pos0, n, n_q_heads, head_dim, dtype, device="cpu"
     return _block(key, pos0 * per_tok, (n, n_q_heads, head_dim), dtype, device)
 
 
+def q_tokens_multi(seed, layer, seqs, pos0s, n, n_q_heads, head_dim, dtype, device="cpu"):
+    """Same values as q_tokens for several sequences at once:
+    [len(seqs), n, n_q_heads, head_dim]."""
+    per_tok = n_q_heads * head_dim
+    keys = torch.tensor([stream_key(seed, _STREAM_Q, layer, int(s)) for s in seqs],
+                        dtype=torch.int64, device=device).view(-1, 1)
+    first = torch.tensor([int(p) * per_tok for p in pos0s], dtype=torch.int64, device=device).view(-1, 1)
+    idx = first + torch.arange(n * per_tok, dtype=torch.int64, device=device).view(1, -1)
+    return unit_normal(keys, idx).to(dtype).reshape(len(seqs), n, n_q_heads, head_dim)
+
+
 def draw_lengths(seed: int, n: int, lo: int, hi: int) -> np.ndarray:
     """n integers uniform on [lo, hi], both ends included."""
     return np.random.default_rng(seed).integers(lo, hi + 1, size=n).astype(np.int64)

@@ -54,3 +54,6 @@ def test_multi_and_head_variants_agree():
     assert torch.equal(Km[0], si.kv_tokens(3, 1, 2, 0, 6, 2, 16, torch.bfloat16)[0])
     Kh, Vh = si.kv_tokens_head(3, 1, 4, 10, 6, 2, 16, 1, torch.bfloat16)
     assert torch.equal(Kh, K[:, 1]) and torch.equal(Vh, V[:, 1])
+    qm = si.q_tokens_multi(3, 2, [2, 4], [5, 10], 3, 4, 16, torch.bfloat16)
+    assert torch.equal(qm[1], si.q_tokens(3, 2, 4, 10, 3, 4, 16, torch.bfloat16))
+    assert torch.equal(qm[0], si.q_tokens(3, 2, 2, 5, 3, 4, 16, torch.bfloat16))
