@@ -40,9 +40,12 @@ from synth import inputs as si
 METRIC = "decode attention HBM GB/s (% of peak) & tokens/s; prefill TFLOP/s (% bf16 peak)"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel from an
-# ncu capture (profiles/); None until captured for the current kernel
-DECODE_FULL_TRAFFIC_BYTES = None
+# (dram__bytes_read.sum + dram__bytes_write.sum) / algorithmic KV bytes of the dominant kernel, from the
+# ncu capture of a batch-4 launch summarised in profiles/decode_split_bf16_kernel.mid_decode.md
+# (541.39 MB moved for 536.95 MB of keys and values).  DRAM traffic grows in proportion to the keys read,
+# so the full-size figure is this ratio times the launch's algorithmic bytes.  Set to None when the
+# kernel changes until the counters are taken again.
+DECODE_FULL_TRAFFIC_RATIO = 541.389056 / 536.952832
 
 
 def load_peaks():
@@ -369,7 +372,8 @@ def run_gpu_arm(args, wl):
     roofline = {
         "kernel": "decode_split_bf16_kernel (standard layer)" if wl.dtype == cf.BF16 else "decode_split_f32_kernel",
         "bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-        "frac": achieved / peaks["hbm_gbs"], "traffic": DECODE_FULL_TRAFFIC_BYTES,
+        "frac": achieved / peaks["hbm_gbs"],
+        "traffic": None if DECODE_FULL_TRAFFIC_RATIO is None else DECODE_FULL_TRAFFIC_RATIO * bytes_per_launch,
         "peak_source": f"of {peaks['_source']}", "bytes_per_launch": bytes_per_launch,
         "us_per_launch": sec_per_launch * 1e6, "frac_of_nominal_8TBs": achieved / 8000.0,
     }
