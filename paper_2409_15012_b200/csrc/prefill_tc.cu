@@ -106,6 +106,15 @@ __device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t adesc, uint6
       "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
       ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
 }
+// Same with the A operand in tensor memory (rows = lanes, two bf16 per 32-bit column).
+__device__ __forceinline__ void umma_bf16_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc, uint32_t idesc,
+                                             uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
@@ -266,9 +275,8 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
 #pragma unroll
         for (int ks = 0; ks < 8; ++ks) {   // 128 keys = 8 steps of 16
           // A = P (K-major over keys), B = V (MN-major: channels contiguous, keys strided)
-          const uint64_t ad = smem_desc(base + kSmP + s * kTileBytes + (ks >> 2) * kHalfBytes + (ks & 3) * 32, 16, 1024);
           const uint64_t bd = smem_desc(base + kSmV + s * kTileBytes + ks * 2048, kHalfBytes, 1024);
-          umma_bf16(tmem + 256, ad, bd, kIdescPV, (j > 0 || ks > 0) ? 1u : 0u);
+          umma_bf16_ts(tmem + 256, tmem + 384 + s * 64 + ks * 8, bd, kIdescPV, (j > 0 || ks > 0) ? 1u : 0u);
         }
         umma_commit(BAR(B_OF + s));   // O tile ready
         umma_commit(BAR(B_VE + s));   // V stage (and P buffer) free
@@ -354,14 +362,11 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
       l += sum0 + sum1;
       // the P buffer was last read by P V(j-2)
       if (j >= 2 && !__all_sync(0xffffffffu, mbar_wait(BAR(B_OF + s), ((j >> 1) - 1) & 1, abort_flag))) { ok = false; break; }
-      unsigned char* prow = gbase + kSmP + s * kTileBytes + r * 128;
-#pragma unroll
-      for (int c16 = 0; c16 < 16; ++c16) {   // 16-byte chunks of 8 keys; key-half c16 >> 3
-        *reinterpret_cast<uint4*>(prow + (c16 >> 3) * kHalfBytes + (((c16 & 7) ^ (r & 7)) << 4)) =
-            make_uint4(pk[c16 * 4], pk[c16 * 4 + 1], pk[c16 * 4 + 2], pk[c16 * 4 + 3]);
-      }
+      // P (bf16 pairs) into tensor memory: columns 384 + 64 s .. of this row
+      tmem_st32(lane_addr + 384 + s * 64, *reinterpret_cast<uint32_t(*)[32]>(&pk[0]));
+      tmem_st32(lane_addr + 384 + s * 64 + 32, *reinterpret_cast<uint32_t(*)[32]>(&pk[32]));
+      tmem_wait_st();
       tc_fence_before();
-      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
       __syncwarp();
       if (lane == 0) mbar_arrive(BAR(B_PF + s));
     }
