@@ -5,18 +5,25 @@
 // one CTA owns a 128-query tile of one (sequence, head) and walks the 128-key tiles that
 // intersect its band; tiles wholly outside the band are never loaded.
 //
-//   warp 0   TMA producer: Q once, then K (2 stages) and V (2 stages) tiles as
-//            128B-swizzled [128 x 64] boxes straight from the caller's tensors
-//   warp 1   one elected thread issues tcgen05.mma: S = Q K^T into TMEM (two S buffers),
-//            O += P V into TMEM (128 x 128 fp32 each)
-//   warps 2-5  softmax: thread r owns query row r (TMEM lane r); reads S with
-//            tcgen05.ld, masks band edges, online softmax in base 2 (fp32), writes P
-//            (bf16) into shared memory in the swizzled K-major layout the MMA reads.
-//            O stays in TMEM; its rows are rescaled lazily (only when the running max
-//            grew by more than 2^8), then normalised and stored at the end.
+// One CTA owns TWO 128-query tiles that share their K/V band: the same query positions of
+// two query heads of one KV head (grouped-query attention), so every K/V tile staged in
+// shared memory feeds two S products and two P V products.
 //
-// S(j+1) is issued before P V(j), so the tensor core works on the next scores while the
-// softmax warps are busy.  All mbarrier waits are bounded; on time-out a status word is
+//   warp 0     TMA producer: both Q tiles once, then K (2 stages) and V (2 stages) tiles as
+//              128B-swizzled [128 x 64] boxes straight from the caller's tensors
+//   warp 1     one elected thread issues tcgen05.mma (M128 N128 K16, bf16 -> fp32 in TMEM):
+//              S_t = Q_t K^T (both operands from shared memory) and O_t += P_t V with P_t
+//              read from tensor memory and V MN-major from its row-major tile
+//   warps 2-5  softmax of tile A, warps 6-9 softmax of tile B: thread r owns query row r
+//              (TMEM lane r): tcgen05.ld of the S row, band masks on edge tiles only,
+//              base-2 online softmax with one MUFU ex2 per score, P written back as bf16
+//              pairs over the first 64 columns of the S row (tcgen05.st).  O stays in TMEM;
+//              its rows are rescaled lazily (only when the running max grew by more than
+//              2^8), normalised and stored at the end.
+//
+// The two tiles ping-pong: while one group computes exponentials, the tensor core runs the
+// other tile's P V and next S, and the other group loads or stores.  TMEM: S_A, S_B, O_A,
+// O_B = 4 x 128 columns.  All mbarrier waits are bounded; on time-out a status word is
 // raised, every role leaves its loop, and TMEM is released at the common exit.
 #include <cuda.h>
 #include <cuda_bf16.h>
@@ -27,21 +34,21 @@ namespace mixattn {
 
 namespace {
 
-constexpr int kBM = 128;                       // queries per CTA
+constexpr int kBM = 128;                       // queries per tile (two tiles per CTA)
 constexpr int kBN = 128;                       // keys per tile
 constexpr int kHalfBytes = 128 * 128;          // one [128 rows x 64 bf16] swizzled block
 constexpr int kTileBytes = 2 * kHalfBytes;     // a 128 x 128 bf16 operand tile
-constexpr int kThreads = 192;
-constexpr int kSmQ = 0;
-constexpr int kSmK = kSmQ + kTileBytes;        // 2 stages
+constexpr int kThreads = 320;                  // TMA warp, MMA warp, 2 x 4 softmax warps
+constexpr int kSmQ = 0;                        // Q_A, Q_B
+constexpr int kSmK = kSmQ + 2 * kTileBytes;    // 2 stages
 constexpr int kSmV = kSmK + 2 * kTileBytes;    // 2 stages
-constexpr int kSmP = kSmV + 2 * kTileBytes;    // 2 buffers
-constexpr int kSmBar = kSmP + 2 * kTileBytes;  // barriers, TMEM pointer, abort flag
+constexpr int kSmBar = kSmV + 2 * kTileBytes;  // barriers, TMEM pointer, abort flag
 constexpr int kSmemBytes = kSmBar + 256 + 1024;  // + slack to align the base to 1024 B
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;
+constexpr uint32_t kColS = 0, kColO = 256;     // TMEM columns: S_t at 128 t, O_t at 256 + 128 t
 
-// barrier indices
-enum { B_Q = 0, B_KF = 1, B_KE = 3, B_VF = 5, B_VE = 7, B_SF = 9, B_SE = 11, B_PF = 13, B_OF = 15, B_N = 17 };
+// barrier indices (two each: K/V stages, or tile A / tile B)
+enum { B_Q = 0, B_KF = 1, B_KE = 3, B_VF = 5, B_VE = 7, B_SF = 9, B_PF = 11, B_OF = 13, B_N = 15 };
 
 struct TcParams {
   int32_t n_q_heads, group, window, n_seqs;
@@ -169,13 +176,17 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
 #define BAR(i) (bar0 + 8u * (i))
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int b = blockIdx.z, h = blockIdx.y;
+  const int b = blockIdx.z;
+  const int pairs_per_group = (p.group + 1) >> 1;
+  const int g = blockIdx.y / pairs_per_group;                 // KV head
+  const int hA = g * p.group + (blockIdx.y % pairs_per_group) * 2;
+  const bool has_b = (hA + 1) < (g + 1) * p.group;            // odd group size: last pair is a single
+  const int n_act = has_b ? 2 : 1;
   const int S = p.row0[b + 1] - p.row0[b];
   const int n_qt = (S + kBM - 1) / kBM;
   const int qt = n_qt - 1 - (int)blockIdx.x;   // heaviest (latest) query tiles first
   if (qt < 0) return;                          // uniform per CTA: before any barrier or TMEM use
   const int i0 = qt * kBM;
-  const int g = h / p.group;
   const int row_base = p.row0[b];
   const int key_hi = min(i0 + kBM - 1, S - 1);
   const int key_lo = p.window > 0 ? max(0, i0 - p.window + 1) : 0;
@@ -190,7 +201,6 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
       mbar_init(BAR(B_VF + s), 1);
       mbar_init(BAR(B_VE + s), 1);
       mbar_init(BAR(B_SF + s), 1);
-      mbar_init(BAR(B_SE + s), 4);
       mbar_init(BAR(B_PF + s), 4);
       mbar_init(BAR(B_OF + s), 1);
     }
@@ -198,7 +208,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     abort_flag[1] = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  if (warp == 1) {  // TMEM: all 512 columns (two S buffers, two O-tile buffers)
+  if (warp == 1) {  // TMEM: all 512 columns
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(smem_u32(tmem_slot)) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
@@ -213,9 +223,11 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
       asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_q) : "memory");
       asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_k) : "memory");
       asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_v) : "memory");
-      mbar_expect_tx(BAR(B_Q), kTileBytes);
-      tma_load_3d(base + kSmQ, &tm_q, 0, h, row_base + i0, BAR(B_Q));
-      tma_load_3d(base + kSmQ + kHalfBytes, &tm_q, 64, h, row_base + i0, BAR(B_Q));
+      mbar_expect_tx(BAR(B_Q), n_act * kTileBytes);
+      for (int t = 0; t < n_act; ++t) {
+        tma_load_3d(base + kSmQ + t * kTileBytes, &tm_q, 0, hA + t, row_base + i0, BAR(B_Q));
+        tma_load_3d(base + kSmQ + t * kTileBytes + kHalfBytes, &tm_q, 64, hA + t, row_base + i0, BAR(B_Q));
+      }
       bool ok = true;
       int issued_k = 0, issued_v = 0;
       for (int j = 0; j < n_tiles && ok; ++j) {
@@ -249,66 +261,82 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
       constexpr uint32_t kIdescS = idesc_bf16(0);
       constexpr uint32_t kIdescPV = idesc_bf16(1);
       bool ok = mbar_wait(BAR(B_Q), 0, abort_flag);
-      auto issue_s = [&](int j) -> bool {   // S(j) = Q K_j^T into S buffer j & 1
+      // S_t(j) = Q_t K_j^T into the S columns of tile t (which also hold P_t(j-1): the
+      // tensor pipe runs this thread's MMAs in order, so P V_t(j-1) has read it by then)
+      auto issue_s = [&](int t, int j) {
         const int s = j & 1;
-        if (!mbar_wait(BAR(B_KF + s), (j >> 1) & 1, abort_flag)) return false;
-        if (j >= 2 && !mbar_wait(BAR(B_SE + s), ((j >> 1) - 1) & 1, abort_flag)) return false;
-        tc_fence_after();
 #pragma unroll
         for (int ks = 0; ks < 8; ++ks) {   // head_dim 128 = 8 steps of 16
           const uint32_t off = (ks >> 2) * kHalfBytes + (ks & 3) * 32;
-          umma_bf16(tmem + s * 128, smem_desc(base + kSmQ + off, 16, 1024),
+          umma_bf16(tmem + kColS + t * 128, smem_desc(base + kSmQ + t * kTileBytes + off, 16, 1024),
                     smem_desc(base + kSmK + s * kTileBytes + off, 16, 1024), kIdescS, ks > 0);
         }
-        umma_commit(BAR(B_SF + s));   // scores ready
-        umma_commit(BAR(B_KE + s));   // K stage free
-        return true;
+        umma_commit(BAR(B_SF + t));
       };
-      if (ok) ok = issue_s(0);
-      for (int j = 0; j < n_tiles && ok; ++j) {
-        if (j + 1 < n_tiles) ok = issue_s(j + 1);
-        if (!ok) break;
+      // O_t += P_t(j) V_j: A = P from tensor memory (two bf16 per column), B = V MN-major
+      auto issue_pv = [&](int t, int j) {
         const int s = j & 1;
-        if (!mbar_wait(BAR(B_PF + s), (j >> 1) & 1, abort_flag)) { ok = false; break; }
-        if (!mbar_wait(BAR(B_VF + s), (j >> 1) & 1, abort_flag)) { ok = false; break; }
-        tc_fence_after();
 #pragma unroll
         for (int ks = 0; ks < 8; ++ks) {   // 128 keys = 8 steps of 16
-          // A = P (K-major over keys), B = V (MN-major: channels contiguous, keys strided)
           const uint64_t bd = smem_desc(base + kSmV + s * kTileBytes + ks * 2048, kHalfBytes, 1024);
-          umma_bf16_ts(tmem + 256, tmem + 384 + s * 64 + ks * 8, bd, kIdescPV, (j > 0 || ks > 0) ? 1u : 0u);
+          umma_bf16_ts(tmem + kColO + t * 128, tmem + kColS + t * 128 + ks * 8, bd, kIdescPV,
+                       (j > 0 || ks > 0) ? 1u : 0u);
         }
-        umma_commit(BAR(B_OF + s));   // O tile ready
-        umma_commit(BAR(B_VE + s));   // V stage (and P buffer) free
+        umma_commit(BAR(B_OF + t));
+      };
+      if (ok) ok = mbar_wait(BAR(B_KF + 0), 0, abort_flag);
+      if (ok) {
+        tc_fence_after();
+        for (int t = 0; t < n_act; ++t) issue_s(t, 0);
+        umma_commit(BAR(B_KE + 0));
+      }
+      for (int j = 0; j < n_tiles && ok; ++j) {
+        const int s = j & 1;
+        const bool more = j + 1 < n_tiles;
+        for (int t = 0; t < n_act && ok; ++t) {
+          ok = mbar_wait(BAR(B_PF + t), j & 1, abort_flag);
+          if (ok && t == 0) ok = mbar_wait(BAR(B_VF + s), (j >> 1) & 1, abort_flag);
+          if (!ok) break;
+          tc_fence_after();
+          issue_pv(t, j);
+          if (t == n_act - 1) umma_commit(BAR(B_VE + s));   // V stage free once both P V are done
+          if (more) {
+            if (t == 0) ok = mbar_wait(BAR(B_KF + (s ^ 1)), ((j + 1) >> 1) & 1, abort_flag);
+            if (!ok) break;
+            tc_fence_after();
+            issue_s(t, j + 1);
+            if (t == n_act - 1) umma_commit(BAR(B_KE + (s ^ 1)));
+          }
+        }
       }
       if (!ok) atomicExch(p.status, kDevWaitTimeout);
     }
   } else {
     // ------------------------------ softmax warps ------------------------------
+    const int t = (warp - 2) >> 2;        // tile A (warps 2-5) or B (warps 6-9)
     const int qd = warp & 3;              // TMEM lane quarter this warp may access
     const int r = qd * 32 + lane;         // query row within the tile
     const int i = i0 + r;                 // query position
-    const uint32_t lane_addr = tmem + ((uint32_t)(qd * 32) << 16);
+    const int h = hA + t;
+    const uint32_t s_addr = tmem + ((uint32_t)(qd * 32) << 16) + kColS + t * 128;
+    const uint32_t o_addr = tmem + ((uint32_t)(qd * 32) << 16) + kColO + t * 128;
     // O stays in TMEM and P V accumulates into it.  m_ref is the exponent reference of the
     // row: it follows the running max lazily (only when the max grew by more than
     // kRescaleGap, in log2 units), so the read-scale-write of the O row is rare.
     constexpr float kRescaleGap = 8.f;
     float m_ref = -INFINITY, l = 0.f;
-    bool ok = true;
-    for (int j = 0; j < n_tiles; ++j) {
-      const int s = j & 1;
+    bool ok = t < n_act;
+    for (int j = 0; ok && j < n_tiles; ++j) {
       const int j0 = (jt_lo + j) * kBN;
-      if (!__all_sync(0xffffffffu, mbar_wait(BAR(B_SF + s), (j >> 1) & 1, abort_flag))) { ok = false; break; }
+      // S_t(j) complete; being committed after P V_t(j-1) it also tells that O_t is up to date
+      if (!__all_sync(0xffffffffu, mbar_wait(BAR(B_SF + t), j & 1, abort_flag))) { ok = false; break; }
       tc_fence_after();
       uint32_t sv[128];
-      tmem_ld32(lane_addr + s * 128, *reinterpret_cast<uint32_t(*)[32]>(&sv[0]));
-      tmem_ld32(lane_addr + s * 128 + 32, *reinterpret_cast<uint32_t(*)[32]>(&sv[32]));
-      tmem_ld32(lane_addr + s * 128 + 64, *reinterpret_cast<uint32_t(*)[32]>(&sv[64]));
-      tmem_ld32(lane_addr + s * 128 + 96, *reinterpret_cast<uint32_t(*)[32]>(&sv[96]));
+      tmem_ld32(s_addr, *reinterpret_cast<uint32_t(*)[32]>(&sv[0]));
+      tmem_ld32(s_addr + 32, *reinterpret_cast<uint32_t(*)[32]>(&sv[32]));
+      tmem_ld32(s_addr + 64, *reinterpret_cast<uint32_t(*)[32]>(&sv[64]));
+      tmem_ld32(s_addr + 96, *reinterpret_cast<uint32_t(*)[32]>(&sv[96]));
       tmem_wait_ld();
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(BAR(B_SE + s));   // scores are in registers: the S buffer is free
       // band edges: causal (keys after the query) and window (keys older than i - window)
       const bool edge = (j0 + kBN - 1 > i0) || (p.window > 0 && j0 <= i0 + kBM - 1 - p.window);
       if (edge) {
@@ -330,20 +358,16 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
       const bool grow = mt > m_ref + kRescaleGap;    // also true for the first visible key (m_ref = -inf)
       if (__any_sync(0xffffffffu, grow)) {
         const float alpha = grow ? ex2_approx(m_ref - mt) : 1.f;   // m_ref = -inf gives 0
-        if (j > 0) {   // the O row holds earlier tiles: rescale it once P V(j-1) has landed
-          const int sp = (j - 1) & 1;
-          if (!__all_sync(0xffffffffu, mbar_wait(BAR(B_OF + sp), ((j - 1) >> 1) & 1, abort_flag))) { ok = false; break; }
-          tc_fence_after();
+        if (j > 0) {   // the O row holds earlier tiles (all landed, see above): rescale it
 #pragma unroll
           for (int c = 0; c < 4; ++c) {
             uint32_t ov[32];
-            tmem_ld32(lane_addr + 256 + c * 32, ov);
+            tmem_ld32(o_addr + c * 32, ov);
             tmem_wait_ld();
 #pragma unroll
             for (int e = 0; e < 32; ++e) ov[e] = __float_as_uint(__uint_as_float(ov[e]) * alpha);
-            tmem_st32(lane_addr + 256 + c * 32, ov);
+            tmem_st32(o_addr + c * 32, ov);
           }
-          tmem_wait_st();
         }
         l *= alpha;
         if (grow) m_ref = mt;
@@ -360,19 +384,16 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         pk[e >> 1] = pack_bf16(p0, p1);
       }
       l += sum0 + sum1;
-      // the P buffer was last read by P V(j-2)
-      if (j >= 2 && !__all_sync(0xffffffffu, mbar_wait(BAR(B_OF + s), ((j >> 1) - 1) & 1, abort_flag))) { ok = false; break; }
-      // P (bf16 pairs) into tensor memory: columns 384 + 64 s .. of this row
-      tmem_st32(lane_addr + 384 + s * 64, *reinterpret_cast<uint32_t(*)[32]>(&pk[0]));
-      tmem_st32(lane_addr + 384 + s * 64 + 32, *reinterpret_cast<uint32_t(*)[32]>(&pk[32]));
+      // P (bf16 pairs) over the first 64 columns of this row's scores
+      tmem_st32(s_addr, *reinterpret_cast<uint32_t(*)[32]>(&pk[0]));
+      tmem_st32(s_addr + 32, *reinterpret_cast<uint32_t(*)[32]>(&pk[32]));
       tmem_wait_st();
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(BAR(B_PF + s));
+      if (lane == 0) mbar_arrive(BAR(B_PF + t));
     }
     if (ok) {
-      const int sp = (n_tiles - 1) & 1;
-      ok = __all_sync(0xffffffffu, mbar_wait(BAR(B_OF + sp), ((n_tiles - 1) >> 1) & 1, abort_flag));
+      ok = __all_sync(0xffffffffu, mbar_wait(BAR(B_OF + t), (n_tiles - 1) & 1, abort_flag));
       if (ok) {
         tc_fence_after();
         const float inv = 1.f / l;
@@ -380,7 +401,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
           uint32_t ov[32];
-          tmem_ld32(lane_addr + 256 + c * 32, ov);
+          tmem_ld32(o_addr + c * 32, ov);
           tmem_wait_ld();
           if (i < S) {
 #pragma unroll
@@ -396,7 +417,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         tc_fence_before();
       }
     }
-    if (!ok && lane == 0) atomicExch(p.status, kDevWaitTimeout);
+    if (t < n_act && !ok && lane == 0) atomicExch(p.status, kDevWaitTimeout);
   }
   // common exit: everyone is past its last TMEM access
   tc_fence_before();
@@ -464,7 +485,8 @@ cudaError_t launch_prefill_tc(const PrefillParams& pp, int max_len, cudaStream_t
   p.status = pp.status;
   p.out = static_cast<__nv_bfloat16*>(pp.out);
   for (int i = 0; i <= pp.n_seqs; ++i) p.row0[i] = pp.row0[i];
-  dim3 grid((max_len + kBM - 1) / kBM, pp.n_q_heads, pp.n_seqs);
+  const int group = pp.n_q_heads / pp.n_kv_heads;
+  dim3 grid((max_len + kBM - 1) / kBM, pp.n_kv_heads * ((group + 1) / 2), pp.n_seqs);   // two heads per CTA
   prefill_tc_kernel<<<grid, kThreads, kSmemBytes, st>>>(tq, tk, tv, p);
   return cudaGetLastError();
 }
