@@ -5,26 +5,28 @@
 // one CTA owns a 128-query tile of one (sequence, head) and walks the 128-key tiles that
 // intersect its band; tiles wholly outside the band are never loaded.
 //
-// One CTA owns TWO 128-query tiles that share their K/V band: the same query positions of
-// two query heads of one KV head (grouped-query attention), so every K/V tile staged in
-// shared memory feeds two S products and two P V products.
+//   warp 0     TMA producer: Q once, then K and V tiles (3 stages each) as 128B-swizzled
+//              [128 x 64] boxes straight from the caller's tensors
+//   warp 1     one elected thread issues the tcgen05.mma (K16 steps, bf16 -> fp32 in TMEM) of
+//              S = Q K^T (M128 N128, both operands from shared memory) into one of two S
+//              buffers, two tiles ahead of the softmax
+//   warp 10    one elected thread issues O_h += P_h V_h with P_h read from tensor memory
+//              and V MN-major from its row-major tile
+//   warps 2-5  softmax stream "lo": key columns 0-63 of every tile; warps 6-9 stream "hi":
+//              columns 64-127.  The two streams are independent flash-attention passes
+//              over interleaved halves of the keys (own running max, own row sum, own O
+//              accumulator in TMEM), merged exactly at the end like split-KV partials.
+//              Thread r of a stream owns query row r (TMEM lane r): tcgen05.ld of its half
+//              of the S row, band masks on edge tiles only, base-2 online softmax with
+//              one MUFU ex2 per score, P written back as bf16 pairs over its own columns
+//              of the S buffer (tcgen05.st).  O rows are rescaled lazily (only when the
+//              running max grew by more than 2^8).
 //
-//   warp 0     TMA producer: both Q tiles once, then K (2 stages) and V (2 stages) tiles as
-//              128B-swizzled [128 x 64] boxes straight from the caller's tensors
-//   warp 1     one elected thread issues tcgen05.mma (M128 N128 K16, bf16 -> fp32 in TMEM):
-//              S_t = Q_t K^T (both operands from shared memory) and O_t += P_t V with P_t
-//              read from tensor memory and V MN-major from its row-major tile
-//   warps 2-5  softmax of tile A, warps 6-9 softmax of tile B: thread r owns query row r
-//              (TMEM lane r): tcgen05.ld of the S row, band masks on edge tiles only,
-//              base-2 online softmax with one MUFU ex2 per score, P written back as bf16
-//              pairs over the first 64 columns of the S row (tcgen05.st).  O stays in TMEM;
-//              its rows are rescaled lazily (only when the running max grew by more than
-//              2^8), normalised and stored at the end.
-//
-// The two tiles ping-pong: while one group computes exponentials, the tensor core runs the
-// other tile's P V and next S, and the other group loads or stores.  TMEM: S_A, S_B, O_A,
-// O_B = 4 x 128 columns.  All mbarrier waits are bounded; on time-out a status word is
-// raised, every role leaves its loop, and TMEM is released at the common exit.
+// Two warps per scheduler work on independent data, the scores of the next two tiles are
+// always ready, and the P V products are issued in whichever order the streams finish.
+// TMEM: S0, S1, O_lo, O_hi = 4 x 128 columns.  All mbarrier waits are bounded; on
+// time-out a status word is raised, every role leaves its loop, and TMEM is released at
+// the common exit.
 #include <cuda.h>
 #include <cuda_bf16.h>
 
@@ -34,21 +36,24 @@ namespace mixattn {
 
 namespace {
 
-constexpr int kBM = 128;                       // queries per tile (two tiles per CTA)
+constexpr int kBM = 128;                       // queries per CTA
 constexpr int kBN = 128;                       // keys per tile
 constexpr int kHalfBytes = 128 * 128;          // one [128 rows x 64 bf16] swizzled block
 constexpr int kTileBytes = 2 * kHalfBytes;     // a 128 x 128 bf16 operand tile
-constexpr int kThreads = 320;                  // TMA warp, MMA warp, 2 x 4 softmax warps
-constexpr int kSmQ = 0;                        // Q_A, Q_B
-constexpr int kSmK = kSmQ + 2 * kTileBytes;    // 2 stages
-constexpr int kSmV = kSmK + 2 * kTileBytes;    // 2 stages
-constexpr int kSmBar = kSmV + 2 * kTileBytes;  // barriers, TMEM pointer, abort flag
-constexpr int kSmemBytes = kSmBar + 256 + 1024;  // + slack to align the base to 1024 B
+constexpr int kThreads = 352;                  // TMA warp, S-MMA warp, 2 x 4 softmax warps, PV-MMA warp
+constexpr int kStages = 3;                     // K and V stages
+constexpr int kSmQ = 0;
+constexpr int kSmK = kSmQ + kTileBytes;
+constexpr int kSmV = kSmK + kStages * kTileBytes;
+constexpr int kSmBar = kSmV + kStages * kTileBytes;   // barriers, TMEM pointer, abort flag
+constexpr int kSmXchg = kSmBar + 256;                  // [2 streams][128 rows] (max, sum)
+constexpr int kSmemBytes = kSmXchg + 2 * 128 * 8 + 768;  // + slack to align a 256-B aligned base to 1024 B
+static_assert(kSmemBytes <= 227 * 1024, "shared memory budget");
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;
-constexpr uint32_t kColS = 0, kColO = 256;     // TMEM columns: S_t at 128 t, O_t at 256 + 128 t
+constexpr uint32_t kColS = 0, kColO = 256;     // TMEM columns: S buffer b at 128 b, O of stream h at 256 + 128 h
 
-// barrier indices (two each: K/V stages, or tile A / tile B)
-enum { B_Q = 0, B_KF = 1, B_KE = 3, B_VF = 5, B_VE = 7, B_SF = 9, B_PF = 11, B_OF = 13, B_N = 15 };
+// barrier indices
+enum { B_Q = 0, B_KF = 1, B_KE = 4, B_VF = 7, B_VE = 10, B_SF = 13, B_PF = 15, B_OF = 17, B_XC = 19, B_SR = 20, B_N = 22 };   // B_SR: S buffer (and the P in it) consumed by both P V
 
 struct TcParams {
   int32_t n_q_heads, group, window, n_seqs;
@@ -73,6 +78,16 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   asm volatile(
       "{\n\t.reg .pred p;\n\t"
       "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+// Non-blocking probe (try_wait may suspend the thread for a while before it answers).
+__device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
       "selp.u32 %0, 1, 0, p;\n\t}"
       : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
   return ok != 0;
@@ -167,7 +182,7 @@ __host__ __device__ constexpr uint32_t idesc_bf16(int b_mn) {
 __global__ void __launch_bounds__(kThreads, 1)
 prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                   const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ TcParams p) {
-  extern __shared__ unsigned char smem_raw[];
+  extern __shared__ __align__(1024) unsigned char smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   unsigned char* gbase = smem_raw + (base - smem_u32(smem_raw));
   const uint32_t bar0 = base + kSmBar;
@@ -176,17 +191,13 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
 #define BAR(i) (bar0 + 8u * (i))
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int b = blockIdx.z;
-  const int pairs_per_group = (p.group + 1) >> 1;
-  const int g = blockIdx.y / pairs_per_group;                 // KV head
-  const int hA = g * p.group + (blockIdx.y % pairs_per_group) * 2;
-  const bool has_b = (hA + 1) < (g + 1) * p.group;            // odd group size: last pair is a single
-  const int n_act = has_b ? 2 : 1;
+  const int b = blockIdx.z, h = blockIdx.y;
   const int S = p.row0[b + 1] - p.row0[b];
   const int n_qt = (S + kBM - 1) / kBM;
   const int qt = n_qt - 1 - (int)blockIdx.x;   // heaviest (latest) query tiles first
   if (qt < 0) return;                          // uniform per CTA: before any barrier or TMEM use
   const int i0 = qt * kBM;
+  const int g = h / p.group;
   const int row_base = p.row0[b];
   const int key_hi = min(i0 + kBM - 1, S - 1);
   const int key_lo = p.window > 0 ? max(0, i0 - p.window + 1) : 0;
@@ -195,15 +206,19 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
 
   if (threadIdx.x == 0) {
     mbar_init(BAR(B_Q), 1);
-    for (int s = 0; s < 2; ++s) {
+    for (int s = 0; s < kStages; ++s) {
       mbar_init(BAR(B_KF + s), 1);
       mbar_init(BAR(B_KE + s), 1);
       mbar_init(BAR(B_VF + s), 1);
       mbar_init(BAR(B_VE + s), 1);
+    }
+    for (int s = 0; s < 2; ++s) {
       mbar_init(BAR(B_SF + s), 1);
       mbar_init(BAR(B_PF + s), 4);
       mbar_init(BAR(B_OF + s), 1);
+      mbar_init(BAR(B_SR + s), 1);
     }
+    mbar_init(BAR(B_XC), 8);
     abort_flag[0] = 0;
     abort_flag[1] = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -223,23 +238,22 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
       asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_q) : "memory");
       asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_k) : "memory");
       asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_v) : "memory");
-      mbar_expect_tx(BAR(B_Q), n_act * kTileBytes);
-      for (int t = 0; t < n_act; ++t) {
-        tma_load_3d(base + kSmQ + t * kTileBytes, &tm_q, 0, hA + t, row_base + i0, BAR(B_Q));
-        tma_load_3d(base + kSmQ + t * kTileBytes + kHalfBytes, &tm_q, 64, hA + t, row_base + i0, BAR(B_Q));
-      }
+      mbar_expect_tx(BAR(B_Q), kTileBytes);
+      tma_load_3d(base + kSmQ, &tm_q, 0, h, row_base + i0, BAR(B_Q));
+      tma_load_3d(base + kSmQ + kHalfBytes, &tm_q, 64, h, row_base + i0, BAR(B_Q));
       bool ok = true;
       int issued_k = 0, issued_v = 0;
       for (int j = 0; j < n_tiles && ok; ++j) {
-        const int s = j & 1;
+        const int s = j % kStages;
+        const int use = j / kStages;            // how many times this stage was used before
         const int row = row_base + (jt_lo + j) * kBN;
-        if (j >= 2) ok = mbar_wait(BAR(B_KE + s), ((j >> 1) - 1) & 1, abort_flag);
+        if (use > 0) ok = mbar_wait(BAR(B_KE + s), (use - 1) & 1, abort_flag);
         if (!ok) break;
         mbar_expect_tx(BAR(B_KF + s), kTileBytes);
         tma_load_3d(base + kSmK + s * kTileBytes, &tm_k, 0, g, row, BAR(B_KF + s));
         tma_load_3d(base + kSmK + s * kTileBytes + kHalfBytes, &tm_k, 64, g, row, BAR(B_KF + s));
         ++issued_k;
-        if (j >= 2) ok = mbar_wait(BAR(B_VE + s), ((j >> 1) - 1) & 1, abort_flag);
+        if (use > 0) ok = mbar_wait(BAR(B_VE + s), (use - 1) & 1, abort_flag);
         if (!ok) break;
         mbar_expect_tx(BAR(B_VF + s), kTileBytes);
         tma_load_3d(base + kSmV + s * kTileBytes, &tm_v, 0, g, row, BAR(B_VF + s));
@@ -249,106 +263,108 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
       if (!ok) {  // leave only after the copies already issued have landed (bounded)
         atomicExch(p.status, kDevWaitTimeout);
         mbar_wait(BAR(B_Q), 0, abort_flag + 1);
-        for (int back = 1; back <= 2 && issued_k - back >= 0; ++back)
-          mbar_wait(BAR(B_KF + ((issued_k - back) & 1)), ((issued_k - back) >> 1) & 1, abort_flag + 1);
-        for (int back = 1; back <= 2 && issued_v - back >= 0; ++back)
-          mbar_wait(BAR(B_VF + ((issued_v - back) & 1)), ((issued_v - back) >> 1) & 1, abort_flag + 1);
+        for (int back = 1; back <= kStages && issued_k - back >= 0; ++back)
+          mbar_wait(BAR(B_KF + (issued_k - back) % kStages), ((issued_k - back) / kStages) & 1, abort_flag + 1);
+        for (int back = 1; back <= kStages && issued_v - back >= 0; ++back)
+          mbar_wait(BAR(B_VF + (issued_v - back) % kStages), ((issued_v - back) / kStages) & 1, abort_flag + 1);
       }
     }
   } else if (warp == 1) {
-    // ------------------------------ MMA issuer ------------------------------
+    // ------------------------------ MMA issuer, scores ------------------------------
+    // Two threads issue MMAs (this one S = Q K^T, warp 10 the P V products): issuing is a
+    // serial, latency-bound instruction stream, and one thread alone was the bottleneck.
     if (lane == 0) {
       constexpr uint32_t kIdescS = idesc_bf16(0);
-      constexpr uint32_t kIdescPV = idesc_bf16(1);
       bool ok = mbar_wait(BAR(B_Q), 0, abort_flag);
-      // S_t(j) = Q_t K_j^T into the S columns of tile t (which also hold P_t(j-1): the
-      // tensor pipe runs this thread's MMAs in order, so P V_t(j-1) has read it by then)
-      auto issue_s = [&](int t, int j) {
-        const int s = j & 1;
+      uint64_t qdesc[8];
 #pragma unroll
-        for (int ks = 0; ks < 8; ++ks) {   // head_dim 128 = 8 steps of 16
-          const uint32_t off = (ks >> 2) * kHalfBytes + (ks & 3) * 32;
-          umma_bf16(tmem + kColS + t * 128, smem_desc(base + kSmQ + t * kTileBytes + off, 16, 1024),
-                    smem_desc(base + kSmK + s * kTileBytes + off, 16, 1024), kIdescS, ks > 0);
-        }
-        umma_commit(BAR(B_SF + t));
-      };
-      // O_t += P_t(j) V_j: A = P from tensor memory (two bf16 per column), B = V MN-major
-      auto issue_pv = [&](int t, int j) {
-        const int s = j & 1;
-#pragma unroll
-        for (int ks = 0; ks < 8; ++ks) {   // 128 keys = 8 steps of 16
-          const uint64_t bd = smem_desc(base + kSmV + s * kTileBytes + ks * 2048, kHalfBytes, 1024);
-          umma_bf16_ts(tmem + kColO + t * 128, tmem + kColS + t * 128 + ks * 8, bd, kIdescPV,
-                       (j > 0 || ks > 0) ? 1u : 0u);
-        }
-        umma_commit(BAR(B_OF + t));
-      };
-      if (ok) ok = mbar_wait(BAR(B_KF + 0), 0, abort_flag);
-      if (ok) {
-        tc_fence_after();
-        for (int t = 0; t < n_act; ++t) issue_s(t, 0);
-        umma_commit(BAR(B_KE + 0));
-      }
+      for (int ks = 0; ks < 8; ++ks)   // head_dim 128 = 8 steps of 16 channels
+        qdesc[ks] = smem_desc(base + kSmQ + (ks >> 2) * kHalfBytes + (ks & 3) * 32, 16, 1024);
       for (int j = 0; j < n_tiles && ok; ++j) {
-        const int s = j & 1;
-        const bool more = j + 1 < n_tiles;
-        for (int t = 0; t < n_act && ok; ++t) {
-          ok = mbar_wait(BAR(B_PF + t), j & 1, abort_flag);
-          if (ok && t == 0) ok = mbar_wait(BAR(B_VF + s), (j >> 1) & 1, abort_flag);
-          if (!ok) break;
-          tc_fence_after();
-          issue_pv(t, j);
-          if (t == n_act - 1) umma_commit(BAR(B_VE + s));   // V stage free once both P V are done
-          if (more) {
-            if (t == 0) ok = mbar_wait(BAR(B_KF + (s ^ 1)), ((j + 1) >> 1) & 1, abort_flag);
-            if (!ok) break;
-            tc_fence_after();
-            issue_s(t, j + 1);
-            if (t == n_act - 1) umma_commit(BAR(B_KE + (s ^ 1)));
+        // S(j) = Q K_j^T into S buffer j & 1, which held S(j-2) / P(j-2): wait until both
+        // P V(j-2) have consumed it (they are issued by another thread)
+        const int ks_ = j % kStages;
+        if (j >= 2) ok = mbar_wait(BAR(B_SR + (j & 1)), ((j >> 1) - 1) & 1, abort_flag);
+        if (ok) ok = mbar_wait(BAR(B_KF + ks_), (j / kStages) & 1, abort_flag);
+        if (!ok) break;
+        tc_fence_after();
+        const uint64_t kdesc = smem_desc(base + kSmK + ks_ * kTileBytes, 16, 1024);
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks)
+          umma_bf16(tmem + kColS + (j & 1) * 128, qdesc[ks], kdesc + (uint64_t)((ks >> 2) * (kHalfBytes >> 4) + (ks & 3) * 2),
+                    kIdescS, ks > 0);
+        umma_commit(BAR(B_SF + (j & 1)));   // scores ready
+        umma_commit(BAR(B_KE + ks_));       // K stage free
+      }
+      if (!ok) atomicExch(p.status, kDevWaitTimeout);
+    }
+  } else if (warp == 10) {
+    // ------------------------------ MMA issuer, P V ------------------------------
+    if (lane == 0) {
+      constexpr uint32_t kIdescPV = idesc_bf16(1);
+      bool ok = true;
+      for (int j = 0; j < n_tiles && ok; ++j) {
+        const int vs = j % kStages;
+        ok = mbar_wait(BAR(B_VF + vs), (j / kStages) & 1, abort_flag);
+        const uint64_t vdesc = smem_desc(base + kSmV + vs * kTileBytes, kHalfBytes, 1024);
+        // serve the two streams in the order their P arrives (bounded polling)
+        bool done[2] = {false, false};
+        const unsigned long long t0 = global_ns();
+        for (uint32_t it = 1; ok && !(done[0] && done[1]); ++it) {
+#pragma unroll
+          for (int hs = 0; hs < 2; ++hs) {
+            if (!done[hs] && mbar_test_wait(BAR(B_PF + hs), j & 1)) {
+              tc_fence_after();
+              // O_h += P_h(j) V_j[64 h .. 64 h + 63]: A = P from tensor memory (two bf16 per
+              // column), B = V MN-major (channels contiguous, keys strided by 128 B)
+#pragma unroll
+              for (int ks = 0; ks < 4; ++ks)   // 64 keys = 4 steps of 16
+                umma_bf16_ts(tmem + kColO + hs * 128, tmem + kColS + (j & 1) * 128 + hs * 64 + ks * 8,
+                             vdesc + (uint64_t)((hs * 4 + ks) * (2048 >> 4)), kIdescPV, (j > 0 || ks > 0) ? 1u : 0u);
+              umma_commit(BAR(B_OF + hs));
+              done[hs] = true;
+            }
           }
+          if ((it & 1023u) == 0 && (*abort_flag || global_ns() - t0 > kWaitLimitNs)) { *abort_flag = 1; ok = false; }
         }
+        if (!ok) break;
+        umma_commit(BAR(B_VE + vs));          // V stage free once both P V are done
+        umma_commit(BAR(B_SR + (j & 1)));     // and so is the S buffer
       }
       if (!ok) atomicExch(p.status, kDevWaitTimeout);
     }
   } else {
     // ------------------------------ softmax warps ------------------------------
-    const int t = (warp - 2) >> 2;        // tile A (warps 2-5) or B (warps 6-9)
+    const int hs = (warp - 2) >> 2;       // stream: key columns [64 hs, 64 hs + 64) of every tile
     const int qd = warp & 3;              // TMEM lane quarter this warp may access
     const int r = qd * 32 + lane;         // query row within the tile
     const int i = i0 + r;                 // query position
-    const int h = hA + t;
-    const uint32_t s_addr = tmem + ((uint32_t)(qd * 32) << 16) + kColS + t * 128;
-    const uint32_t o_addr = tmem + ((uint32_t)(qd * 32) << 16) + kColO + t * 128;
-    // O stays in TMEM and P V accumulates into it.  m_ref is the exponent reference of the
-    // row: it follows the running max lazily (only when the max grew by more than
-    // kRescaleGap, in log2 units), so the read-scale-write of the O row is rare.
-    constexpr float kRescaleGap = 8.f;
+    const uint32_t lane_base = tmem + ((uint32_t)(qd * 32) << 16);
+    const uint32_t o_addr = lane_base + kColO + hs * 128;
+    constexpr float kRescaleGap = 8.f;    // the exponent reference may lag the running max by 2^8
     float m_ref = -INFINITY, l = 0.f;
-    bool ok = t < n_act;
-    for (int j = 0; ok && j < n_tiles; ++j) {
-      const int j0 = (jt_lo + j) * kBN;
-      // S_t(j) complete; being committed after P V_t(j-1) it also tells that O_t is up to date
-      if (!__all_sync(0xffffffffu, mbar_wait(BAR(B_SF + t), j & 1, abort_flag))) { ok = false; break; }
+    bool ok = true;
+    for (int j = 0; j < n_tiles; ++j) {
+      const int j0 = (jt_lo + j) * kBN + hs * 64;   // first key of this stream's columns
+      const uint32_t s_addr = lane_base + kColS + (j & 1) * 128 + hs * 64;
+      if (!__all_sync(0xffffffffu, mbar_wait(BAR(B_SF + (j & 1)), (j >> 1) & 1, abort_flag))) { ok = false; break; }
       tc_fence_after();
-      uint32_t sv[128];
+      uint32_t sv[64];
       tmem_ld32(s_addr, *reinterpret_cast<uint32_t(*)[32]>(&sv[0]));
       tmem_ld32(s_addr + 32, *reinterpret_cast<uint32_t(*)[32]>(&sv[32]));
-      tmem_ld32(s_addr + 64, *reinterpret_cast<uint32_t(*)[32]>(&sv[64]));
-      tmem_ld32(s_addr + 96, *reinterpret_cast<uint32_t(*)[32]>(&sv[96]));
       tmem_wait_ld();
       // band edges: causal (keys after the query) and window (keys older than i - window)
-      const bool edge = (j0 + kBN - 1 > i0) || (p.window > 0 && j0 <= i0 + kBM - 1 - p.window);
+      const bool edge = (j0 + 63 > i0) || (p.window > 0 && j0 <= i0 + kBM - 1 - p.window);
       if (edge) {
         const int k_max = i - j0;                                      // columns <= k_max are causal-visible
         const int k_min = p.window > 0 ? i - p.window + 1 - j0 : 0;    // columns >= k_min are inside the window
 #pragma unroll
-        for (int e = 0; e < 128; ++e)
+        for (int e = 0; e < 64; ++e)
           if (e > k_max || e < k_min) sv[e] = 0xff800000u;             // -inf
       }
       float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
 #pragma unroll
-      for (int e = 0; e < 128; e += 4) {
+      for (int e = 0; e < 64; e += 4) {
         mx0 = fmaxf(mx0, __uint_as_float(sv[e]));
         mx1 = fmaxf(mx1, __uint_as_float(sv[e + 1]));
         mx2 = fmaxf(mx2, __uint_as_float(sv[e + 2]));
@@ -358,7 +374,9 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
       const bool grow = mt > m_ref + kRescaleGap;    // also true for the first visible key (m_ref = -inf)
       if (__any_sync(0xffffffffu, grow)) {
         const float alpha = grow ? ex2_approx(m_ref - mt) : 1.f;   // m_ref = -inf gives 0
-        if (j > 0) {   // the O row holds earlier tiles (all landed, see above): rescale it
+        if (j > 0) {   // the O row holds earlier tiles: rescale it once this stream's P V(j-1) has landed
+          if (!__all_sync(0xffffffffu, mbar_wait(BAR(B_OF + hs), (j - 1) & 1, abort_flag))) { ok = false; break; }
+          tc_fence_after();
 #pragma unroll
           for (int c = 0; c < 4; ++c) {
             uint32_t ov[32];
@@ -372,11 +390,11 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         l *= alpha;
         if (grow) m_ref = mt;
       }
-      const float neg_m = m_ref == -INFINITY ? 0.f : -m_ref;   // row with no visible key yet: weights 0, no NaN
+      const float neg_m = m_ref == -INFINITY ? 0.f : -m_ref;   // no visible key yet: weights 0, no NaN
       float sum0 = 0.f, sum1 = 0.f;
-      uint32_t pk[64];
+      uint32_t pk[32];
 #pragma unroll
-      for (int e = 0; e < 128; e += 2) {
+      for (int e = 0; e < 64; e += 2) {
         const float p0 = ex2_approx(fmaf(__uint_as_float(sv[e]), p.scale_log2e, neg_m));
         const float p1 = ex2_approx(fmaf(__uint_as_float(sv[e + 1]), p.scale_log2e, neg_m));
         sum0 += p0;
@@ -384,40 +402,60 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         pk[e >> 1] = pack_bf16(p0, p1);
       }
       l += sum0 + sum1;
-      // P (bf16 pairs) over the first 64 columns of this row's scores
-      tmem_st32(s_addr, *reinterpret_cast<uint32_t(*)[32]>(&pk[0]));
-      tmem_st32(s_addr + 32, *reinterpret_cast<uint32_t(*)[32]>(&pk[32]));
+      // P (bf16 pairs) over the first 32 of this stream's 64 score columns
+      tmem_st32(s_addr, pk);
       tmem_wait_st();
       tc_fence_before();
+      // back-pressure: P(j) may only be announced once P V(j-1) of this stream has run, so the
+      // announcement barrier is never more than one phase ahead of the MMA thread
+      if (j > 0 && !__all_sync(0xffffffffu, mbar_wait(BAR(B_OF + hs), (j - 1) & 1, abort_flag))) { ok = false; break; }
       __syncwarp();
-      if (lane == 0) mbar_arrive(BAR(B_PF + t));
+      if (lane == 0) mbar_arrive(BAR(B_PF + hs));
+    }
+    if (ok) ok = __all_sync(0xffffffffu, mbar_wait(BAR(B_OF + hs), (n_tiles - 1) & 1, abort_flag));
+    if (ok) {
+      // merge the two streams like split-KV partials: exchange (reference, sum) per row
+      tc_fence_after();
+      float2* xchg = reinterpret_cast<float2*>(gbase + kSmXchg);
+      xchg[hs * 128 + r] = make_float2(m_ref, l);
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(BAR(B_XC));
+      ok = __all_sync(0xffffffffu, mbar_wait(BAR(B_XC), 0, abort_flag));
     }
     if (ok) {
-      ok = __all_sync(0xffffffffu, mbar_wait(BAR(B_OF + t), (n_tiles - 1) & 1, abort_flag));
-      if (ok) {
-        tc_fence_after();
-        const float inv = 1.f / l;
-        __nv_bfloat16* orow = p.out + ((int64_t)(row_base + i) * p.n_q_heads + h) * 128;
+      tc_fence_after();
+      const float2* xchg = reinterpret_cast<const float2*>(gbase + kSmXchg);
+      const float2 other = xchg[(hs ^ 1) * 128 + r];
+      const float m_all = fmaxf(m_ref, other.x);          // finite for every valid row (key i is visible)
+      const float w_me = ex2_approx(m_ref - m_all), w_ot = ex2_approx(other.x - m_all);   // 2^-inf = 0
+      const float inv = 1.f / (l * w_me + other.y * w_ot);
+      const float w_lo = (hs == 0 ? w_me : w_ot) * inv, w_hi = (hs == 0 ? w_ot : w_me) * inv;
+      // this thread writes channels [64 hs, 64 hs + 64) of its row from both accumulators
+      __nv_bfloat16* orow = p.out + ((int64_t)(row_base + i) * p.n_q_heads + h) * 128 + hs * 64;
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {
-          uint32_t ov[32];
-          tmem_ld32(o_addr + c * 32, ov);
-          tmem_wait_ld();
-          if (i < S) {
+      for (int c = 0; c < 2; ++c) {
+        uint32_t olo[32], ohi[32];
+        tmem_ld32(lane_base + kColO + hs * 64 + c * 32, olo);
+        tmem_ld32(lane_base + kColO + 128 + hs * 64 + c * 32, ohi);
+        tmem_wait_ld();
+        if (i < S) {
 #pragma unroll
-            for (int q4 = 0; q4 < 4; ++q4) {
-              uint32_t w[4];
+          for (int q4 = 0; q4 < 4; ++q4) {
+            uint32_t w[4];
 #pragma unroll
-              for (int e = 0; e < 4; ++e)
-                w[e] = pack_bf16(__uint_as_float(ov[q4 * 8 + e * 2]) * inv, __uint_as_float(ov[q4 * 8 + e * 2 + 1]) * inv);
-              *reinterpret_cast<uint4*>(orow + c * 32 + q4 * 8) = make_uint4(w[0], w[1], w[2], w[3]);
+            for (int e = 0; e < 4; ++e) {
+              const int d = q4 * 8 + e * 2;
+              w[e] = pack_bf16(__uint_as_float(olo[d]) * w_lo + __uint_as_float(ohi[d]) * w_hi,
+                               __uint_as_float(olo[d + 1]) * w_lo + __uint_as_float(ohi[d + 1]) * w_hi);
             }
+            *reinterpret_cast<uint4*>(orow + c * 32 + q4 * 8) = make_uint4(w[0], w[1], w[2], w[3]);
           }
         }
-        tc_fence_before();
       }
+      tc_fence_before();
     }
-    if (t < n_act && !ok && lane == 0) atomicExch(p.status, kDevWaitTimeout);
+    if (!ok && lane == 0) atomicExch(p.status, kDevWaitTimeout);
   }
   // common exit: everyone is past its last TMEM access
   tc_fence_before();
@@ -485,8 +523,7 @@ cudaError_t launch_prefill_tc(const PrefillParams& pp, int max_len, cudaStream_t
   p.status = pp.status;
   p.out = static_cast<__nv_bfloat16*>(pp.out);
   for (int i = 0; i <= pp.n_seqs; ++i) p.row0[i] = pp.row0[i];
-  const int group = pp.n_q_heads / pp.n_kv_heads;
-  dim3 grid((max_len + kBM - 1) / kBM, pp.n_kv_heads * ((group + 1) / 2), pp.n_seqs);   // two heads per CTA
+  dim3 grid((max_len + kBM - 1) / kBM, pp.n_q_heads, pp.n_seqs);
   prefill_tc_kernel<<<grid, kThreads, kSmemBytes, st>>>(tq, tk, tv, p);
   return cudaGetLastError();
 }
