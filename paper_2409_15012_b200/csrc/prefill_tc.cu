@@ -49,7 +49,7 @@ constexpr int kSmBar = kSmV + kStages * kTileBytes;   // barriers, TMEM pointer,
 constexpr int kSmXchg = kSmBar + 256;                  // [2 streams][128 rows] (max, sum)
 constexpr int kSmemBytes = kSmXchg + 2 * 128 * 8 + 768;  // + slack to align a 256-B aligned base to 1024 B
 static_assert(kSmemBytes <= 227 * 1024, "shared memory budget");
-constexpr unsigned long long kWaitLimitNs = 2000000000ull;
+constexpr long long kWaitLimitCycles = 4000000000ll;   // about two seconds of SM clock
 constexpr uint32_t kColS = 0, kColO = 256;     // TMEM columns: S buffer b at 128 b, O of stream h at 256 + 128 h
 
 // barrier indices
@@ -92,19 +92,14 @@ __device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
       : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
   return ok != 0;
 }
-__device__ __forceinline__ unsigned long long global_ns() {
-  unsigned long long t;
-  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-  return t;
-}
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
   if (mbar_try_wait(bar, parity)) return true;
-  const unsigned long long t0 = global_ns();
+  const long long t0 = clock64();   // (the SM clock is cheap to read; the global timer is not)
   for (uint32_t it = 1;; ++it) {
     if (mbar_try_wait(bar, parity)) return true;
     if ((it & 1023u) == 0) {
       if (*abort_flag) return false;
-      if (global_ns() - t0 > kWaitLimitNs) { *abort_flag = 1; return false; }
+      if (clock64() - t0 > kWaitLimitCycles) { *abort_flag = 1; return false; }
     }
   }
 }
@@ -309,7 +304,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         const uint64_t vdesc = smem_desc(base + kSmV + vs * kTileBytes, kHalfBytes, 1024);
         // serve the two streams in the order their P arrives (bounded polling)
         bool done[2] = {false, false};
-        const unsigned long long t0 = global_ns();
+        const long long t0 = clock64();
         for (uint32_t it = 1; ok && !(done[0] && done[1]); ++it) {
 #pragma unroll
           for (int hs = 0; hs < 2; ++hs) {
@@ -325,7 +320,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
               done[hs] = true;
             }
           }
-          if ((it & 1023u) == 0 && (*abort_flag || global_ns() - t0 > kWaitLimitNs)) { *abort_flag = 1; ok = false; }
+          if ((it & 1023u) == 0 && (*abort_flag || clock64() - t0 > kWaitLimitCycles)) { *abort_flag = 1; ok = false; }
         }
         if (!ok) break;
         umma_commit(BAR(B_VE + vs));          // V stage free once both P V are done
