@@ -477,7 +477,7 @@ int mixattn_prefill(mixattn_ctx* c, int32_t layer, int32_t n_seqs, const int32_t
     // head_dim 64) on the exact CUDA-core kernel
     const bool tc = prefill_tc_supported(c->cfg.dtype, D, p.q, p.k, p.v) && (((size_t)p.out) & 15) == 0;
     cudaError_t e = launch_recorded(c, cls, st, [&] {
-      return tc ? launch_prefill_tc(p, mlen, st) : launch_prefill_simple(p, c->cfg.dtype, mlen, st);
+      return tc ? launch_prefill_tc(p, mlen, c->sm_count, st) : launch_prefill_simple(p, c->cfg.dtype, mlen, st);
     });
     if (e != cudaSuccess) return MIXATTN_ERR_CUDA;
   }

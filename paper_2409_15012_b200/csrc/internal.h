@@ -129,6 +129,6 @@ cudaError_t launch_decode_combine(const DecodeParams& p, int dtype, cudaStream_t
 cudaError_t launch_prefill_simple(const PrefillParams& p, int dtype, int max_len, cudaStream_t st);
 bool prefill_tc_supported(int dtype, int head_dim, const void* q, const void* k, const void* v);
 cudaError_t prepare_prefill_tc();
-cudaError_t launch_prefill_tc(const PrefillParams& p, int max_len, cudaStream_t st);
+cudaError_t launch_prefill_tc(const PrefillParams& p, int max_len, int sm_count, cudaStream_t st);
 
 }  // namespace mixattn

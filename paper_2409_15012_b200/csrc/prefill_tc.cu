@@ -36,16 +36,16 @@ namespace mixattn {
 
 namespace {
 
-constexpr int kBM = 128;                       // queries per CTA
+constexpr int kBM = 128;                       // queries per work item
 constexpr int kBN = 128;                       // keys per tile
 constexpr int kHalfBytes = 128 * 128;          // one [128 rows x 64 bf16] swizzled block
 constexpr int kTileBytes = 2 * kHalfBytes;     // a 128 x 128 bf16 operand tile
 constexpr int kThreads = 352;                  // TMA warp, S-MMA warp, 2 x 4 softmax warps, PV-MMA warp
-constexpr int kStages = 3;                     // K and V stages
-constexpr int kSmQ = 0;
-constexpr int kSmK = kSmQ + kTileBytes;
-constexpr int kSmV = kSmK + kStages * kTileBytes;
-constexpr int kSmBar = kSmV + kStages * kTileBytes;   // barriers, TMEM pointer, abort flag
+constexpr int kKStages = 3, kVStages = 2;
+constexpr int kSmQ = 0;                        // two Q buffers (this item / next item)
+constexpr int kSmK = kSmQ + 2 * kTileBytes;
+constexpr int kSmV = kSmK + kKStages * kTileBytes;
+constexpr int kSmBar = kSmV + kVStages * kTileBytes;   // barriers, TMEM pointer, abort flag
 constexpr int kSmXchg = kSmBar + 256;                  // [2 streams][128 rows] (max, sum)
 constexpr int kSmemBytes = kSmXchg + 2 * 128 * 8 + 768;  // + slack to align a 256-B aligned base to 1024 B
 static_assert(kSmemBytes <= 227 * 1024, "shared memory budget");
@@ -53,10 +53,19 @@ constexpr long long kWaitLimitCycles = 4000000000ll;   // about two seconds of S
 constexpr uint32_t kColS = 0, kColO = 256;     // TMEM columns: S buffer b at 128 b, O of stream h at 256 + 128 h
 
 // barrier indices
-enum { B_Q = 0, B_KF = 1, B_KE = 4, B_VF = 7, B_VE = 10, B_SF = 13, B_PF = 15, B_OF = 17, B_XC = 19, B_SR = 20, B_N = 22 };   // B_SR: S buffer (and the P in it) consumed by both P V
+enum {
+  B_QF = 0, B_QE = 2,            // Q buffer full / free (per buffer)
+  B_KF = 4, B_KE = 7,            // K stage full / free
+  B_VF = 10, B_VE = 12,          // V stage full / free
+  B_SF = 14, B_SR = 16,          // S buffer: scores ready / buffer (with the P in it) consumed by both P V
+  B_PF = 18, B_OF = 20,          // per stream: P announced / P V done
+  B_XC = 22, B_OR = 23,          // per item: streams exchanged (max, sum) / streams have read the O accumulators
+  B_N = 24
+};
 
 struct TcParams {
   int32_t n_q_heads, group, window, n_seqs;
+  int32_t max_qt;        // query tiles of the longest sequence
   float scale_log2e;
   int32_t* status;
   __nv_bfloat16* out;
@@ -174,6 +183,33 @@ __host__ __device__ constexpr uint32_t idesc_bf16(int b_mn) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)b_mn << 16) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
 }
 
+// One work item: query tile qt of head h of sequence b.  Ids enumerate (reverse tile
+// index, sequence, head), so the heaviest tiles of all heads come first and the heads of
+// a KV group, which read the same K/V tiles, run at the same time on neighbouring SMs.
+struct WorkItem {
+  int h, g, row_base, S, i0, jt_lo, n_tiles;
+  bool valid;
+};
+__device__ __forceinline__ WorkItem get_item(const TcParams& p, int id) {
+  WorkItem w;
+  const int per_tile = p.n_seqs * p.n_q_heads;
+  const int qt_rev = id / per_tile;
+  const int rem = id - qt_rev * per_tile;
+  const int b = rem / p.n_q_heads;
+  w.h = rem - b * p.n_q_heads;
+  w.g = w.h / p.group;
+  w.row_base = p.row0[b];
+  w.S = p.row0[b + 1] - p.row0[b];
+  const int qt = (w.S + kBM - 1) / kBM - 1 - qt_rev;
+  w.valid = qt >= 0;
+  w.i0 = qt * kBM;
+  const int key_hi = min(w.i0 + kBM - 1, w.S - 1);
+  const int key_lo = p.window > 0 ? max(0, w.i0 - p.window + 1) : 0;
+  w.jt_lo = key_lo / kBN;
+  w.n_tiles = key_hi / kBN - w.jt_lo + 1;
+  return w;
+}
+
 __global__ void __launch_bounds__(kThreads, 1)
 prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                   const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ TcParams p) {
@@ -186,34 +222,25 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
 #define BAR(i) (bar0 + 8u * (i))
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int b = blockIdx.z, h = blockIdx.y;
-  const int S = p.row0[b + 1] - p.row0[b];
-  const int n_qt = (S + kBM - 1) / kBM;
-  const int qt = n_qt - 1 - (int)blockIdx.x;   // heaviest (latest) query tiles first
-  if (qt < 0) return;                          // uniform per CTA: before any barrier or TMEM use
-  const int i0 = qt * kBM;
-  const int g = h / p.group;
-  const int row_base = p.row0[b];
-  const int key_hi = min(i0 + kBM - 1, S - 1);
-  const int key_lo = p.window > 0 ? max(0, i0 - p.window + 1) : 0;
-  const int jt_lo = key_lo / kBN;
-  const int n_tiles = key_hi / kBN - jt_lo + 1;
+  const int n_ids = p.max_qt * p.n_seqs * p.n_q_heads;
 
   if (threadIdx.x == 0) {
-    mbar_init(BAR(B_Q), 1);
-    for (int s = 0; s < kStages; ++s) {
-      mbar_init(BAR(B_KF + s), 1);
-      mbar_init(BAR(B_KE + s), 1);
+    for (int s = 0; s < 2; ++s) {
+      mbar_init(BAR(B_QF + s), 1);
+      mbar_init(BAR(B_QE + s), 1);
       mbar_init(BAR(B_VF + s), 1);
       mbar_init(BAR(B_VE + s), 1);
-    }
-    for (int s = 0; s < 2; ++s) {
       mbar_init(BAR(B_SF + s), 1);
+      mbar_init(BAR(B_SR + s), 1);
       mbar_init(BAR(B_PF + s), 4);
       mbar_init(BAR(B_OF + s), 1);
-      mbar_init(BAR(B_SR + s), 1);
+    }
+    for (int s = 0; s < kKStages; ++s) {
+      mbar_init(BAR(B_KF + s), 1);
+      mbar_init(BAR(B_KE + s), 1);
     }
     mbar_init(BAR(B_XC), 8);
+    mbar_init(BAR(B_OR), 8);
     abort_flag[0] = 0;
     abort_flag[1] = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -227,41 +254,56 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
 
+  // Every role walks the same item list and keeps the same counters: G = key tiles
+  // processed so far by this CTA (all items), it = items processed so far.  Per-tile
+  // barriers are indexed by G, per-item barriers by it, so phases carry over.
   if (warp == 0) {
     // ------------------------------ TMA producer ------------------------------
     if (lane == 0) {
       asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_q) : "memory");
       asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_k) : "memory");
       asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_v) : "memory");
-      mbar_expect_tx(BAR(B_Q), kTileBytes);
-      tma_load_3d(base + kSmQ, &tm_q, 0, h, row_base + i0, BAR(B_Q));
-      tma_load_3d(base + kSmQ + kHalfBytes, &tm_q, 64, h, row_base + i0, BAR(B_Q));
       bool ok = true;
-      int issued_k = 0, issued_v = 0;
-      for (int j = 0; j < n_tiles && ok; ++j) {
-        const int s = j % kStages;
-        const int use = j / kStages;            // how many times this stage was used before
-        const int row = row_base + (jt_lo + j) * kBN;
-        if (use > 0) ok = mbar_wait(BAR(B_KE + s), (use - 1) & 1, abort_flag);
+      int G = 0, it = 0, q_issued = 0, k_issued = 0, v_issued = 0;
+      for (int id = blockIdx.x; id < n_ids && ok; id += gridDim.x) {
+        const WorkItem w = get_item(p, id);
+        if (!w.valid) continue;
+        const int qb = it & 1;
+        if (it >= 2) ok = mbar_wait(BAR(B_QE + qb), ((it >> 1) - 1) & 1, abort_flag);
         if (!ok) break;
-        mbar_expect_tx(BAR(B_KF + s), kTileBytes);
-        tma_load_3d(base + kSmK + s * kTileBytes, &tm_k, 0, g, row, BAR(B_KF + s));
-        tma_load_3d(base + kSmK + s * kTileBytes + kHalfBytes, &tm_k, 64, g, row, BAR(B_KF + s));
-        ++issued_k;
-        if (use > 0) ok = mbar_wait(BAR(B_VE + s), (use - 1) & 1, abort_flag);
-        if (!ok) break;
-        mbar_expect_tx(BAR(B_VF + s), kTileBytes);
-        tma_load_3d(base + kSmV + s * kTileBytes, &tm_v, 0, g, row, BAR(B_VF + s));
-        tma_load_3d(base + kSmV + s * kTileBytes + kHalfBytes, &tm_v, 64, g, row, BAR(B_VF + s));
-        ++issued_v;
+        mbar_expect_tx(BAR(B_QF + qb), kTileBytes);
+        tma_load_3d(base + kSmQ + qb * kTileBytes, &tm_q, 0, w.h, w.row_base + w.i0, BAR(B_QF + qb));
+        tma_load_3d(base + kSmQ + qb * kTileBytes + kHalfBytes, &tm_q, 64, w.h, w.row_base + w.i0, BAR(B_QF + qb));
+        ++q_issued;
+        for (int j = 0; j < w.n_tiles && ok; ++j) {
+          const int Gj = G + j;
+          const int row = w.row_base + (w.jt_lo + j) * kBN;
+          const int ks = Gj % kKStages, ku = Gj / kKStages;
+          if (ku > 0) ok = mbar_wait(BAR(B_KE + ks), (ku - 1) & 1, abort_flag);
+          if (!ok) break;
+          mbar_expect_tx(BAR(B_KF + ks), kTileBytes);
+          tma_load_3d(base + kSmK + ks * kTileBytes, &tm_k, 0, w.g, row, BAR(B_KF + ks));
+          tma_load_3d(base + kSmK + ks * kTileBytes + kHalfBytes, &tm_k, 64, w.g, row, BAR(B_KF + ks));
+          ++k_issued;
+          const int vs = Gj % kVStages, vu = Gj / kVStages;
+          if (vu > 0) ok = mbar_wait(BAR(B_VE + vs), (vu - 1) & 1, abort_flag);
+          if (!ok) break;
+          mbar_expect_tx(BAR(B_VF + vs), kTileBytes);
+          tma_load_3d(base + kSmV + vs * kTileBytes, &tm_v, 0, w.g, row, BAR(B_VF + vs));
+          tma_load_3d(base + kSmV + vs * kTileBytes + kHalfBytes, &tm_v, 64, w.g, row, BAR(B_VF + vs));
+          ++v_issued;
+        }
+        G += w.n_tiles;
+        ++it;
       }
       if (!ok) {  // leave only after the copies already issued have landed (bounded)
         atomicExch(p.status, kDevWaitTimeout);
-        mbar_wait(BAR(B_Q), 0, abort_flag + 1);
-        for (int back = 1; back <= kStages && issued_k - back >= 0; ++back)
-          mbar_wait(BAR(B_KF + (issued_k - back) % kStages), ((issued_k - back) / kStages) & 1, abort_flag + 1);
-        for (int back = 1; back <= kStages && issued_v - back >= 0; ++back)
-          mbar_wait(BAR(B_VF + (issued_v - back) % kStages), ((issued_v - back) / kStages) & 1, abort_flag + 1);
+        for (int back = 1; back <= 2 && q_issued - back >= 0; ++back)
+          mbar_wait(BAR(B_QF + ((q_issued - back) & 1)), ((q_issued - back) >> 1) & 1, abort_flag + 1);
+        for (int back = 1; back <= kKStages && k_issued - back >= 0; ++back)
+          mbar_wait(BAR(B_KF + (k_issued - back) % kKStages), ((k_issued - back) / kKStages) & 1, abort_flag + 1);
+        for (int back = 1; back <= kVStages && v_issued - back >= 0; ++back)
+          mbar_wait(BAR(B_VF + (v_issued - back) % kVStages), ((v_issued - back) / kVStages) & 1, abort_flag + 1);
       }
     }
   } else if (warp == 1) {
@@ -270,26 +312,36 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     // serial, latency-bound instruction stream, and one thread alone was the bottleneck.
     if (lane == 0) {
       constexpr uint32_t kIdescS = idesc_bf16(0);
-      bool ok = mbar_wait(BAR(B_Q), 0, abort_flag);
-      uint64_t qdesc[8];
+      bool ok = true;
+      int G = 0, it = 0;
+      for (int id = blockIdx.x; id < n_ids && ok; id += gridDim.x) {
+        const WorkItem w = get_item(p, id);
+        if (!w.valid) continue;
+        const int qb = it & 1;
+        ok = mbar_wait(BAR(B_QF + qb), (it >> 1) & 1, abort_flag);
+        uint64_t qdesc[8];
 #pragma unroll
-      for (int ks = 0; ks < 8; ++ks)   // head_dim 128 = 8 steps of 16 channels
-        qdesc[ks] = smem_desc(base + kSmQ + (ks >> 2) * kHalfBytes + (ks & 3) * 32, 16, 1024);
-      for (int j = 0; j < n_tiles && ok; ++j) {
-        // S(j) = Q K_j^T into S buffer j & 1, which held S(j-2) / P(j-2): wait until both
-        // P V(j-2) have consumed it (they are issued by another thread)
-        const int ks_ = j % kStages;
-        if (j >= 2) ok = mbar_wait(BAR(B_SR + (j & 1)), ((j >> 1) - 1) & 1, abort_flag);
-        if (ok) ok = mbar_wait(BAR(B_KF + ks_), (j / kStages) & 1, abort_flag);
-        if (!ok) break;
-        tc_fence_after();
-        const uint64_t kdesc = smem_desc(base + kSmK + ks_ * kTileBytes, 16, 1024);
+        for (int ks = 0; ks < 8; ++ks)   // head_dim 128 = 8 steps of 16 channels
+          qdesc[ks] = smem_desc(base + kSmQ + qb * kTileBytes + (ks >> 2) * kHalfBytes + (ks & 3) * 32, 16, 1024);
+        for (int j = 0; j < w.n_tiles && ok; ++j) {
+          // S(G) = Q K^T into S buffer G & 1, which held S(G-2) / P(G-2): wait until both
+          // P V(G-2) have consumed it (they are issued by another thread)
+          const int Gj = G + j, sb = Gj & 1, ks_ = Gj % kKStages;
+          if (Gj >= 2) ok = mbar_wait(BAR(B_SR + sb), ((Gj >> 1) - 1) & 1, abort_flag);
+          if (ok) ok = mbar_wait(BAR(B_KF + ks_), (Gj / kKStages) & 1, abort_flag);
+          if (!ok) break;
+          tc_fence_after();
+          const uint64_t kdesc = smem_desc(base + kSmK + ks_ * kTileBytes, 16, 1024);
 #pragma unroll
-        for (int ks = 0; ks < 8; ++ks)
-          umma_bf16(tmem + kColS + (j & 1) * 128, qdesc[ks], kdesc + (uint64_t)((ks >> 2) * (kHalfBytes >> 4) + (ks & 3) * 2),
-                    kIdescS, ks > 0);
-        umma_commit(BAR(B_SF + (j & 1)));   // scores ready
-        umma_commit(BAR(B_KE + ks_));       // K stage free
+          for (int ks = 0; ks < 8; ++ks)
+            umma_bf16(tmem + kColS + sb * 128, qdesc[ks],
+                      kdesc + (uint64_t)((ks >> 2) * (kHalfBytes >> 4) + (ks & 3) * 2), kIdescS, ks > 0);
+          umma_commit(BAR(B_SF + sb));    // scores ready
+          umma_commit(BAR(B_KE + ks_));   // K stage free
+        }
+        if (ok) umma_commit(BAR(B_QE + qb));   // Q buffer free once this item's S products are done
+        G += w.n_tiles;
+        ++it;
       }
       if (!ok) atomicExch(p.status, kDevWaitTimeout);
     }
@@ -298,33 +350,43 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     if (lane == 0) {
       constexpr uint32_t kIdescPV = idesc_bf16(1);
       bool ok = true;
-      for (int j = 0; j < n_tiles && ok; ++j) {
-        const int vs = j % kStages;
-        ok = mbar_wait(BAR(B_VF + vs), (j / kStages) & 1, abort_flag);
-        const uint64_t vdesc = smem_desc(base + kSmV + vs * kTileBytes, kHalfBytes, 1024);
-        // serve the two streams in the order their P arrives (bounded polling)
-        bool done[2] = {false, false};
-        const long long t0 = clock64();
-        for (uint32_t it = 1; ok && !(done[0] && done[1]); ++it) {
+      int G = 0, it = 0;
+      for (int id = blockIdx.x; id < n_ids && ok; id += gridDim.x) {
+        const WorkItem w = get_item(p, id);
+        if (!w.valid) continue;
+        // the first P V of an item overwrites the O accumulators: the streams must have
+        // read the previous item's result
+        if (it >= 1) ok = mbar_wait(BAR(B_OR), (it - 1) & 1, abort_flag);
+        for (int j = 0; j < w.n_tiles && ok; ++j) {
+          const int Gj = G + j, sb = Gj & 1, vs = Gj % kVStages;
+          ok = mbar_wait(BAR(B_VF + vs), (Gj / kVStages) & 1, abort_flag);
+          const uint64_t vdesc = smem_desc(base + kSmV + vs * kTileBytes, kHalfBytes, 1024);
+          // serve the two streams in the order their P arrives (bounded polling)
+          bool done[2] = {false, false};
+          const long long t0 = clock64();
+          for (uint32_t n = 1; ok && !(done[0] && done[1]); ++n) {
 #pragma unroll
-          for (int hs = 0; hs < 2; ++hs) {
-            if (!done[hs] && mbar_test_wait(BAR(B_PF + hs), j & 1)) {
-              tc_fence_after();
-              // O_h += P_h(j) V_j[64 h .. 64 h + 63]: A = P from tensor memory (two bf16 per
-              // column), B = V MN-major (channels contiguous, keys strided by 128 B)
+            for (int hs = 0; hs < 2; ++hs) {
+              if (!done[hs] && mbar_test_wait(BAR(B_PF + hs), Gj & 1)) {
+                tc_fence_after();
+                // O_h += P_h V[64 h .. 64 h + 63]: A = P from tensor memory (two bf16 per
+                // column), B = V MN-major (channels contiguous, keys strided by 128 B)
 #pragma unroll
-              for (int ks = 0; ks < 4; ++ks)   // 64 keys = 4 steps of 16
-                umma_bf16_ts(tmem + kColO + hs * 128, tmem + kColS + (j & 1) * 128 + hs * 64 + ks * 8,
-                             vdesc + (uint64_t)((hs * 4 + ks) * (2048 >> 4)), kIdescPV, (j > 0 || ks > 0) ? 1u : 0u);
-              umma_commit(BAR(B_OF + hs));
-              done[hs] = true;
+                for (int ks = 0; ks < 4; ++ks)   // 64 keys = 4 steps of 16
+                  umma_bf16_ts(tmem + kColO + hs * 128, tmem + kColS + sb * 128 + hs * 64 + ks * 8,
+                               vdesc + (uint64_t)((hs * 4 + ks) * (2048 >> 4)), kIdescPV, (j > 0 || ks > 0) ? 1u : 0u);
+                umma_commit(BAR(B_OF + hs));
+                done[hs] = true;
+              }
             }
+            if ((n & 1023u) == 0 && (*abort_flag || clock64() - t0 > kWaitLimitCycles)) { *abort_flag = 1; ok = false; }
           }
-          if ((it & 1023u) == 0 && (*abort_flag || clock64() - t0 > kWaitLimitCycles)) { *abort_flag = 1; ok = false; }
+          if (!ok) break;
+          umma_commit(BAR(B_VE + vs));   // V stage free once both P V are done
+          umma_commit(BAR(B_SR + sb));   // and so is the S buffer
         }
-        if (!ok) break;
-        umma_commit(BAR(B_VE + vs));          // V stage free once both P V are done
-        umma_commit(BAR(B_SR + (j & 1)));     // and so is the S buffer
+        G += w.n_tiles;
+        ++it;
       }
       if (!ok) atomicExch(p.status, kDevWaitTimeout);
     }
@@ -333,122 +395,129 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     const int hs = (warp - 2) >> 2;       // stream: key columns [64 hs, 64 hs + 64) of every tile
     const int qd = warp & 3;              // TMEM lane quarter this warp may access
     const int r = qd * 32 + lane;         // query row within the tile
-    const int i = i0 + r;                 // query position
     const uint32_t lane_base = tmem + ((uint32_t)(qd * 32) << 16);
     const uint32_t o_addr = lane_base + kColO + hs * 128;
+    float2* xchg = reinterpret_cast<float2*>(gbase + kSmXchg);
     constexpr float kRescaleGap = 8.f;    // the exponent reference may lag the running max by 2^8
-    float m_ref = -INFINITY, l = 0.f;
     bool ok = true;
-    for (int j = 0; j < n_tiles; ++j) {
-      const int j0 = (jt_lo + j) * kBN + hs * 64;   // first key of this stream's columns
-      const uint32_t s_addr = lane_base + kColS + (j & 1) * 128 + hs * 64;
-      if (!__all_sync(0xffffffffu, mbar_wait(BAR(B_SF + (j & 1)), (j >> 1) & 1, abort_flag))) { ok = false; break; }
-      tc_fence_after();
-      uint32_t sv[64];
-      tmem_ld32(s_addr, *reinterpret_cast<uint32_t(*)[32]>(&sv[0]));
-      tmem_ld32(s_addr + 32, *reinterpret_cast<uint32_t(*)[32]>(&sv[32]));
-      tmem_wait_ld();
-      // band edges: causal (keys after the query) and window (keys older than i - window)
-      const bool edge = (j0 + 63 > i0) || (p.window > 0 && j0 <= i0 + kBM - 1 - p.window);
-      if (edge) {
-        const int k_max = i - j0;                                      // columns <= k_max are causal-visible
-        const int k_min = p.window > 0 ? i - p.window + 1 - j0 : 0;    // columns >= k_min are inside the window
-#pragma unroll
-        for (int e = 0; e < 64; ++e)
-          if (e > k_max || e < k_min) sv[e] = 0xff800000u;             // -inf
-      }
-      float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
-#pragma unroll
-      for (int e = 0; e < 64; e += 4) {
-        mx0 = fmaxf(mx0, __uint_as_float(sv[e]));
-        mx1 = fmaxf(mx1, __uint_as_float(sv[e + 1]));
-        mx2 = fmaxf(mx2, __uint_as_float(sv[e + 2]));
-        mx3 = fmaxf(mx3, __uint_as_float(sv[e + 3]));
-      }
-      const float mt = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * p.scale_log2e;
-      const bool grow = mt > m_ref + kRescaleGap;    // also true for the first visible key (m_ref = -inf)
-      if (__any_sync(0xffffffffu, grow)) {
-        const float alpha = grow ? ex2_approx(m_ref - mt) : 1.f;   // m_ref = -inf gives 0
-        if (j > 0) {   // the O row holds earlier tiles: rescale it once this stream's P V(j-1) has landed
-          if (!__all_sync(0xffffffffu, mbar_wait(BAR(B_OF + hs), (j - 1) & 1, abort_flag))) { ok = false; break; }
-          tc_fence_after();
-#pragma unroll
-          for (int c = 0; c < 4; ++c) {
-            uint32_t ov[32];
-            tmem_ld32(o_addr + c * 32, ov);
-            tmem_wait_ld();
-#pragma unroll
-            for (int e = 0; e < 32; ++e) ov[e] = __float_as_uint(__uint_as_float(ov[e]) * alpha);
-            tmem_st32(o_addr + c * 32, ov);
-          }
-        }
-        l *= alpha;
-        if (grow) m_ref = mt;
-      }
-      const float neg_m = m_ref == -INFINITY ? 0.f : -m_ref;   // no visible key yet: weights 0, no NaN
-      float sum0 = 0.f, sum1 = 0.f;
-      uint32_t pk[32];
-#pragma unroll
-      for (int e = 0; e < 64; e += 2) {
-        const float p0 = ex2_approx(fmaf(__uint_as_float(sv[e]), p.scale_log2e, neg_m));
-        const float p1 = ex2_approx(fmaf(__uint_as_float(sv[e + 1]), p.scale_log2e, neg_m));
-        sum0 += p0;
-        sum1 += p1;
-        pk[e >> 1] = pack_bf16(p0, p1);
-      }
-      l += sum0 + sum1;
-      // P (bf16 pairs) over the first 32 of this stream's 64 score columns
-      tmem_st32(s_addr, pk);
-      tmem_wait_st();
-      tc_fence_before();
-      // back-pressure: P(j) may only be announced once P V(j-1) of this stream has run, so the
-      // announcement barrier is never more than one phase ahead of the MMA thread
-      if (j > 0 && !__all_sync(0xffffffffu, mbar_wait(BAR(B_OF + hs), (j - 1) & 1, abort_flag))) { ok = false; break; }
-      __syncwarp();
-      if (lane == 0) mbar_arrive(BAR(B_PF + hs));
-    }
-    if (ok) ok = __all_sync(0xffffffffu, mbar_wait(BAR(B_OF + hs), (n_tiles - 1) & 1, abort_flag));
-    if (ok) {
-      // merge the two streams like split-KV partials: exchange (reference, sum) per row
-      tc_fence_after();
-      float2* xchg = reinterpret_cast<float2*>(gbase + kSmXchg);
-      xchg[hs * 128 + r] = make_float2(m_ref, l);
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(BAR(B_XC));
-      ok = __all_sync(0xffffffffu, mbar_wait(BAR(B_XC), 0, abort_flag));
-    }
-    if (ok) {
-      tc_fence_after();
-      const float2* xchg = reinterpret_cast<const float2*>(gbase + kSmXchg);
-      const float2 other = xchg[(hs ^ 1) * 128 + r];
-      const float m_all = fmaxf(m_ref, other.x);          // finite for every valid row (key i is visible)
-      const float w_me = ex2_approx(m_ref - m_all), w_ot = ex2_approx(other.x - m_all);   // 2^-inf = 0
-      const float inv = 1.f / (l * w_me + other.y * w_ot);
-      const float w_lo = (hs == 0 ? w_me : w_ot) * inv, w_hi = (hs == 0 ? w_ot : w_me) * inv;
-      // this thread writes channels [64 hs, 64 hs + 64) of its row from both accumulators
-      __nv_bfloat16* orow = p.out + ((int64_t)(row_base + i) * p.n_q_heads + h) * 128 + hs * 64;
-#pragma unroll
-      for (int c = 0; c < 2; ++c) {
-        uint32_t olo[32], ohi[32];
-        tmem_ld32(lane_base + kColO + hs * 64 + c * 32, olo);
-        tmem_ld32(lane_base + kColO + 128 + hs * 64 + c * 32, ohi);
+    int G = 0, it = 0;
+    for (int id = blockIdx.x; id < n_ids && ok; id += gridDim.x) {
+      const WorkItem w = get_item(p, id);
+      if (!w.valid) continue;
+      const int i = w.i0 + r;             // query position
+      float m_ref = -INFINITY, l = 0.f;
+      for (int j = 0; j < w.n_tiles; ++j) {
+        const int Gj = G + j, sb = Gj & 1;
+        const int j0 = (w.jt_lo + j) * kBN + hs * 64;   // first key of this stream's columns
+        const uint32_t s_addr = lane_base + kColS + sb * 128 + hs * 64;
+        if (!__all_sync(0xffffffffu, mbar_wait(BAR(B_SF + sb), (Gj >> 1) & 1, abort_flag))) { ok = false; break; }
+        tc_fence_after();
+        uint32_t sv[64];
+        tmem_ld32(s_addr, *reinterpret_cast<uint32_t(*)[32]>(&sv[0]));
+        tmem_ld32(s_addr + 32, *reinterpret_cast<uint32_t(*)[32]>(&sv[32]));
         tmem_wait_ld();
-        if (i < S) {
+        // band edges: causal (keys after the query) and window (keys older than i - window)
+        const bool edge = (j0 + 63 > w.i0) || (p.window > 0 && j0 <= w.i0 + kBM - 1 - p.window);
+        if (edge) {
+          const int k_max = i - j0;                                      // columns <= k_max are causal-visible
+          const int k_min = p.window > 0 ? i - p.window + 1 - j0 : 0;    // columns >= k_min are inside the window
 #pragma unroll
-          for (int q4 = 0; q4 < 4; ++q4) {
-            uint32_t w[4];
+          for (int e = 0; e < 64; ++e)
+            if (e > k_max || e < k_min) sv[e] = 0xff800000u;             // -inf
+        }
+        float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
+#pragma unroll
+        for (int e = 0; e < 64; e += 4) {
+          mx0 = fmaxf(mx0, __uint_as_float(sv[e]));
+          mx1 = fmaxf(mx1, __uint_as_float(sv[e + 1]));
+          mx2 = fmaxf(mx2, __uint_as_float(sv[e + 2]));
+          mx3 = fmaxf(mx3, __uint_as_float(sv[e + 3]));
+        }
+        const float mt = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * p.scale_log2e;
+        const bool grow = mt > m_ref + kRescaleGap;    // also true for the first visible key (m_ref = -inf)
+        if (__any_sync(0xffffffffu, grow)) {
+          const float alpha = grow ? ex2_approx(m_ref - mt) : 1.f;   // m_ref = -inf gives 0
+          if (j > 0) {   // the O row holds earlier tiles: rescale it once this stream's previous P V has landed
+            if (!__all_sync(0xffffffffu, mbar_wait(BAR(B_OF + hs), (Gj - 1) & 1, abort_flag))) { ok = false; break; }
+            tc_fence_after();
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+              uint32_t ov[32];
+              tmem_ld32(o_addr + c * 32, ov);
+              tmem_wait_ld();
+#pragma unroll
+              for (int e = 0; e < 32; ++e) ov[e] = __float_as_uint(__uint_as_float(ov[e]) * alpha);
+              tmem_st32(o_addr + c * 32, ov);
+            }
+          }
+          l *= alpha;
+          if (grow) m_ref = mt;
+        }
+        const float neg_m = m_ref == -INFINITY ? 0.f : -m_ref;   // no visible key yet: weights 0, no NaN
+        float sum0 = 0.f, sum1 = 0.f;
+        uint32_t pk[32];
+#pragma unroll
+        for (int e = 0; e < 64; e += 2) {
+          const float p0 = ex2_approx(fmaf(__uint_as_float(sv[e]), p.scale_log2e, neg_m));
+          const float p1 = ex2_approx(fmaf(__uint_as_float(sv[e + 1]), p.scale_log2e, neg_m));
+          sum0 += p0;
+          sum1 += p1;
+          pk[e >> 1] = pack_bf16(p0, p1);
+        }
+        l += sum0 + sum1;
+        // P (bf16 pairs) over the first 32 of this stream's 64 score columns
+        tmem_st32(s_addr, pk);
+        tmem_wait_st();
+        tc_fence_before();
+        // back-pressure: P may only be announced once this stream's previous P V has run, so
+        // the announcement barrier is never more than one phase ahead of the MMA thread
+        if (Gj > 0 && !__all_sync(0xffffffffu, mbar_wait(BAR(B_OF + hs), (Gj - 1) & 1, abort_flag))) { ok = false; break; }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(BAR(B_PF + hs));
+      }
+      G += w.n_tiles;
+      if (ok) ok = __all_sync(0xffffffffu, mbar_wait(BAR(B_OF + hs), (G - 1) & 1, abort_flag));
+      if (ok) {
+        // merge the two streams like split-KV partials: exchange (reference, sum) per row
+        tc_fence_after();
+        xchg[hs * 128 + r] = make_float2(m_ref, l);
+        __syncwarp();
+        if (lane == 0) mbar_arrive(BAR(B_XC));
+        ok = __all_sync(0xffffffffu, mbar_wait(BAR(B_XC), it & 1, abort_flag));
+      }
+      if (ok) {
+        tc_fence_after();
+        const float2 other = xchg[(hs ^ 1) * 128 + r];
+        const float m_all = fmaxf(m_ref, other.x);          // finite for every valid row (key i is visible)
+        const float w_me = ex2_approx(m_ref - m_all), w_ot = ex2_approx(other.x - m_all);   // 2^-inf = 0
+        const float inv = 1.f / (l * w_me + other.y * w_ot);
+        const float w_lo = (hs == 0 ? w_me : w_ot) * inv, w_hi = (hs == 0 ? w_ot : w_me) * inv;
+        // this thread writes channels [64 hs, 64 hs + 64) of its row from both accumulators
+        uint32_t olo[64], ohi[64];
+        tmem_ld32(lane_base + kColO + hs * 64, *reinterpret_cast<uint32_t(*)[32]>(&olo[0]));
+        tmem_ld32(lane_base + kColO + hs * 64 + 32, *reinterpret_cast<uint32_t(*)[32]>(&olo[32]));
+        tmem_ld32(lane_base + kColO + 128 + hs * 64, *reinterpret_cast<uint32_t(*)[32]>(&ohi[0]));
+        tmem_ld32(lane_base + kColO + 128 + hs * 64 + 32, *reinterpret_cast<uint32_t(*)[32]>(&ohi[32]));
+        tmem_wait_ld();
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(BAR(B_OR));   // the accumulators may be overwritten by the next item
+        if (i < w.S) {
+          __nv_bfloat16* orow = p.out + ((int64_t)(w.row_base + i) * p.n_q_heads + w.h) * 128 + hs * 64;
+#pragma unroll
+          for (int q8 = 0; q8 < 8; ++q8) {
+            uint32_t o4[4];
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
-              const int d = q4 * 8 + e * 2;
-              w[e] = pack_bf16(__uint_as_float(olo[d]) * w_lo + __uint_as_float(ohi[d]) * w_hi,
-                               __uint_as_float(olo[d + 1]) * w_lo + __uint_as_float(ohi[d + 1]) * w_hi);
+              const int d = q8 * 8 + e * 2;
+              o4[e] = pack_bf16(__uint_as_float(olo[d]) * w_lo + __uint_as_float(ohi[d]) * w_hi,
+                                __uint_as_float(olo[d + 1]) * w_lo + __uint_as_float(ohi[d + 1]) * w_hi);
             }
-            *reinterpret_cast<uint4*>(orow + c * 32 + q4 * 8) = make_uint4(w[0], w[1], w[2], w[3]);
+            *reinterpret_cast<uint4*>(orow + q8 * 8) = make_uint4(o4[0], o4[1], o4[2], o4[3]);
           }
         }
       }
-      tc_fence_before();
+      ++it;
     }
     if (!ok && lane == 0) atomicExch(p.status, kDevWaitTimeout);
   }
@@ -502,7 +571,7 @@ cudaError_t prepare_prefill_tc() {
   return cudaFuncSetAttribute(prefill_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
 }
 
-cudaError_t launch_prefill_tc(const PrefillParams& pp, int max_len, cudaStream_t st) {
+cudaError_t launch_prefill_tc(const PrefillParams& pp, int max_len, int sm_count, cudaStream_t st) {
   if (pp.n_seqs <= 0 || max_len <= 0) return cudaSuccess;
   const int64_t rows = pp.row0[pp.n_seqs];
   CUtensorMap tq, tk, tv;
@@ -518,7 +587,9 @@ cudaError_t launch_prefill_tc(const PrefillParams& pp, int max_len, cudaStream_t
   p.status = pp.status;
   p.out = static_cast<__nv_bfloat16*>(pp.out);
   for (int i = 0; i <= pp.n_seqs; ++i) p.row0[i] = pp.row0[i];
-  dim3 grid((max_len + kBM - 1) / kBM, pp.n_q_heads, pp.n_seqs);
+  p.max_qt = (max_len + kBM - 1) / kBM;
+  const int64_t n_ids = (int64_t)p.max_qt * pp.n_seqs * pp.n_q_heads;
+  const int grid = (int)(n_ids < sm_count ? n_ids : sm_count);   // persistent: one CTA per SM
   prefill_tc_kernel<<<grid, kThreads, kSmemBytes, st>>>(tq, tk, tv, p);
   return cudaGetLastError();
 }
