@@ -10,8 +10,8 @@
 //   warp 1     one elected thread issues the tcgen05.mma (K16 steps, bf16 -> fp32 in TMEM) of
 //              S = Q K^T (M128 N128, both operands from shared memory) into one of two S
 //              buffers, two tiles ahead of the softmax
-//   warp 10    one elected thread issues O_h += P_h V_h with P_h read from tensor memory
-//              and V MN-major from its row-major tile
+//   warps 10-11  one elected thread per stream issues O_h += P_h V_h with P_h read from
+//              tensor memory and V MN-major from its row-major tile
 //   warps 2-5  softmax stream "lo": key columns 0-63 of every tile; warps 6-9 stream "hi":
 //              columns 64-127.  The two streams are independent flash-attention passes
 //              over interleaved halves of the keys (own running max, own row sum, own O
@@ -40,7 +40,7 @@ constexpr int kBM = 128;                       // queries per work item
 constexpr int kBN = 128;                       // keys per tile
 constexpr int kHalfBytes = 128 * 128;          // one [128 rows x 64 bf16] swizzled block
 constexpr int kTileBytes = 2 * kHalfBytes;     // a 128 x 128 bf16 operand tile
-constexpr int kThreads = 352;                  // TMA warp, S-MMA warp, 2 x 4 softmax warps, PV-MMA warp
+constexpr int kThreads = 384;                  // TMA warp, S-MMA warp, 2 x 4 softmax warps, 2 PV-MMA warps
 constexpr int kKStages = 3, kVStages = 2;
 constexpr int kSmQ = 0;                        // two Q buffers (this item / next item)
 constexpr int kSmK = kSmQ + 2 * kTileBytes;
@@ -87,16 +87,6 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   asm volatile(
       "{\n\t.reg .pred p;\n\t"
       "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-  return ok != 0;
-}
-// Non-blocking probe (try_wait may suspend the thread for a while before it answers).
-__device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
       "selp.u32 %0, 1, 0, p;\n\t}"
       : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
   return ok != 0;
@@ -229,9 +219,9 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
       mbar_init(BAR(B_QF + s), 1);
       mbar_init(BAR(B_QE + s), 1);
       mbar_init(BAR(B_VF + s), 1);
-      mbar_init(BAR(B_VE + s), 1);
+      mbar_init(BAR(B_VE + s), 2);   // both P V issuers
       mbar_init(BAR(B_SF + s), 1);
-      mbar_init(BAR(B_SR + s), 1);
+      mbar_init(BAR(B_SR + s), 2);   // both P V issuers
       mbar_init(BAR(B_PF + s), 4);
       mbar_init(BAR(B_OF + s), 1);
     }
@@ -308,8 +298,9 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     }
   } else if (warp == 1) {
     // ------------------------------ MMA issuer, scores ------------------------------
-    // Two threads issue MMAs (this one S = Q K^T, warp 10 the P V products): issuing is a
-    // serial, latency-bound instruction stream, and one thread alone was the bottleneck.
+    // Three threads issue MMAs (this one S = Q K^T, warps 10 and 11 the P V products of the
+    // two streams): issuing is a serial, latency-bound instruction stream, and one thread
+    // alone was the bottleneck.
     if (lane == 0) {
       constexpr uint32_t kIdescS = idesc_bf16(0);
       bool ok = true;
@@ -345,44 +336,34 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
       }
       if (!ok) atomicExch(p.status, kDevWaitTimeout);
     }
-  } else if (warp == 10) {
-    // ------------------------------ MMA issuer, P V ------------------------------
+  } else if (warp >= 10) {
+    // ------------------------------ MMA issuers, P V (one per stream) ------------------------------
     if (lane == 0) {
       constexpr uint32_t kIdescPV = idesc_bf16(1);
+      const int hs = warp - 10;
       bool ok = true;
       int G = 0, it = 0;
       for (int id = blockIdx.x; id < n_ids && ok; id += gridDim.x) {
         const WorkItem w = get_item(p, id);
         if (!w.valid) continue;
-        // the first P V of an item overwrites the O accumulators: the streams must have
+        // the first P V of an item overwrites the O accumulator: the streams must have
         // read the previous item's result
         if (it >= 1) ok = mbar_wait(BAR(B_OR), (it - 1) & 1, abort_flag);
         for (int j = 0; j < w.n_tiles && ok; ++j) {
           const int Gj = G + j, sb = Gj & 1, vs = Gj % kVStages;
           ok = mbar_wait(BAR(B_VF + vs), (Gj / kVStages) & 1, abort_flag);
-          const uint64_t vdesc = smem_desc(base + kSmV + vs * kTileBytes, kHalfBytes, 1024);
-          // serve the two streams in the order their P arrives (bounded polling)
-          bool done[2] = {false, false};
-          const long long t0 = clock64();
-          for (uint32_t n = 1; ok && !(done[0] && done[1]); ++n) {
-#pragma unroll
-            for (int hs = 0; hs < 2; ++hs) {
-              if (!done[hs] && mbar_test_wait(BAR(B_PF + hs), Gj & 1)) {
-                tc_fence_after();
-                // O_h += P_h V[64 h .. 64 h + 63]: A = P from tensor memory (two bf16 per
-                // column), B = V MN-major (channels contiguous, keys strided by 128 B)
-#pragma unroll
-                for (int ks = 0; ks < 4; ++ks)   // 64 keys = 4 steps of 16
-                  umma_bf16_ts(tmem + kColO + hs * 128, tmem + kColS + sb * 128 + hs * 64 + ks * 8,
-                               vdesc + (uint64_t)((hs * 4 + ks) * (2048 >> 4)), kIdescPV, (j > 0 || ks > 0) ? 1u : 0u);
-                umma_commit(BAR(B_OF + hs));
-                done[hs] = true;
-              }
-            }
-            if ((n & 1023u) == 0 && (*abort_flag || clock64() - t0 > kWaitLimitCycles)) { *abort_flag = 1; ok = false; }
-          }
+          if (ok) ok = mbar_wait(BAR(B_PF + hs), Gj & 1, abort_flag);
           if (!ok) break;
-          umma_commit(BAR(B_VE + vs));   // V stage free once both P V are done
+          tc_fence_after();
+          // O_h += P_h V[64 h .. 64 h + 63]: A = P from tensor memory (two bf16 per column),
+          // B = V MN-major (channels contiguous, keys strided by 128 B)
+          const uint64_t vdesc = smem_desc(base + kSmV + vs * kTileBytes + hs * 4 * 2048, kHalfBytes, 1024);
+#pragma unroll
+          for (int ks = 0; ks < 4; ++ks)   // 64 keys = 4 steps of 16
+            umma_bf16_ts(tmem + kColO + hs * 128, tmem + kColS + sb * 128 + hs * 64 + ks * 8,
+                         vdesc + (uint64_t)(ks * (2048 >> 4)), kIdescPV, (j > 0 || ks > 0) ? 1u : 0u);
+          umma_commit(BAR(B_OF + hs));   // this stream's accumulator is up to date
+          umma_commit(BAR(B_VE + vs));   // V stage free once both streams' P V are done (count 2)
           umma_commit(BAR(B_SR + sb));   // and so is the S buffer
         }
         G += w.n_tiles;
