@@ -232,6 +232,16 @@ def prefill_figures(mx, runner, peaks, device):
     return res
 
 
+def reduce_over_ranks(dist, times, work, device):
+    """Replicas-only aggregation: times -> max over ranks, work -> sum over ranks.
+    (No data-path collective exists; this is the only communication of a run.)"""
+    t = torch.tensor([float(x) for x in times], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    w = torch.tensor([float(x) for x in work], device=device, dtype=torch.float64)
+    dist.all_reduce(w, op=dist.ReduceOp.SUM)
+    return t.tolist(), w.tolist()
+
+
 def run_gpu_arm(args, wl):
     from paper_2409_15012_b200 import build as mbuild
     rank = int(os.environ.get("RANK", "0"))
@@ -353,12 +363,8 @@ def run_gpu_arm(args, wl):
 
     # ---- max over ranks, sum of work ----
     if dist is not None:
-        t = torch.tensor([ms, e2e_ms], device=sess.dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms, e2e_ms = t.tolist()
-        w = torch.tensor([float(kv_bytes), float(e2e_bytes), float(launches)], device=sess.dev, dtype=torch.float64)
-        dist.all_reduce(w, op=dist.ReduceOp.SUM)
-        kv_bytes, e2e_bytes, launches = w.tolist()
+        (ms, e2e_ms), (kv_bytes, e2e_bytes, launches) = reduce_over_ranks(
+            dist, [ms, e2e_ms], [kv_bytes, e2e_bytes, launches], sess.dev)
     if rank != 0:
         sess.close()
         dist.destroy_process_group()
