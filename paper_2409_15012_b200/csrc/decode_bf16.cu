@@ -137,11 +137,11 @@ __device__ __forceinline__ Item decode_item(const DecodeParams& p, int it) {
   int r = it / p.head_chunks;
   x.g = r % p.geom.n_kv_heads;
   const int cg = r / p.geom.n_kv_heads;  // global split index
-  int lo = 0, hi = p.n_seqs;             // last i with chunk_base[i] <= cg
-  while (hi - lo > 1) {
-    const int mid = (lo + hi) >> 1;
-    if (p.chunk_base[mid] <= cg) lo = mid; else hi = mid;
-  }
+  // last i with chunk_base[i] <= cg: proportional guess, then a short walk (batches of equal
+  // lengths hit at once; each probe is a dependent parameter load, so few probes matter)
+  int lo = (int)(((long long)cg * p.n_seqs) / p.chunk_base[p.n_seqs]);
+  while (p.chunk_base[lo] > cg) --lo;
+  while (p.chunk_base[lo + 1] <= cg) ++lo;
   x.i = lo;
   x.c = cg - p.chunk_base[lo];
   x.n_splits = p.chunk_base[lo + 1] - p.chunk_base[lo];
@@ -171,6 +171,10 @@ decode_split_bf16_kernel(const __grid_constant__ DecodeParams p, const int n_sta
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
 
+  // Programmatic dependent launch: let the next kernel of the stream begin its launch and
+  // set-up as soon as every CTA of this one is running ...
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+
   if (threadIdx.x == 0) {
     for (int s = 0; s < n_stages; ++s) {
       mbar_init(full0 + 8 * s, 1);
@@ -181,6 +185,9 @@ decode_split_bf16_kernel(const __grid_constant__ DecodeParams p, const int n_sta
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   __syncthreads();
+  // ... and do not touch global memory before the kernels ahead in the stream have
+  // completed and flushed (a no-op when this kernel was launched the ordinary way)
+  asm volatile("griddepcontrol.wait;" ::: "memory");
 
   const KvGeom& ge = p.geom;
 
@@ -414,11 +421,21 @@ cudaError_t launch_decode_split_bf16(const DecodeParams& p, int sm_count, cudaSt
   const size_t smem = smem_bytes(D, p.group, n_stages);
   const int grid = p.total_items < sm_count ? p.total_items : sm_count;
   if (grid <= 0) return cudaSuccess;
-  if (D == 128)
-    decode_split_bf16_kernel<128><<<grid, kThreads, smem, st>>>(p, n_stages);
-  else
-    decode_split_bf16_kernel<64><<<grid, kThreads, smem, st>>>(p, n_stages);
-  return cudaGetLastError();
+  // launched with programmatic stream serialization: the kernel's set-up may overlap the
+  // tail of the previous kernel in the stream; it waits (griddepcontrol.wait) before its
+  // first global access
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(grid);
+  cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  if (D == 128) return cudaLaunchKernelEx(&cfg, decode_split_bf16_kernel<128>, p, n_stages);
+  return cudaLaunchKernelEx(&cfg, decode_split_bf16_kernel<64>, p, n_stages);
 }
 
 }  // namespace mixattn
