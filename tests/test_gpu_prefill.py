@@ -88,3 +88,53 @@ def test_prefill_errors():
         torch.cuda.synchronize()
     finally:
         sess.close()
+
+
+def _prefill_direct(mx, wl, seq_lens, layer):
+    """One prefill call with per-sequence lengths (packed tensors); returns (out, q, k, v) on the CPU."""
+    dt = torch_dt(wl.dtype)
+    kind, W, owner = wl.layout[layer]
+    qs, ks, vs = [], [], []
+    for b, S in enumerate(seq_lens):
+        qs.append(si.q_tokens(wl.seed, layer, b, 0, S, wl.n_q_heads, wl.head_dim, dt))
+        K, V = si.kv_tokens(wl.seed, owner, b, 0, S, wl.n_kv_heads, wl.head_dim, dt)
+        ks.append(K)
+        vs.append(V)
+    return torch.cat(qs), torch.cat(ks), torch.cat(vs)
+
+
+@pytest.mark.parametrize("hq,hkv,d,dtype", [(8, 8, 128, cf.BF16), (12, 3, 128, cf.BF16), (2, 1, 128, cf.BF16),
+                                            (8, 2, 64, cf.BF16), (6, 3, 128, cf.F32)])
+def test_prefill_head_shapes_and_ragged_lengths(hq, hkv, d, dtype):
+    # MHA, the paper's 12/3, a single pair, head_dim 64 (CUDA-core path), fp32; sequences of
+    # different lengths packed in one call, one of them a single token
+    mx, runner = load_lib()
+    seq_lens = [333, 129, 1, 128]
+    wl = cf.prefill_chunk().scaled(layout=cf.layout_tiny(100), batch=len(seq_lens), seq_len=max(seq_lens),
+                                   n_q_heads=hq, n_kv_heads=hkv, head_dim=d, dtype=dtype)
+    sess = runner.Session(wl, [0] * wl.batch, headroom_tokens=2)
+    ph = mo.PhysicalCache(wl.layout, hkv, d, wl.batch, sess.n_pages, store_values=False)
+    try:
+        ids = list(range(wl.batch))
+        for l, (kind, W, owner) in enumerate(wl.layout):
+            q, k, v = _prefill_direct(mx, wl, seq_lens, l)
+            qd, kd, vd = q.cuda(), k.cuda(), v.cuda()
+            out = torch.full_like(qd, float("nan"))
+            sess.ctx.prefill(l, ids, seq_lens, qd, kd, vd, out)
+            if owner == l:
+                ph.append(l, ids, seq_lens)
+            torch.cuda.synchronize()
+            got = out.float().cpu().double().numpy()
+            row = 0
+            for b, S in enumerate(seq_lens):
+                ref = mo.prefill_attention(q[row:row + S], k[row:row + S], v[row:row + S], kind, W)
+                check_close(got[row:row + S], ref, wl.dtype, f"layer {l} seq {b} len {S}")
+                row += S
+        assert sess.ctx.get_device_status() == 0
+        compare_state(sess.ctx, ph, wl)
+        sess.pos[:] = seq_lens
+        for b, S in enumerate(seq_lens):
+            check_stored_bits(sess.ctx, ph, wl, 1, b, sorted({max(0, S - 100), S - 1}))
+            check_stored_bits(sess.ctx, ph, wl, 0, b, sorted({0, S // 2, S - 1}))
+    finally:
+        sess.close()
