@@ -131,9 +131,9 @@ cudaError_t launch_recorded(mixattn_ctx* c, int cls, cudaStream_t st, F&& f) {
   return e;
 }
 
-int validate_config(const mixattn_config* cfg, CacheManager* cm) {
+int validate_config(const mixattn_config* cfg, CacheManager* cm, bool allocate = true) {
   if (cfg == nullptr) return MIXATTN_ERR_INVALID_ARG;
-  int rc = cm->init(*cfg);
+  int rc = cm->init(*cfg, allocate);
   if (rc != MIXATTN_OK) return rc;
   if (cfg->softmax_scale < 0.f || !isfinite(cfg->softmax_scale)) return MIXATTN_ERR_INVALID_ARG;
   if (cm->n_full_owners() > 0 && cfg->n_pages < 1) return MIXATTN_ERR_INVALID_ARG;
@@ -220,7 +220,7 @@ extern "C" {
 int mixattn_arena_bytes(const mixattn_config* cfg, size_t* out_bytes) {
   if (out_bytes == nullptr) return MIXATTN_ERR_INVALID_ARG;
   CacheManager cm;
-  int rc = validate_config(cfg, &cm);
+  int rc = validate_config(cfg, &cm, false);
   if (rc != MIXATTN_OK) return rc;
   *out_bytes = plan_arena(cm, *cfg).total;
   return MIXATTN_OK;
@@ -229,7 +229,7 @@ int mixattn_arena_bytes(const mixattn_config* cfg, size_t* out_bytes) {
 int mixattn_cache_bytes(const mixattn_config* cfg, size_t* out_bytes) {
   if (out_bytes == nullptr) return MIXATTN_ERR_INVALID_ARG;
   CacheManager cm;
-  int rc = validate_config(cfg, &cm);
+  int rc = validate_config(cfg, &cm, false);
   if (rc != MIXATTN_OK) return rc;
   *out_bytes = plan_arena(cm, *cfg).cache_bytes;
   return MIXATTN_OK;

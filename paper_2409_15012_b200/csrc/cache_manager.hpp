@@ -33,7 +33,8 @@ class CacheManager {
   static constexpr int kPageSize = 16;
 
   // Validates the config; returns MIXATTN_OK or an error code (then *this is unusable).
-  int init(const mixattn_config& cfg) {
+  // `allocate` false: only resolve the layout and sizes (for the byte-count queries).
+  int init(const mixattn_config& cfg, bool allocate = true) {
     if (cfg.n_layers <= 0 || cfg.layers == nullptr) return MIXATTN_ERR_INVALID_LAYOUT;
     if (cfg.n_q_heads <= 0 || cfg.n_kv_heads <= 0 || cfg.n_q_heads % cfg.n_kv_heads != 0)
       return MIXATTN_ERR_INVALID_ARG;
@@ -78,14 +79,16 @@ class CacheManager {
         int32_t pg = cfg.free_order[i];
         if (pg < 0 || pg >= cfg.n_pages || seen[pg]) return MIXATTN_ERR_INVALID_ARG;
         seen[pg] = 1;
-        free_.push_back(pg);
+        if (allocate) free_.push_back(pg);
       }
-    } else {
+    } else if (allocate) {
       for (int i = 0; i < cfg.n_pages; ++i) free_.push_back(i);
     }
-    table_.assign((size_t)max_seqs_ * max_blocks_, -1);
-    n_blocks_.assign(max_seqs_, 0);
-    len_.assign(owners_.size() * (size_t)max_seqs_, 0);
+    if (allocate) {
+      table_.assign((size_t)max_seqs_ * max_blocks_, -1);
+      n_blocks_.assign(max_seqs_, 0);
+      len_.assign(owners_.size() * (size_t)max_seqs_, 0);
+    }
     return MIXATTN_OK;
   }
 
