@@ -173,20 +173,21 @@ __host__ __device__ constexpr uint32_t idesc_bf16(int b_mn) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)b_mn << 16) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
 }
 
-// One work item: query tile qt of head h of sequence b.  Ids enumerate (reverse tile
-// index, sequence, head), so the heaviest tiles of all heads come first and the heads of
-// a KV group, which read the same K/V tiles, run at the same time on neighbouring SMs.
+// One work item: query tile qt of head h of sequence b.  Ids enumerate (sequence, reverse
+// tile index, head): the CTAs of the grid work on one sequence at a time, whose K/V stays
+// in L2 (a pass over all sequences at once re-read K/V from HBM 5x), heaviest tiles first,
+// and the heads of a KV group, which read the same K/V tiles, run at the same time.
 struct WorkItem {
   int h, g, row_base, S, i0, jt_lo, n_tiles;
   bool valid;
 };
 __device__ __forceinline__ WorkItem get_item(const TcParams& p, int id) {
   WorkItem w;
-  const int per_tile = p.n_seqs * p.n_q_heads;
-  const int qt_rev = id / per_tile;
-  const int rem = id - qt_rev * per_tile;
-  const int b = rem / p.n_q_heads;
-  w.h = rem - b * p.n_q_heads;
+  const int per_seq = p.max_qt * p.n_q_heads;
+  const int b = id / per_seq;
+  const int rem = id - b * per_seq;
+  const int qt_rev = rem / p.n_q_heads;
+  w.h = rem - qt_rev * p.n_q_heads;
   w.g = w.h / p.group;
   w.row_base = p.row0[b];
   w.S = p.row0[b + 1] - p.row0[b];
