@@ -115,3 +115,47 @@ def test_decode_errors_write_nothing():
         assert sess.ctx.get_launch_count() > 0
     finally:
         sess.close()
+
+
+def test_repeated_calls_are_bit_identical_and_profile_hooks_count():
+    # the same decode / prefill call twice gives the same bits (no order-dependent reduction
+    # across CTAs), and the per-kernel event hooks see every launch
+    from gpu_common import load_lib
+    mx, runner = load_lib()
+    wl = cf.mid_decode().scaled(batch=5, context=9000)
+    sess = runner.Session(wl, [9000, 4097, 1024, 300, 17], headroom_tokens=2)
+    try:
+        sess.fill(1500)
+        inputs = sess.step_inputs()
+        outs = sess.alloc_outputs()
+        sess.decode_step(inputs, outs)
+        ids = list(range(wl.batch))
+        sess.ctx.profile_enable(True)
+        for l in (0, 1, 5, 12, 23):
+            a = torch.empty_like(outs[l])
+            b = torch.empty_like(outs[l])
+            sess.ctx.decode(l, ids, inputs[l]["q"], a)
+            sess.ctx.decode(l, ids, inputs[l]["q"], b)
+            torch.cuda.synchronize()
+            assert torch.equal(a.view(torch.int16), b.view(torch.int16))
+            assert torch.equal(a.view(torch.int16), outs[l].view(torch.int16))
+        n_full, ms_full = sess.ctx.profile_read(mx.K_DECODE_FULL)
+        n_slide, ms_slide = sess.ctx.profile_read(mx.K_DECODE_SLIDING)
+        n_comb, _ = sess.ctx.profile_read(mx.K_COMBINE)
+        assert (n_full, n_slide) == (4, 6) and ms_full > 0 and ms_slide > 0 and n_comb == 4
+        sess.ctx.profile_enable(False)
+        assert sess.ctx.get_device_status() == 0
+    finally:
+        sess.close()
+    wl = cf.prefill_chunk().scaled(layout=cf.layout_tiny(256), batch=2, seq_len=700)
+    sess = runner.Session(wl, [0, 0])
+    try:
+        for l in (2, 3):      # readers: repeatable, store nothing
+            q, k, v = sess.prefill_inputs(l)
+            a, b = torch.empty_like(q), torch.empty_like(q)
+            sess.prefill_layer(l, q, k, v, a)
+            sess.prefill_layer(l, q, k, v, b)
+            torch.cuda.synchronize()
+            assert torch.equal(a.view(torch.int16), b.view(torch.int16))
+    finally:
+        sess.close()
