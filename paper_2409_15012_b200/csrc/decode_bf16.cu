@@ -31,9 +31,7 @@ namespace mixattn {
 
 namespace {
 
-constexpr int kConsumerWarps = 8;
 constexpr int kGroupWarps = 4;                      // warps (= pages) per stage
-constexpr int kThreads = (kConsumerWarps + 1) * 32;
 constexpr int kTileKeys = kGroupWarps * kPage;      // 64 keys per stage
 constexpr int kMaxStages = 8;
 constexpr long long kWaitLimitCycles = 4000000000ll;   // about two seconds of SM clock
@@ -118,8 +116,9 @@ __device__ __forceinline__ uint32_t movmatrix_t(uint32_t a) {  // transpose an 8
   asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(d) : "r"(a));
   return d;
 }
-__device__ __forceinline__ void consumer_bar() {  // the 256 consumer threads only
-  asm volatile("bar.sync 1, %0;" ::"n"(kConsumerWarps * 32) : "memory");
+template <int NCW>
+__device__ __forceinline__ void consumer_bar() {  // the consumer threads only
+  asm volatile("bar.sync 1, %0;" ::"n"(NCW * 32) : "memory");
 }
 
 struct Item {
@@ -150,9 +149,14 @@ __device__ __forceinline__ Item decode_item(const DecodeParams& p, int it) {
   return x;
 }
 
-template <int D>
-__global__ void __launch_bounds__(kThreads, 1)
+// NCW consumer warps: 8 (two groups alternating stages; one CTA per SM with a deep ring, for
+// long key streams) or 4 (one group; two CTAs per SM with short rings, so that a launch with
+// few, short work items keeps every item in flight at once instead of queueing two per SM).
+template <int D, int NCW>
+__global__ void __launch_bounds__((NCW + 1) * 32, NCW == 8 ? 1 : 2)
 decode_split_bf16_kernel(const __grid_constant__ DecodeParams p, const int n_stages) {
+  constexpr int kConsumerWarps = NCW;
+  constexpr int kGroups = NCW / kGroupWarps;
   constexpr int kRowBytes = D * 2;
   constexpr int kBlkBytes = 2 * kPage * kRowBytes;       // K+V of one (page, head)
   constexpr int kStageBytes = kGroupWarps * kBlkBytes;
@@ -282,7 +286,7 @@ decode_split_bf16_kernel(const __grid_constant__ DecodeParams p, const int n_sta
     const int n_tiles = ((x.t1 + kPage - 1) / kPage - x.t0 / kPage + kGroupWarps - 1) / kGroupWarps;
     for (int k = 0; k < n_tiles; ++k) {
       const int Kg = K + k;
-      if ((Kg & 1) != grp) continue;
+      if ((Kg % kGroups) != grp) continue;
       const int s = Kg % n_stages;
       // every lane waits (each needs to observe the copy), the verdict is warp-uniform
       if (!__all_sync(0xffffffffu, mbar_wait(full0 + 8 * s, (Kg / n_stages) & 1, abort_flag))) break;
@@ -367,7 +371,7 @@ decode_split_bf16_kernel(const __grid_constant__ DecodeParams p, const int n_sta
         if (frow == 0) { mml[r * 2] = m[e]; mml[r * 2 + 1] = l[e]; }
       }
     }
-    consumer_bar();
+    consumer_bar<NCW>();
     if (*abort_flag) {  // uniform: set before the barrier by whichever role gave up
       if (threadIdx.x == 0) atomicExch(p.status, kDevWaitTimeout);
       return;
@@ -394,39 +398,48 @@ decode_split_bf16_kernel(const __grid_constant__ DecodeParams p, const int n_sta
         if (d == 0) p.part_ml[slot] = make_float2(M, L);
       }
     }
-    consumer_bar();
+    consumer_bar<NCW>();
   }
 }
 
-size_t smem_bytes(int D, int group, int n_stages) {
+size_t smem_bytes(int D, int group, int n_stages, int ncw) {
   const int rows_cap = group < kMaxGroupRows ? group : kMaxGroupRows;
   size_t stage = (size_t)kGroupWarps * 2 * kPage * D * 2;
-  return n_stages * stage + (size_t)kConsumerWarps * rows_cap * (D + 2) * 4 + 2 * kMaxStages * 8 + 32;
+  return n_stages * stage + (size_t)ncw * rows_cap * (D + 2) * 4 + 2 * kMaxStages * 8 + 32;
 }
 
 }  // namespace
 
 cudaError_t prepare_decode_bf16() {
-  cudaError_t e = cudaFuncSetAttribute(decode_split_bf16_kernel<128>,
-                                       cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
-  if (e != cudaSuccess) return e;
-  return cudaFuncSetAttribute(decode_split_bf16_kernel<64>,
-                              cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+  cudaError_t e = cudaFuncSetAttribute(decode_split_bf16_kernel<128, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(decode_split_bf16_kernel<64, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(decode_split_bf16_kernel<128, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, 113 * 1024);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(decode_split_bf16_kernel<64, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, 113 * 1024);
+  return e;
 }
 
 cudaError_t launch_decode_split_bf16(const DecodeParams& p, int sm_count, cudaStream_t st) {
   const int D = p.geom.head_dim;
+  if (p.total_items <= 0) return cudaSuccess;
+  // Few, short items (more than one but at most two per SM, e.g. one 1024-key window per
+  // (sequence, KV head)): two small CTAs per SM keep all of them streaming at once, and the
+  // launch is bound by HBM instead of by the SM that drew two items.
+  int64_t max_keys = 0;
+  for (int i = 0; i < p.n_seqs; ++i) max_keys = p.chunk_len[i] > max_keys ? p.chunk_len[i] : max_keys;
+  const bool small = p.total_items > sm_count && p.total_items <= 2 * sm_count && max_keys <= 2048;
+  const int ncw = small ? 4 : 8;
+  const size_t budget = small ? 110 * 1024 : 220 * 1024;
   int n_stages = kMaxStages;
-  while (n_stages > 2 && smem_bytes(D, p.group, n_stages) > 220 * 1024) --n_stages;
-  const size_t smem = smem_bytes(D, p.group, n_stages);
-  const int grid = p.total_items < sm_count ? p.total_items : sm_count;
-  if (grid <= 0) return cudaSuccess;
+  while (n_stages > 2 && smem_bytes(D, p.group, n_stages, ncw) > budget) --n_stages;
+  const size_t smem = smem_bytes(D, p.group, n_stages, ncw);
+  const int slots = small ? 2 * sm_count : sm_count;
+  const int grid = p.total_items < slots ? p.total_items : slots;
   // launched with programmatic stream serialization: the kernel's set-up may overlap the
   // tail of the previous kernel in the stream; it waits (griddepcontrol.wait) before its
   // first global access
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(grid);
-  cfg.blockDim = dim3(kThreads);
+  cfg.blockDim = dim3((ncw + 1) * 32);
   cfg.dynamicSmemBytes = smem;
   cfg.stream = st;
   cudaLaunchAttribute attr[1];
@@ -434,8 +447,12 @@ cudaError_t launch_decode_split_bf16(const DecodeParams& p, int sm_count, cudaSt
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  if (D == 128) return cudaLaunchKernelEx(&cfg, decode_split_bf16_kernel<128>, p, n_stages);
-  return cudaLaunchKernelEx(&cfg, decode_split_bf16_kernel<64>, p, n_stages);
+  if (D == 128) {
+    if (small) return cudaLaunchKernelEx(&cfg, decode_split_bf16_kernel<128, 4>, p, n_stages);
+    return cudaLaunchKernelEx(&cfg, decode_split_bf16_kernel<128, 8>, p, n_stages);
+  }
+  if (small) return cudaLaunchKernelEx(&cfg, decode_split_bf16_kernel<64, 4>, p, n_stages);
+  return cudaLaunchKernelEx(&cfg, decode_split_bf16_kernel<64, 8>, p, n_stages);
 }
 
 }  // namespace mixattn
