@@ -5,25 +5,31 @@
 // one CTA owns a 128-query tile of one (sequence, head) and walks the 128-key tiles that
 // intersect its band; tiles wholly outside the band are never loaded.
 //
-//   warp 0     TMA producer: Q once, then K and V tiles (3 stages each) as 128B-swizzled
+//   warp 0     TMA producer: Q once, then K and V tiles (3 / 2 stages) as 128B-swizzled
 //              [128 x 64] boxes straight from the caller's tensors
 //   warp 1     one elected thread issues the tcgen05.mma (K16 steps, bf16 -> fp32 in TMEM) of
 //              S = Q K^T (M128 N128, both operands from shared memory) into one of two S
 //              buffers, two tiles ahead of the softmax
-//   warps 10-11  one elected thread per stream issues O_h += P_h V_h with P_h read from
+//   warps 2-3  one elected thread per stream issues O_h += P_h V_h with P_h read from
 //              tensor memory and V MN-major from its row-major tile
-//   warps 2-5  softmax stream "lo": key columns 0-63 of every tile; warps 6-9 stream "hi":
+//   warps 4-7  softmax stream "lo": key columns 0-63 of every tile; warps 8-11 stream "hi":
 //              columns 64-127.  The two streams are independent flash-attention passes
-//              over interleaved halves of the keys (own running max, own row sum, own O
-//              accumulator in TMEM), merged exactly at the end like split-KV partials.
+//              over interleaved halves of the keys (own exponent reference, own row sum,
+//              own O accumulator in TMEM), merged exactly at the end like split-KV partials.
 //              Thread r of a stream owns query row r (TMEM lane r): tcgen05.ld of its half
-//              of the S row, band masks on edge tiles only, base-2 online softmax with
-//              one MUFU ex2 per score, P written back as bf16 pairs over its own columns
-//              of the S buffer (tcgen05.st).  O rows are rescaled lazily (only when the
-//              running max grew by more than 2^8).
+//              of the S row, band masks on edge tiles only, base-2 softmax weights with one
+//              MUFU ex2 per score, P written back as bf16 pairs over its own columns of the
+//              S buffer (tcgen05.st).  The exponent reference of a row is the maximum of the
+//              first tile in which the row saw a key and is only moved (accumulators
+//              rescaled, weights recomputed) when a later score leads it by more than 2^64,
+//              so the exponentials of a tile never wait for the tile maximum.
+//   warps 12-15  epilogue: thread r merges the two accumulators of row r, normalises and
+//              writes the row while the softmax warps are already on the next work item.
 //
-// Two warps per scheduler work on independent data, the scores of the next two tiles are
-// always ready, and the P V products are issued in whichever order the streams finish.
+// Registers are moved between the roles with setmaxnreg (48 for the single-thread roles,
+// 168 for the softmax warps, 128 for the epilogue).  Two softmax warps per scheduler work on
+// independent data, the scores of the next two tiles are always ready, and the P V products
+// are issued in whichever order the streams finish.
 // TMEM: S0, S1, O_lo, O_hi = 4 x 128 columns.  All mbarrier waits are bounded; on
 // time-out a status word is raised, every role leaves its loop, and TMEM is released at
 // the common exit.
@@ -40,7 +46,7 @@ constexpr int kBM = 128;                       // queries per work item
 constexpr int kBN = 128;                       // keys per tile
 constexpr int kHalfBytes = 128 * 128;          // one [128 rows x 64 bf16] swizzled block
 constexpr int kTileBytes = 2 * kHalfBytes;     // a 128 x 128 bf16 operand tile
-constexpr int kThreads = 384;                  // TMA warp, S-MMA warp, 2 x 4 softmax warps, 2 PV-MMA warps
+constexpr int kThreads = 512;                  // 4 single-thread roles, 2 x 4 softmax warps, 4 epilogue warps
 constexpr int kKStages = 3, kVStages = 2;
 constexpr int kSmQ = 0;                        // two Q buffers (this item / next item)
 constexpr int kSmK = kSmQ + 2 * kTileBytes;
@@ -160,6 +166,27 @@ __device__ __forceinline__ float ex2_approx(float x) {   // 2^x, single MUFU op;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
+__device__ __forceinline__ float fmax3(float a, float b, float c) {   // three-input maximum, one instruction
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
+// Waits for the tensor-memory loads in flight; the registers they fill are named as operands
+// so that no use of them can be scheduled before the wait.
+__device__ __forceinline__ void tmem_wait_ld_pin(uint32_t (&a)[32], uint32_t (&b)[32]) {
+  asm volatile("tcgen05.wait::ld.sync.aligned;"
+      : "+r"(a[0]), "+r"(a[1]), "+r"(a[2]), "+r"(a[3]), "+r"(a[4]), "+r"(a[5]), "+r"(a[6]), "+r"(a[7]),
+        "+r"(a[8]), "+r"(a[9]), "+r"(a[10]), "+r"(a[11]), "+r"(a[12]), "+r"(a[13]), "+r"(a[14]), "+r"(a[15]),
+        "+r"(a[16]), "+r"(a[17]), "+r"(a[18]), "+r"(a[19]), "+r"(a[20]), "+r"(a[21]), "+r"(a[22]), "+r"(a[23]),
+        "+r"(a[24]), "+r"(a[25]), "+r"(a[26]), "+r"(a[27]), "+r"(a[28]), "+r"(a[29]), "+r"(a[30]), "+r"(a[31])
+      :: "memory");
+  asm volatile(""
+      : "+r"(b[0]), "+r"(b[1]), "+r"(b[2]), "+r"(b[3]), "+r"(b[4]), "+r"(b[5]), "+r"(b[6]), "+r"(b[7]),
+        "+r"(b[8]), "+r"(b[9]), "+r"(b[10]), "+r"(b[11]), "+r"(b[12]), "+r"(b[13]), "+r"(b[14]), "+r"(b[15]),
+        "+r"(b[16]), "+r"(b[17]), "+r"(b[18]), "+r"(b[19]), "+r"(b[20]), "+r"(b[21]), "+r"(b[22]), "+r"(b[23]),
+        "+r"(b[24]), "+r"(b[25]), "+r"(b[26]), "+r"(b[27]), "+r"(b[28]), "+r"(b[29]), "+r"(b[30]), "+r"(b[31])
+      :: "memory");
+}
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
@@ -231,7 +258,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
       mbar_init(BAR(B_KE + s), 1);
     }
     mbar_init(BAR(B_XC), 8);
-    mbar_init(BAR(B_OR), 8);
+    mbar_init(BAR(B_OR), 4);
     abort_flag[0] = 0;
     abort_flag[1] = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -248,139 +275,203 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
   // Every role walks the same item list and keeps the same counters: G = key tiles
   // processed so far by this CTA (all items), it = items processed so far.  Per-tile
   // barriers are indexed by G, per-item barriers by it, so phases carry over.
-  if (warp == 0) {
-    // ------------------------------ TMA producer ------------------------------
-    if (lane == 0) {
-      asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_q) : "memory");
-      asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_k) : "memory");
-      asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_v) : "memory");
-      bool ok = true;
-      int G = 0, it = 0, q_issued = 0, k_issued = 0, v_issued = 0;
-      for (int id = blockIdx.x; id < n_ids && ok; id += gridDim.x) {
-        const WorkItem w = get_item(p, id);
-        if (!w.valid) continue;
-        const int qb = it & 1;
-        if (it >= 2) ok = mbar_wait(BAR(B_QE + qb), ((it >> 1) - 1) & 1, abort_flag);
-        if (!ok) break;
-        mbar_expect_tx(BAR(B_QF + qb), kTileBytes);
-        tma_load_3d(base + kSmQ + qb * kTileBytes, &tm_q, 0, w.h, w.row_base + w.i0, BAR(B_QF + qb));
-        tma_load_3d(base + kSmQ + qb * kTileBytes + kHalfBytes, &tm_q, 64, w.h, w.row_base + w.i0, BAR(B_QF + qb));
-        ++q_issued;
-        for (int j = 0; j < w.n_tiles && ok; ++j) {
-          const int Gj = G + j;
-          const int row = w.row_base + (w.jt_lo + j) * kBN;
-          const int ks = Gj % kKStages, ku = Gj / kKStages;
-          if (ku > 0) ok = mbar_wait(BAR(B_KE + ks), (ku - 1) & 1, abort_flag);
+  if (warp < 4) {
+    // single-thread roles: give registers back to the pool
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 48;");
+    if (warp == 0) {
+      // ------------------------------ TMA producer ------------------------------
+      if (lane == 0) {
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_q) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_k) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_v) : "memory");
+        bool ok = true;
+        int G = 0, it = 0, q_issued = 0, k_issued = 0, v_issued = 0;
+        for (int id = blockIdx.x; id < n_ids && ok; id += gridDim.x) {
+          const WorkItem w = get_item(p, id);
+          if (!w.valid) continue;
+          const int qb = it & 1;
+          if (it >= 2) ok = mbar_wait(BAR(B_QE + qb), ((it >> 1) - 1) & 1, abort_flag);
           if (!ok) break;
-          mbar_expect_tx(BAR(B_KF + ks), kTileBytes);
-          tma_load_3d(base + kSmK + ks * kTileBytes, &tm_k, 0, w.g, row, BAR(B_KF + ks));
-          tma_load_3d(base + kSmK + ks * kTileBytes + kHalfBytes, &tm_k, 64, w.g, row, BAR(B_KF + ks));
-          ++k_issued;
-          const int vs = Gj % kVStages, vu = Gj / kVStages;
-          if (vu > 0) ok = mbar_wait(BAR(B_VE + vs), (vu - 1) & 1, abort_flag);
-          if (!ok) break;
-          mbar_expect_tx(BAR(B_VF + vs), kTileBytes);
-          tma_load_3d(base + kSmV + vs * kTileBytes, &tm_v, 0, w.g, row, BAR(B_VF + vs));
-          tma_load_3d(base + kSmV + vs * kTileBytes + kHalfBytes, &tm_v, 64, w.g, row, BAR(B_VF + vs));
-          ++v_issued;
+          mbar_expect_tx(BAR(B_QF + qb), kTileBytes);
+          tma_load_3d(base + kSmQ + qb * kTileBytes, &tm_q, 0, w.h, w.row_base + w.i0, BAR(B_QF + qb));
+          tma_load_3d(base + kSmQ + qb * kTileBytes + kHalfBytes, &tm_q, 64, w.h, w.row_base + w.i0, BAR(B_QF + qb));
+          ++q_issued;
+          for (int j = 0; j < w.n_tiles && ok; ++j) {
+            const int Gj = G + j;
+            const int row = w.row_base + (w.jt_lo + j) * kBN;
+            const int ks = Gj % kKStages, ku = Gj / kKStages;
+            if (ku > 0) ok = mbar_wait(BAR(B_KE + ks), (ku - 1) & 1, abort_flag);
+            if (!ok) break;
+            mbar_expect_tx(BAR(B_KF + ks), kTileBytes);
+            tma_load_3d(base + kSmK + ks * kTileBytes, &tm_k, 0, w.g, row, BAR(B_KF + ks));
+            tma_load_3d(base + kSmK + ks * kTileBytes + kHalfBytes, &tm_k, 64, w.g, row, BAR(B_KF + ks));
+            ++k_issued;
+            const int vs = Gj % kVStages, vu = Gj / kVStages;
+            if (vu > 0) ok = mbar_wait(BAR(B_VE + vs), (vu - 1) & 1, abort_flag);
+            if (!ok) break;
+            mbar_expect_tx(BAR(B_VF + vs), kTileBytes);
+            tma_load_3d(base + kSmV + vs * kTileBytes, &tm_v, 0, w.g, row, BAR(B_VF + vs));
+            tma_load_3d(base + kSmV + vs * kTileBytes + kHalfBytes, &tm_v, 64, w.g, row, BAR(B_VF + vs));
+            ++v_issued;
+          }
+          G += w.n_tiles;
+          ++it;
         }
-        G += w.n_tiles;
-        ++it;
+        if (!ok) {  // leave only after the copies already issued have landed (bounded)
+          atomicExch(p.status, kDevWaitTimeout);
+          for (int back = 1; back <= 2 && q_issued - back >= 0; ++back)
+            mbar_wait(BAR(B_QF + ((q_issued - back) & 1)), ((q_issued - back) >> 1) & 1, abort_flag + 1);
+          for (int back = 1; back <= kKStages && k_issued - back >= 0; ++back)
+            mbar_wait(BAR(B_KF + (k_issued - back) % kKStages), ((k_issued - back) / kKStages) & 1, abort_flag + 1);
+          for (int back = 1; back <= kVStages && v_issued - back >= 0; ++back)
+            mbar_wait(BAR(B_VF + (v_issued - back) % kVStages), ((v_issued - back) / kVStages) & 1, abort_flag + 1);
+        }
       }
-      if (!ok) {  // leave only after the copies already issued have landed (bounded)
-        atomicExch(p.status, kDevWaitTimeout);
-        for (int back = 1; back <= 2 && q_issued - back >= 0; ++back)
-          mbar_wait(BAR(B_QF + ((q_issued - back) & 1)), ((q_issued - back) >> 1) & 1, abort_flag + 1);
-        for (int back = 1; back <= kKStages && k_issued - back >= 0; ++back)
-          mbar_wait(BAR(B_KF + (k_issued - back) % kKStages), ((k_issued - back) / kKStages) & 1, abort_flag + 1);
-        for (int back = 1; back <= kVStages && v_issued - back >= 0; ++back)
-          mbar_wait(BAR(B_VF + (v_issued - back) % kVStages), ((v_issued - back) / kVStages) & 1, abort_flag + 1);
+    } else if (warp == 1) {
+      // ------------------------------ MMA issuer, scores ------------------------------
+      // Three threads issue MMAs (this one S = Q K^T, warps 2 and 3 the P V products of the
+      // two streams): issuing is a serial, latency-bound instruction stream, and one thread
+      // alone was the bottleneck.
+      if (lane == 0) {
+        constexpr uint32_t kIdescS = idesc_bf16(0);
+        bool ok = true;
+        int G = 0, it = 0;
+        for (int id = blockIdx.x; id < n_ids && ok; id += gridDim.x) {
+          const WorkItem w = get_item(p, id);
+          if (!w.valid) continue;
+          const int qb = it & 1;
+          ok = mbar_wait(BAR(B_QF + qb), (it >> 1) & 1, abort_flag);
+          uint64_t qdesc[8];
+  #pragma unroll
+          for (int ks = 0; ks < 8; ++ks)   // head_dim 128 = 8 steps of 16 channels
+            qdesc[ks] = smem_desc(base + kSmQ + qb * kTileBytes + (ks >> 2) * kHalfBytes + (ks & 3) * 32, 16, 1024);
+          for (int j = 0; j < w.n_tiles && ok; ++j) {
+            // S(G) = Q K^T into S buffer G & 1, which held S(G-2) / P(G-2): wait until both
+            // P V(G-2) have consumed it (they are issued by another thread)
+            const int Gj = G + j, sb = Gj & 1, ks_ = Gj % kKStages;
+            if (Gj >= 2) ok = mbar_wait(BAR(B_SR + sb), ((Gj >> 1) - 1) & 1, abort_flag);
+            if (ok) ok = mbar_wait(BAR(B_KF + ks_), (Gj / kKStages) & 1, abort_flag);
+            if (!ok) break;
+            tc_fence_after();
+            const uint64_t kdesc = smem_desc(base + kSmK + ks_ * kTileBytes, 16, 1024);
+  #pragma unroll
+            for (int ks = 0; ks < 8; ++ks)
+              umma_bf16(tmem + kColS + sb * 128, qdesc[ks],
+                        kdesc + (uint64_t)((ks >> 2) * (kHalfBytes >> 4) + (ks & 3) * 2), kIdescS, ks > 0);
+            umma_commit(BAR(B_SF + sb));    // scores ready
+            umma_commit(BAR(B_KE + ks_));   // K stage free
+          }
+          if (ok) umma_commit(BAR(B_QE + qb));   // Q buffer free once this item's S products are done
+          G += w.n_tiles;
+          ++it;
+        }
+        if (!ok) atomicExch(p.status, kDevWaitTimeout);
+      }
+    } else {
+      // ------------------------------ MMA issuers, P V (one per stream) ------------------------------
+      if (lane == 0) {
+        constexpr uint32_t kIdescPV = idesc_bf16(1);
+        const int hs = warp - 2;
+        bool ok = true;
+        int G = 0, it = 0;
+        for (int id = blockIdx.x; id < n_ids && ok; id += gridDim.x) {
+          const WorkItem w = get_item(p, id);
+          if (!w.valid) continue;
+          // the first P V of an item overwrites the O accumulator: the streams must have
+          // read the previous item's result
+          if (it >= 1) ok = mbar_wait(BAR(B_OR), (it - 1) & 1, abort_flag);
+          for (int j = 0; j < w.n_tiles && ok; ++j) {
+            const int Gj = G + j, sb = Gj & 1, vs = Gj % kVStages;
+            ok = mbar_wait(BAR(B_VF + vs), (Gj / kVStages) & 1, abort_flag);
+            if (ok) ok = mbar_wait(BAR(B_PF + hs), Gj & 1, abort_flag);
+            if (!ok) break;
+            tc_fence_after();
+            // O_h += P_h V[64 h .. 64 h + 63]: A = P from tensor memory (two bf16 per column),
+            // B = V MN-major (channels contiguous, keys strided by 128 B)
+            const uint64_t vdesc = smem_desc(base + kSmV + vs * kTileBytes + hs * 4 * 2048, kHalfBytes, 1024);
+  #pragma unroll
+            for (int ks = 0; ks < 4; ++ks)   // 64 keys = 4 steps of 16
+              umma_bf16_ts(tmem + kColO + hs * 128, tmem + kColS + sb * 128 + hs * 64 + ks * 8,
+                           vdesc + (uint64_t)(ks * (2048 >> 4)), kIdescPV, (j > 0 || ks > 0) ? 1u : 0u);
+            umma_commit(BAR(B_OF + hs));   // this stream's accumulator is up to date
+            umma_commit(BAR(B_VE + vs));   // V stage free once both streams' P V are done (count 2)
+            umma_commit(BAR(B_SR + sb));   // and so is the S buffer
+          }
+          G += w.n_tiles;
+          ++it;
+        }
+        if (!ok) atomicExch(p.status, kDevWaitTimeout);
       }
     }
-  } else if (warp == 1) {
-    // ------------------------------ MMA issuer, scores ------------------------------
-    // Three threads issue MMAs (this one S = Q K^T, warps 10 and 11 the P V products of the
-    // two streams): issuing is a serial, latency-bound instruction stream, and one thread
-    // alone was the bottleneck.
-    if (lane == 0) {
-      constexpr uint32_t kIdescS = idesc_bf16(0);
-      bool ok = true;
-      int G = 0, it = 0;
-      for (int id = blockIdx.x; id < n_ids && ok; id += gridDim.x) {
-        const WorkItem w = get_item(p, id);
-        if (!w.valid) continue;
-        const int qb = it & 1;
-        ok = mbar_wait(BAR(B_QF + qb), (it >> 1) & 1, abort_flag);
-        uint64_t qdesc[8];
+  } else if (warp >= 12) {
+    // ------------------------------ epilogue warps ------------------------------
+    // Thread r merges the two streams' accumulators of query row r like split-KV partials
+    // and writes the row, while the softmax warps already work on the next item.
+    const int qd = warp & 3;
+    const int r = qd * 32 + lane;
+    const uint32_t lane_base = tmem + ((uint32_t)(qd * 32) << 16);
+    const float2* xchg = reinterpret_cast<const float2*>(gbase + kSmXchg);
+    bool ok = true;
+    int G = 0, it = 0;
+    for (int id = blockIdx.x; id < n_ids && ok; id += gridDim.x) {
+      const WorkItem w = get_item(p, id);
+      if (!w.valid) continue;
+      G += w.n_tiles;
+      ok = __all_sync(0xffffffffu, mbar_wait(BAR(B_XC), it & 1, abort_flag));
+      if (!ok) break;
+      const float2 lo = xchg[r], hi = xchg[128 + r];
+      // both streams' last P V of the item have landed
+      ok = __all_sync(0xffffffffu, mbar_wait(BAR(B_OF + 0), (G - 1) & 1, abort_flag) &&
+                                   mbar_wait(BAR(B_OF + 1), (G - 1) & 1, abort_flag));
+      if (!ok) break;
+      tc_fence_after();
+      const float m_all = fmaxf(lo.x, hi.x);              // finite for every valid row (key i is visible)
+      const float e_lo = ex2_approx(lo.x - m_all), e_hi = ex2_approx(hi.x - m_all);   // 2^-inf = 0
+      const float inv = 1.f / (lo.y * e_lo + hi.y * e_hi);
+      const float w_lo = e_lo * inv, w_hi = e_hi * inv;
+      const int i = w.i0 + r;
+      __nv_bfloat16* orow = p.out + ((int64_t)(w.row_base + i) * p.n_q_heads + w.h) * 128;
 #pragma unroll
-        for (int ks = 0; ks < 8; ++ks)   // head_dim 128 = 8 steps of 16 channels
-          qdesc[ks] = smem_desc(base + kSmQ + qb * kTileBytes + (ks >> 2) * kHalfBytes + (ks & 3) * 32, 16, 1024);
-        for (int j = 0; j < w.n_tiles && ok; ++j) {
-          // S(G) = Q K^T into S buffer G & 1, which held S(G-2) / P(G-2): wait until both
-          // P V(G-2) have consumed it (they are issued by another thread)
-          const int Gj = G + j, sb = Gj & 1, ks_ = Gj % kKStages;
-          if (Gj >= 2) ok = mbar_wait(BAR(B_SR + sb), ((Gj >> 1) - 1) & 1, abort_flag);
-          if (ok) ok = mbar_wait(BAR(B_KF + ks_), (Gj / kKStages) & 1, abort_flag);
-          if (!ok) break;
-          tc_fence_after();
-          const uint64_t kdesc = smem_desc(base + kSmK + ks_ * kTileBytes, 16, 1024);
-#pragma unroll
-          for (int ks = 0; ks < 8; ++ks)
-            umma_bf16(tmem + kColS + sb * 128, qdesc[ks],
-                      kdesc + (uint64_t)((ks >> 2) * (kHalfBytes >> 4) + (ks & 3) * 2), kIdescS, ks > 0);
-          umma_commit(BAR(B_SF + sb));    // scores ready
-          umma_commit(BAR(B_KE + ks_));   // K stage free
+      for (int c = 0; c < 4; ++c) {
+        uint32_t olo[32], ohi[32];
+        tmem_ld32(lane_base + kColO + c * 32, olo);
+        tmem_ld32(lane_base + kColO + 128 + c * 32, ohi);
+        tmem_wait_ld();
+        if (c == 3) {   // the accumulators may be overwritten by the next item
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(BAR(B_OR));
         }
-        if (ok) umma_commit(BAR(B_QE + qb));   // Q buffer free once this item's S products are done
-        G += w.n_tiles;
-        ++it;
-      }
-      if (!ok) atomicExch(p.status, kDevWaitTimeout);
-    }
-  } else if (warp >= 10) {
-    // ------------------------------ MMA issuers, P V (one per stream) ------------------------------
-    if (lane == 0) {
-      constexpr uint32_t kIdescPV = idesc_bf16(1);
-      const int hs = warp - 10;
-      bool ok = true;
-      int G = 0, it = 0;
-      for (int id = blockIdx.x; id < n_ids && ok; id += gridDim.x) {
-        const WorkItem w = get_item(p, id);
-        if (!w.valid) continue;
-        // the first P V of an item overwrites the O accumulator: the streams must have
-        // read the previous item's result
-        if (it >= 1) ok = mbar_wait(BAR(B_OR), (it - 1) & 1, abort_flag);
-        for (int j = 0; j < w.n_tiles && ok; ++j) {
-          const int Gj = G + j, sb = Gj & 1, vs = Gj % kVStages;
-          ok = mbar_wait(BAR(B_VF + vs), (Gj / kVStages) & 1, abort_flag);
-          if (ok) ok = mbar_wait(BAR(B_PF + hs), Gj & 1, abort_flag);
-          if (!ok) break;
-          tc_fence_after();
-          // O_h += P_h V[64 h .. 64 h + 63]: A = P from tensor memory (two bf16 per column),
-          // B = V MN-major (channels contiguous, keys strided by 128 B)
-          const uint64_t vdesc = smem_desc(base + kSmV + vs * kTileBytes + hs * 4 * 2048, kHalfBytes, 1024);
+        if (i < w.S) {
 #pragma unroll
-          for (int ks = 0; ks < 4; ++ks)   // 64 keys = 4 steps of 16
-            umma_bf16_ts(tmem + kColO + hs * 128, tmem + kColS + sb * 128 + hs * 64 + ks * 8,
-                         vdesc + (uint64_t)(ks * (2048 >> 4)), kIdescPV, (j > 0 || ks > 0) ? 1u : 0u);
-          umma_commit(BAR(B_OF + hs));   // this stream's accumulator is up to date
-          umma_commit(BAR(B_VE + vs));   // V stage free once both streams' P V are done (count 2)
-          umma_commit(BAR(B_SR + sb));   // and so is the S buffer
+          for (int q8 = 0; q8 < 4; ++q8) {
+            uint32_t o4[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              const int d = q8 * 8 + e * 2;
+              o4[e] = pack_bf16(__uint_as_float(olo[d]) * w_lo + __uint_as_float(ohi[d]) * w_hi,
+                                __uint_as_float(olo[d + 1]) * w_lo + __uint_as_float(ohi[d + 1]) * w_hi);
+            }
+            *reinterpret_cast<uint4*>(orow + c * 32 + q8 * 8) = make_uint4(o4[0], o4[1], o4[2], o4[3]);
+          }
         }
-        G += w.n_tiles;
-        ++it;
       }
-      if (!ok) atomicExch(p.status, kDevWaitTimeout);
+      ++it;
     }
+    if (!ok && lane == 0) atomicExch(p.status, kDevWaitTimeout);
   } else {
     // ------------------------------ softmax warps ------------------------------
-    const int hs = (warp - 2) >> 2;       // stream: key columns [64 hs, 64 hs + 64) of every tile
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 168;");
+    const int hs = (warp - 4) >> 2;       // stream: key columns [64 hs, 64 hs + 64) of every tile
     const int qd = warp & 3;              // TMEM lane quarter this warp may access
     const int r = qd * 32 + lane;         // query row within the tile
     const uint32_t lane_base = tmem + ((uint32_t)(qd * 32) << 16);
     const uint32_t o_addr = lane_base + kColO + hs * 128;
     float2* xchg = reinterpret_cast<float2*>(gbase + kSmXchg);
-    constexpr float kRescaleGap = 8.f;    // the exponent reference may lag the running max by 2^8
+    // The exponent reference of a row is the maximum of the first tile in which the row saw a
+    // key; it is only moved (and the accumulators rescaled) when a later score leads it by
+    // more than 2^kMaxLead, so the exponentials of a tile do not wait for the tile maximum.
+    constexpr float kMaxLead = 64.f;
     bool ok = true;
     int G = 0, it = 0;
     for (int id = blockIdx.x; id < n_ids && ok; id += gridDim.x) {
@@ -388,41 +479,66 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
       if (!w.valid) continue;
       const int i = w.i0 + r;             // query position
       float m_ref = -INFINITY, l = 0.f;
+      uint32_t sv[64];
+      {
+        if (!__all_sync(0xffffffffu, mbar_wait(BAR(B_SF + (G & 1)), (G >> 1) & 1, abort_flag))) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t s_addr = lane_base + kColS + (G & 1) * 128 + hs * 64;
+        tmem_ld32(s_addr, *reinterpret_cast<uint32_t(*)[32]>(&sv[0]));
+        tmem_ld32(s_addr + 32, *reinterpret_cast<uint32_t(*)[32]>(&sv[32]));
+        tmem_wait_ld_pin(*reinterpret_cast<uint32_t(*)[32]>(&sv[0]), *reinterpret_cast<uint32_t(*)[32]>(&sv[32]));
+      }
       for (int j = 0; j < w.n_tiles; ++j) {
         const int Gj = G + j, sb = Gj & 1;
         const int j0 = (w.jt_lo + j) * kBN + hs * 64;   // first key of this stream's columns
         const uint32_t s_addr = lane_base + kColS + sb * 128 + hs * 64;
-        if (!__all_sync(0xffffffffu, mbar_wait(BAR(B_SF + sb), (Gj >> 1) & 1, abort_flag))) { ok = false; break; }
-        tc_fence_after();
-        uint32_t sv[64];
-        tmem_ld32(s_addr, *reinterpret_cast<uint32_t(*)[32]>(&sv[0]));
-        tmem_ld32(s_addr + 32, *reinterpret_cast<uint32_t(*)[32]>(&sv[32]));
-        tmem_wait_ld();
         // band edges: causal (keys after the query) and window (keys older than i - window)
         const bool edge = (j0 + 63 > w.i0) || (p.window > 0 && j0 <= w.i0 + kBM - 1 - p.window);
-        if (edge) {
+        auto mask_edges = [&]() {
           const int k_max = i - j0;                                      // columns <= k_max are causal-visible
           const int k_min = p.window > 0 ? i - p.window + 1 - j0 : 0;    // columns >= k_min are inside the window
 #pragma unroll
           for (int e = 0; e < 64; ++e)
             if (e > k_max || e < k_min) sv[e] = 0xff800000u;             // -inf
+        };
+        if (edge) mask_edges();
+        // a row that has not seen a key yet takes its reference from this tile
+        const bool fresh = m_ref == -INFINITY;
+        if (__any_sync(0xffffffffu, fresh)) {
+          float mx0 = -INFINITY, mx1 = -INFINITY;
+#pragma unroll
+          for (int e = 0; e < 64; e += 4) {
+            mx0 = fmax3(mx0, __uint_as_float(sv[e]), __uint_as_float(sv[e + 1]));
+            mx1 = fmax3(mx1, __uint_as_float(sv[e + 2]), __uint_as_float(sv[e + 3]));
+          }
+          if (fresh) m_ref = fmaxf(mx0, mx1) * p.scale_log2e;
         }
-        float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
+        float neg_m = m_ref == -INFINITY ? 0.f : -m_ref;   // no visible key yet: weights 0, no NaN
+        float sum0 = 0.f, sum1 = 0.f, mxa = -INFINITY, mxb = -INFINITY;
+        uint32_t pk[32];
 #pragma unroll
         for (int e = 0; e < 64; e += 4) {
-          mx0 = fmaxf(mx0, __uint_as_float(sv[e]));
-          mx1 = fmaxf(mx1, __uint_as_float(sv[e + 1]));
-          mx2 = fmaxf(mx2, __uint_as_float(sv[e + 2]));
-          mx3 = fmaxf(mx3, __uint_as_float(sv[e + 3]));
+          const float p0 = ex2_approx(fmaf(__uint_as_float(sv[e]), p.scale_log2e, neg_m));
+          const float p1 = ex2_approx(fmaf(__uint_as_float(sv[e + 1]), p.scale_log2e, neg_m));
+          const float p2 = ex2_approx(fmaf(__uint_as_float(sv[e + 2]), p.scale_log2e, neg_m));
+          const float p3 = ex2_approx(fmaf(__uint_as_float(sv[e + 3]), p.scale_log2e, neg_m));
+          sum0 += p0 + p2;
+          sum1 += p1 + p3;
+          pk[e >> 1] = pack_bf16(p0, p1);
+          pk[(e >> 1) + 1] = pack_bf16(p2, p3);
+          mxa = fmax3(mxa, __uint_as_float(sv[e]), __uint_as_float(sv[e + 1]));
+          mxb = fmax3(mxb, __uint_as_float(sv[e + 2]), __uint_as_float(sv[e + 3]));
         }
-        const float mt = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * p.scale_log2e;
-        const bool grow = mt > m_ref + kRescaleGap;    // also true for the first visible key (m_ref = -inf)
-        if (__any_sync(0xffffffffu, grow)) {
-          const float alpha = grow ? ex2_approx(m_ref - mt) : 1.f;   // m_ref = -inf gives 0
+        const float mt = fmaxf(mxa, mxb) * p.scale_log2e;
+        const bool far = mt > m_ref + kMaxLead;
+        if (__any_sync(0xffffffffu, far)) {
+          // rare: move the reference of the leading rows up to the tile maximum, rescale what
+          // they have accumulated, and recompute this tile's weights
+          const float alpha = far ? ex2_approx(m_ref - mt) : 1.f;
           if (j > 0) {   // the O row holds earlier tiles: rescale it once this stream's previous P V has landed
             if (!__all_sync(0xffffffffu, mbar_wait(BAR(B_OF + hs), (Gj - 1) & 1, abort_flag))) { ok = false; break; }
             tc_fence_after();
-#pragma unroll
+#pragma unroll 1
             for (int c = 0; c < 4; ++c) {
               uint32_t ov[32];
               tmem_ld32(o_addr + c * 32, ov);
@@ -433,18 +549,23 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
             }
           }
           l *= alpha;
-          if (grow) m_ref = mt;
-        }
-        const float neg_m = m_ref == -INFINITY ? 0.f : -m_ref;   // no visible key yet: weights 0, no NaN
-        float sum0 = 0.f, sum1 = 0.f;
-        uint32_t pk[32];
+          if (far) m_ref = mt;
+          neg_m = m_ref == -INFINITY ? 0.f : -m_ref;
+          sum0 = 0.f;
+          sum1 = 0.f;
+          // the scores are still in the S buffer (P has not been written yet)
+          tmem_ld32(s_addr, *reinterpret_cast<uint32_t(*)[32]>(&sv[0]));
+          tmem_ld32(s_addr + 32, *reinterpret_cast<uint32_t(*)[32]>(&sv[32]));
+          tmem_wait_ld_pin(*reinterpret_cast<uint32_t(*)[32]>(&sv[0]), *reinterpret_cast<uint32_t(*)[32]>(&sv[32]));
+          if (edge) mask_edges();
 #pragma unroll
-        for (int e = 0; e < 64; e += 2) {
-          const float p0 = ex2_approx(fmaf(__uint_as_float(sv[e]), p.scale_log2e, neg_m));
-          const float p1 = ex2_approx(fmaf(__uint_as_float(sv[e + 1]), p.scale_log2e, neg_m));
-          sum0 += p0;
-          sum1 += p1;
-          pk[e >> 1] = pack_bf16(p0, p1);
+          for (int e = 0; e < 64; e += 2) {
+            const float p0 = ex2_approx(fmaf(__uint_as_float(sv[e]), p.scale_log2e, neg_m));
+            const float p1 = ex2_approx(fmaf(__uint_as_float(sv[e + 1]), p.scale_log2e, neg_m));
+            sum0 += p0;
+            sum1 += p1;
+            pk[e >> 1] = pack_bf16(p0, p1);
+          }
         }
         l += sum0 + sum1;
         // P (bf16 pairs) over the first 32 of this stream's 64 score columns
@@ -456,49 +577,26 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         if (Gj > 0 && !__all_sync(0xffffffffu, mbar_wait(BAR(B_OF + hs), (Gj - 1) & 1, abort_flag))) { ok = false; break; }
         __syncwarp();
         if (lane == 0) mbar_arrive(BAR(B_PF + hs));
-      }
-      G += w.n_tiles;
-      if (ok) ok = __all_sync(0xffffffffu, mbar_wait(BAR(B_OF + hs), (G - 1) & 1, abort_flag));
-      if (ok) {
-        // merge the two streams like split-KV partials: exchange (reference, sum) per row
-        tc_fence_after();
-        xchg[hs * 128 + r] = make_float2(m_ref, l);
-        __syncwarp();
-        if (lane == 0) mbar_arrive(BAR(B_XC));
-        ok = __all_sync(0xffffffffu, mbar_wait(BAR(B_XC), it & 1, abort_flag));
-      }
-      if (ok) {
-        tc_fence_after();
-        const float2 other = xchg[(hs ^ 1) * 128 + r];
-        const float m_all = fmaxf(m_ref, other.x);          // finite for every valid row (key i is visible)
-        const float w_me = ex2_approx(m_ref - m_all), w_ot = ex2_approx(other.x - m_all);   // 2^-inf = 0
-        const float inv = 1.f / (l * w_me + other.y * w_ot);
-        const float w_lo = (hs == 0 ? w_me : w_ot) * inv, w_hi = (hs == 0 ? w_ot : w_me) * inv;
-        // this thread writes channels [64 hs, 64 hs + 64) of its row from both accumulators
-        uint32_t olo[64], ohi[64];
-        tmem_ld32(lane_base + kColO + hs * 64, *reinterpret_cast<uint32_t(*)[32]>(&olo[0]));
-        tmem_ld32(lane_base + kColO + hs * 64 + 32, *reinterpret_cast<uint32_t(*)[32]>(&olo[32]));
-        tmem_ld32(lane_base + kColO + 128 + hs * 64, *reinterpret_cast<uint32_t(*)[32]>(&ohi[0]));
-        tmem_ld32(lane_base + kColO + 128 + hs * 64 + 32, *reinterpret_cast<uint32_t(*)[32]>(&ohi[32]));
-        tmem_wait_ld();
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(BAR(B_OR));   // the accumulators may be overwritten by the next item
-        if (i < w.S) {
-          __nv_bfloat16* orow = p.out + ((int64_t)(w.row_base + i) * p.n_q_heads + w.h) * 128 + hs * 64;
-#pragma unroll
-          for (int q8 = 0; q8 < 8; ++q8) {
-            uint32_t o4[4];
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-              const int d = q8 * 8 + e * 2;
-              o4[e] = pack_bf16(__uint_as_float(olo[d]) * w_lo + __uint_as_float(ohi[d]) * w_hi,
-                                __uint_as_float(olo[d + 1]) * w_lo + __uint_as_float(ohi[d + 1]) * w_hi);
-            }
-            *reinterpret_cast<uint4*>(orow + q8 * 8) = make_uint4(o4[0], o4[1], o4[2], o4[3]);
-          }
+        // the next tile's scores
+        const bool more = j + 1 < w.n_tiles;
+        if (more) {
+          if (!__all_sync(0xffffffffu, mbar_wait(BAR(B_SF + (sb ^ 1)), ((Gj + 1) >> 1) & 1, abort_flag))) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t n_addr = lane_base + kColS + (sb ^ 1) * 128 + hs * 64;
+          tmem_ld32(n_addr, *reinterpret_cast<uint32_t(*)[32]>(&sv[0]));
+          tmem_ld32(n_addr + 32, *reinterpret_cast<uint32_t(*)[32]>(&sv[32]));
         }
+        if (more) tmem_wait_ld_pin(*reinterpret_cast<uint32_t(*)[32]>(&sv[0]), *reinterpret_cast<uint32_t(*)[32]>(&sv[32]));
       }
+      if (!ok) break;
+      G += w.n_tiles;
+      // hand (reference, sum) of the row to the epilogue warps; the slot is free once they
+      // have read the previous item's pair
+      if (it >= 1) ok = __all_sync(0xffffffffu, mbar_wait(BAR(B_OR), (it - 1) & 1, abort_flag));
+      if (!ok) break;
+      xchg[hs * 128 + r] = make_float2(m_ref, l);
+      __syncwarp();
+      if (lane == 0) mbar_arrive(BAR(B_XC));
       ++it;
     }
     if (!ok && lane == 0) atomicExch(p.status, kDevWaitTimeout);

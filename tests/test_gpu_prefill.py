@@ -138,3 +138,39 @@ def test_prefill_head_shapes_and_ragged_lengths(hq, hkv, d, dtype):
             check_stored_bits(sess.ctx, ph, wl, 0, b, sorted({0, S // 2, S - 1}))
     finally:
         sess.close()
+
+
+@pytest.mark.parametrize("gain", [40.0, 300.0])
+def test_prefill_scores_that_outrun_the_exponent_reference(gain):
+    # queries scaled so that later tiles hold scores far above the first tile's maximum: the
+    # kernel has to move its exponent reference, rescale what it accumulated and recompute
+    # the tile; the softmax is close to one-hot and must still match
+    mx, runner = load_lib()
+    seq_lens = [700, 300]
+    wl = cf.prefill_chunk().scaled(layout=cf.layout_tiny(256), batch=len(seq_lens), seq_len=max(seq_lens))
+    sess = runner.Session(wl, [0] * wl.batch, headroom_tokens=2)
+    try:
+        ids = list(range(wl.batch))
+        for l in (3, 2):     # readers of the standard and of the sliding cache
+            kind, W, owner = wl.layout[l]
+            q, k, v = _prefill_direct(mx, wl, seq_lens, l)
+            q = (q.float() * gain).to(q.dtype)
+            qd, kd, vd = q.cuda(), k.cuda(), v.cuda()
+            out = torch.full_like(qd, float("nan"))
+            sess.ctx.prefill(l, ids, seq_lens, qd, kd, vd, out)
+            torch.cuda.synchronize()
+            got = out.float().cpu().double().numpy()
+            row = 0
+            for b, S in enumerate(seq_lens):
+                ref = mo.prefill_attention(q[row:row + S], k[row:row + S], v[row:row + S], kind, W)
+                # outputs here are single V rows or mixes of two or three of them, of magnitude up
+                # to ~4, not long averages: bf16 rounding of the output (2^-9 relative) and of the
+                # few weights that matter (2^-9 each, times |v| <= 5) bound the error
+                err = np.abs(got[row:row + S] - ref)
+                bound = 1e-2 + 2.0 ** -8 * np.abs(ref) + 2.0 ** -8 * 5.0
+                assert (err <= bound).all(), f"gain {gain} layer {l} seq {b}: worst excess {(err - bound).max():.3e}"
+                assert err.mean() <= 2e-3
+                row += S
+        assert sess.ctx.get_device_status() == 0
+    finally:
+        sess.close()
