@@ -64,9 +64,10 @@ enum {
   B_KF = 4, B_KE = 7,            // K stage full / free
   B_VF = 10, B_VE = 12,          // V stage full / free
   B_SF = 14, B_SR = 16,          // S buffer: scores ready / buffer (with the P in it) consumed by both P V
-  B_PF = 18, B_OF = 20,          // per stream: P announced / P V done
-  B_XC = 22, B_OR = 23,          // per item: streams exchanged (max, sum) / streams have read the O accumulators
-  B_N = 24
+  B_PF = 18,                     // per stream and S buffer (18 + 2 stream + buffer): P announced
+  B_OF = 22,                     // per stream: P V done
+  B_XC = 24, B_OR = 25,          // per item: streams published (reference, sum) / epilogue has read the O accumulators
+  B_N = 26
 };
 
 struct TcParams {
@@ -93,6 +94,15 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   asm volatile(
       "{\n\t.reg .pred p;\n\t"
       "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {   // one look, never suspends
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
       "selp.u32 %0, 1, 0, p;\n\t}"
       : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
   return ok != 0;
@@ -251,6 +261,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
       mbar_init(BAR(B_SF + s), 1);
       mbar_init(BAR(B_SR + s), 2);   // both P V issuers
       mbar_init(BAR(B_PF + s), 4);
+      mbar_init(BAR(B_PF + 2 + s), 4);
       mbar_init(BAR(B_OF + s), 1);
     }
     for (int s = 0; s < kKStages; ++s) {
@@ -349,8 +360,8 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
             // S(G) = Q K^T into S buffer G & 1, which held S(G-2) / P(G-2): wait until both
             // P V(G-2) have consumed it (they are issued by another thread)
             const int Gj = G + j, sb = Gj & 1, ks_ = Gj % kKStages;
-            if (Gj >= 2) ok = mbar_wait(BAR(B_SR + sb), ((Gj >> 1) - 1) & 1, abort_flag);
-            if (ok) ok = mbar_wait(BAR(B_KF + ks_), (Gj / kKStages) & 1, abort_flag);
+            ok = mbar_wait(BAR(B_KF + ks_), (Gj / kKStages) & 1, abort_flag);   // (long there as a rule)
+            if (ok && Gj >= 2) ok = mbar_wait(BAR(B_SR + sb), ((Gj >> 1) - 1) & 1, abort_flag);
             if (!ok) break;
             tc_fence_after();
             const uint64_t kdesc = smem_desc(base + kSmK + ks_ * kTileBytes, 16, 1024);
@@ -383,7 +394,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
           for (int j = 0; j < w.n_tiles && ok; ++j) {
             const int Gj = G + j, sb = Gj & 1, vs = Gj % kVStages;
             ok = mbar_wait(BAR(B_VF + vs), (Gj / kVStages) & 1, abort_flag);
-            if (ok) ok = mbar_wait(BAR(B_PF + hs), Gj & 1, abort_flag);
+            if (ok) ok = mbar_wait(BAR(B_PF + 2 * hs + sb), (Gj >> 1) & 1, abort_flag);
             if (!ok) break;
             tc_fence_after();
             // O_h += P_h V[64 h .. 64 h + 63]: A = P from tensor memory (two bf16 per column),
@@ -514,6 +525,9 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
           if (fresh) m_ref = fmaxf(mx0, mx1) * p.scale_log2e;
         }
         float neg_m = m_ref == -INFINITY ? 0.f : -m_ref;   // no visible key yet: weights 0, no NaN
+        // probe the next tile's scores now; the answer is read after the exponentials
+        const bool more = j + 1 < w.n_tiles;
+        const bool next_ready = more && mbar_test_wait(BAR(B_SF + (sb ^ 1)), ((Gj + 1) >> 1) & 1);
         float sum0 = 0.f, sum1 = 0.f, mxa = -INFINITY, mxb = -INFINITY;
         uint32_t pk[32];
 #pragma unroll
@@ -572,15 +586,13 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         tmem_st32(s_addr, pk);
         tmem_wait_st();
         tc_fence_before();
-        // back-pressure: P may only be announced once this stream's previous P V has run, so
-        // the announcement barrier is never more than one phase ahead of the MMA thread
-        if (Gj > 0 && !__all_sync(0xffffffffu, mbar_wait(BAR(B_OF + hs), (Gj - 1) & 1, abort_flag))) { ok = false; break; }
+        // (one announcement barrier per S buffer: its next phase cannot complete before the
+        // scores of tile G + 2 exist, that is before the MMA thread has consumed this one)
         __syncwarp();
-        if (lane == 0) mbar_arrive(BAR(B_PF + hs));
+        if (lane == 0) mbar_arrive(BAR(B_PF + 2 * hs + sb));
         // the next tile's scores
-        const bool more = j + 1 < w.n_tiles;
         if (more) {
-          if (!__all_sync(0xffffffffu, mbar_wait(BAR(B_SF + (sb ^ 1)), ((Gj + 1) >> 1) & 1, abort_flag))) { ok = false; break; }
+          if (!__all_sync(0xffffffffu, next_ready || mbar_wait(BAR(B_SF + (sb ^ 1)), ((Gj + 1) >> 1) & 1, abort_flag))) { ok = false; break; }
           tc_fence_after();
           const uint32_t n_addr = lane_base + kColS + (sb ^ 1) * 128 + hs * 64;
           tmem_ld32(n_addr, *reinterpret_cast<uint32_t(*)[32]>(&sv[0]));
