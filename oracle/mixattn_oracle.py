@@ -137,13 +137,20 @@ def decode_attention(q, K_hist, V_hist, kind: int, window: int,
 
 def prefill_attention(q, K, V, kind: int, window: int, scale: Optional[float] = None,
                       rows: Optional[Sequence[int]] = None,
-                      heads: Optional[Sequence[int]] = None) -> np.ndarray:
-    """Prompt attention for one sequence that starts at position 0.
+                      heads: Optional[Sequence[int]] = None,
+                      prefix_len: int = 0) -> np.ndarray:
+    """Prompt attention for one sequence.
 
-    q [S, Hq, D]; K, V [S, Hkv, D].  Row i is the decode definition with the
-    query at position i.  Returns [len(rows), len(heads), D]."""
+    q [S, Hq, D] are the queries of positions prefix_len .. prefix_len + S - 1;
+    K, V [prefix_len + S, Hkv, D] hold every key of the sequence up to the last
+    query (the first prefix_len of them were cached by earlier calls).  Row i is
+    the decode definition with the query at position prefix_len + i; with
+    prefix_len = 0 the sequence starts at position 0.
+    Returns [len(rows), len(heads), D]."""
     q, K, V = _as64(q), _as64(K), _as64(V)
     S, n_q, D = q.shape
+    if K.shape[0] != prefix_len + S or V.shape[0] != prefix_len + S:
+        raise OracleError(ERR_INVALID_ARG, "K, V must hold prefix_len + S keys")
     n_kv = K.shape[1]
     G = n_q // n_kv
     scale = 1.0 / np.sqrt(D) if scale is None else scale
@@ -151,7 +158,7 @@ def prefill_attention(q, K, V, kind: int, window: int, scale: Optional[float] = 
     hs = range(n_q) if heads is None else heads
     out = np.empty((len(rs), len(hs), D))
     for a, i in enumerate(rs):
-        lo, hi = key_range(kind, window, i)
+        lo, hi = key_range(kind, window, prefix_len + i)
         for c, h in enumerate(hs):
             g = h // G
             out[a, c] = softmax_attend(q[i, h], K[lo:hi, g], V[lo:hi, g], scale)

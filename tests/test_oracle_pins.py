@@ -340,3 +340,57 @@ def test_two_full_owners_share_one_block_table():
         ph.append(1, [0])
     assert ph.get_block_table(0) == [0, 1] and ph.n_free_pages() == 6
     assert ph.get_len(0, 0) == 20 and ph.get_len(1, 0) == 20
+
+
+# --------------------------------------------------------------------------
+# chunks of queries behind a cached prefix
+# --------------------------------------------------------------------------
+
+@pytest.mark.parametrize("kind,window", [(FULL, 0), (SLIDING, 1), (SLIDING, 5), (SLIDING, 16), (SLIDING, 100)])
+def test_chunk_behind_prefix_is_the_dense_masked_reference(kind, window):
+    # rows prefix..prefix+S-1 of the dense masked reference over the whole sequence, for chunk
+    # boundaries before, at and after the window length, and a single-token chunk
+    rng = np.random.default_rng(11 + window)
+    n, Hq, Hkv, D = 41, 4, 2, 8
+    q, K, V = rnd(rng, n, Hq, D), rnd(rng, n, Hkv, D), rnd(rng, n, Hkv, D)
+    ref = dense_reference(q, K, V, kind, window)
+    for prefix, S in ((0, n), (1, 40), (4, 9), (5, 1), (16, 25), (17, 3), (40, 1)):
+        got = mo.prefill_attention(q[prefix:prefix + S], K[:prefix + S], V[:prefix + S], kind, window,
+                                   prefix_len=prefix)
+        np.testing.assert_allclose(got, ref[prefix:prefix + S], rtol=0, atol=1e-12)
+
+
+def test_chunk_behind_prefix_matches_torch_sdpa_with_an_explicit_mask():
+    rng = np.random.default_rng(5)
+    prefix, S, Hq, Hkv, D, W = 13, 7, 6, 2, 16, 6
+    n = prefix + S
+    q, K, V = rnd(rng, S, Hq, D), rnd(rng, n, Hkv, D), rnd(rng, n, Hkv, D)
+    G = Hq // Hkv
+    tq = torch.from_numpy(q).permute(1, 0, 2)[None]
+    tk = torch.from_numpy(K).repeat_interleave(G, dim=1).permute(1, 0, 2)[None]
+    tv = torch.from_numpy(V).repeat_interleave(G, dim=1).permute(1, 0, 2)[None]
+    pos_q = torch.arange(prefix, n)[:, None]
+    pos_k = torch.arange(n)[None, :]
+    for kind, window, mask in ((FULL, 0, pos_k <= pos_q),
+                               (SLIDING, W, (pos_k <= pos_q) & (pos_q - pos_k < W))):
+        ref = torch.nn.functional.scaled_dot_product_attention(tq, tk, tv, attn_mask=mask)
+        ref = ref[0].permute(1, 0, 2).numpy()
+        got = mo.prefill_attention(q, K, V, kind, window, prefix_len=prefix)
+        np.testing.assert_allclose(got, ref, rtol=0, atol=1e-12)
+
+
+def test_single_token_chunk_is_decode():
+    rng = np.random.default_rng(9)
+    n, Hq, Hkv, D = 30, 4, 1, 8
+    q, K, V = rnd(rng, 1, Hq, D), rnd(rng, n, Hkv, D), rnd(rng, n, Hkv, D)
+    for kind, window in ((FULL, 0), (SLIDING, 7)):
+        a = mo.prefill_attention(q, K, V, kind, window, prefix_len=n - 1)[0]
+        b = mo.decode_attention(q[0], K, V, kind, window)
+        np.testing.assert_allclose(a, b, rtol=0, atol=1e-13)
+
+
+def test_chunk_needs_every_key_up_to_its_last_query():
+    rng = np.random.default_rng(1)
+    q, K = rnd(rng, 3, 2, 4), rnd(rng, 9, 2, 4)
+    with pytest.raises(mo.OracleError):
+        mo.prefill_attention(q, K, K, FULL, 0, prefix_len=5)
