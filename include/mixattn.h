@@ -75,6 +75,8 @@ typedef struct {
                                        ignores k/v; decode and prefill return MIXATTN_ERR_CUDA)     */
   void* arena;                      /* device memory allocated by the caller, 256-byte aligned      */
   size_t arena_bytes;               /* >= mixattn_arena_bytes(); the library never frees it         */
+  int32_t chunk_scratch_tokens;     /* K/V rows of scratch kept in the arena for
+                                       mixattn_attend_chunk; 0 = that call is unavailable           */
 } mixattn_config;
 
 /* Bytes of device memory a context with this config carves out of `arena`:
@@ -151,6 +153,31 @@ int mixattn_decode(mixattn_ctx* ctx, int32_t layer, int32_t n_seqs, const int32_
 int mixattn_prefill(mixattn_ctx* ctx, int32_t layer, int32_t n_seqs, const int32_t* seq_ids,
                     const int32_t* seq_lens, const void* q, const void* k, const void* v,
                     void* out, void* stream);
+
+/* Attention of a chunk of new tokens behind what the caches already hold
+ * (Section 3's definition with the queries at positions n .. n+S-1; Section 5
+ * serves prompts of tens of thousands of tokens, which arrive in chunks, and a
+ * chunk of a few tokens is a multi-token decode step).  For each sequence, with
+ * n = tokens in the cache `layer` reads, query r of the chunk sits at position
+ * n + r and attends to the cached keys and to the chunk's own keys up to its
+ * position: all of them (standard layer) or the last `window` (sliding window).
+ *   seq_lens host, chunk length S_b of each sequence (>= 1)
+ *   q, out   device, [sum S_b, n_q_heads, head_dim], sequences back to back
+ *   k, v     device, [sum S_b, n_kv_heads, head_dim]: the chunk's K/V as the
+ *            layer's owner computed them (16-byte aligned)
+ * The call STORES NOTHING: once every layer that reads a cache has run on the
+ * chunk, the caller appends the chunk to that cache's owner with
+ * mixattn_append_kv (a ring shared by several layers must still hold the
+ * window of the chunk's first token when the last of them runs).
+ * The cached keys the chunk needs (all of a paged cache, the last window-1
+ * tokens of a ring) and the chunk's are first copied into plain tensors in the
+ * context's chunk scratch, sequences in groups that fit it.
+ * Errors: UNSUPPORTED if the context was created with chunk_scratch_tokens = 0,
+ * TOO_LARGE if one sequence's keys alone exceed the scratch, BAD_SEQ,
+ * INVALID_ARG (null, duplicates, S_b < 1, n + S_b beyond max_seq_len), CUDA. */
+int mixattn_attend_chunk(mixattn_ctx* ctx, int32_t layer, int32_t n_seqs, const int32_t* seq_ids,
+                         const int32_t* seq_lens, const void* q, const void* k, const void* v,
+                         void* out, void* stream);
 
 /* Size of the static device array behind mixattn_decode_static_scratch. */
 #define MIXATTN_STATIC_SCRATCH_BYTES (8u << 20)
@@ -237,7 +264,8 @@ enum {
   MIXATTN_K_COMBINE = 3,
   MIXATTN_K_PREFILL_FULL = 4,
   MIXATTN_K_PREFILL_SLIDING = 5,
-  MIXATTN_K_COUNT = 6
+  MIXATTN_K_GATHER = 6,         /* copy of cached + chunk keys ahead of a chunk's attention */
+  MIXATTN_K_COUNT = 7
 };
 
 /* enable != 0: from now on every kernel launch is bracketed by CUDA events on

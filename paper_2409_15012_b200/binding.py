@@ -27,7 +27,7 @@ ERR_UNSUPPORTED = -7
 ERR_CUDA = -8
 ERR_TOO_LARGE = -9
 
-K_APPEND, K_DECODE_FULL, K_DECODE_SLIDING, K_COMBINE, K_PREFILL_FULL, K_PREFILL_SLIDING = range(6)
+K_APPEND, K_DECODE_FULL, K_DECODE_SLIDING, K_COMBINE, K_PREFILL_FULL, K_PREFILL_SLIDING, K_GATHER = range(7)
 
 _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libmixattn.so")
 
@@ -53,6 +53,7 @@ class Config(C.Structure):
         ("device", C.c_int32),
         ("arena", C.c_void_p),
         ("arena_bytes", C.c_size_t),
+        ("chunk_scratch_tokens", C.c_int32),
     ]
 
 
@@ -73,6 +74,7 @@ def _load() -> C.CDLL:
         "mixattn_append_kv": [vp, i32, i32, p32, p32, vp, vp, vp],
         "mixattn_decode": [vp, i32, i32, p32, vp, vp, vp],
         "mixattn_decode_static_scratch": [vp, i32, i32, p32, vp, vp, vp],
+        "mixattn_attend_chunk": [vp, i32, i32, p32, p32, vp, vp, vp, vp, vp],
         "mixattn_prefill": [vp, i32, i32, p32, p32, vp, vp, vp, vp, vp],
         "mixattn_get_len": [vp, i32, i32, p32],
         "mixattn_get_block_table": [vp, i32, p32, i32, p32],
@@ -99,6 +101,7 @@ lib = _load()
 EXPORTS = [
     "mixattn_arena_bytes", "mixattn_cache_bytes", "mixattn_create", "mixattn_destroy",
     "mixattn_seq_reset", "mixattn_append_kv", "mixattn_decode", "mixattn_decode_static_scratch", "mixattn_prefill",
+    "mixattn_attend_chunk",
     "mixattn_get_len", "mixattn_get_block_table", "mixattn_get_n_free_pages",
     "mixattn_get_ring_state", "mixattn_locate", "mixattn_debug_read_kv",
     "mixattn_get_device_status", "mixattn_set_split_tokens", "mixattn_profile_enable",
@@ -136,14 +139,16 @@ def _stream(stream) -> Optional[int]:
 
 def make_config(layout: Sequence, n_q_heads: int, n_kv_heads: int, head_dim: int, dtype: int,
                 max_seqs: int, n_pages: int, max_seq_len: int = 0, free_order=None,
-                softmax_scale: float = 0.0, device: int = -1, page_size: int = 16):
+                softmax_scale: float = 0.0, device: int = -1, page_size: int = 16,
+                chunk_scratch_tokens: int = 0):
     """Returns (Config, keepalive): keepalive owns the arrays the struct points to."""
     layers = (LayerDesc * max(1, len(layout)))()
     for i, (kind, window, owner) in enumerate(layout):
         layers[i] = LayerDesc(int(kind), int(window), int(owner))
     fo = None if free_order is None else _i32(free_order)
     cfg = Config(len(layout), layers, n_q_heads, n_kv_heads, head_dim, dtype, max_seqs, page_size,
-                 n_pages, max_seq_len, _p32(fo), float(softmax_scale), device, None, 0)
+                 n_pages, max_seq_len, _p32(fo), float(softmax_scale), device, None, 0,
+                 int(chunk_scratch_tokens))
     return cfg, (layers, fo)
 
 
@@ -171,9 +176,10 @@ class Context:
     """
 
     def __init__(self, layout, n_q_heads, n_kv_heads, head_dim, dtype, max_seqs, n_pages,
-                 max_seq_len=0, free_order=None, softmax_scale=0.0, device=-1):
+                 max_seq_len=0, free_order=None, softmax_scale=0.0, device=-1, chunk_scratch_tokens=0):
         self.cfg, self._keep = make_config(layout, n_q_heads, n_kv_heads, head_dim, dtype, max_seqs,
-                                           n_pages, max_seq_len, free_order, softmax_scale, device)
+                                           n_pages, max_seq_len, free_order, softmax_scale, device,
+                                           chunk_scratch_tokens=chunk_scratch_tokens)
         self.arena = None
         if device >= 0:
             import torch
@@ -236,6 +242,16 @@ class Context:
         rc = self.rc_prefill(layer, seq_ids, seq_lens, q, k, v, out, stream)
         if rc:
             raise MixAttnError(rc, "mixattn_prefill")
+
+    def rc_attend_chunk(self, layer, seq_ids, seq_lens, q, k, v, out, stream=None) -> int:
+        s, n = _i32(seq_ids), _i32(seq_lens)
+        return lib.mixattn_attend_chunk(self.h, layer, len(s), _p32(s), _p32(n), _dev(q), _dev(k), _dev(v),
+                                        _dev(out), _stream(stream))
+
+    def attend_chunk(self, layer, seq_ids, seq_lens, q, k, v, out, stream=None):
+        rc = self.rc_attend_chunk(layer, seq_ids, seq_lens, q, k, v, out, stream)
+        if rc:
+            raise MixAttnError(rc, "mixattn_attend_chunk")
 
     def seq_reset(self, seq):
         rc = lib.mixattn_seq_reset(self.h, seq)

@@ -24,6 +24,7 @@ struct ArenaPlan {
   std::vector<size_t> owner_bytes;
   size_t table_off = 0, table_bytes = 0;
   size_t part_o_off = 0, part_ml_off = 0, status_off = 0;
+  size_t chunk_k_off = 0, chunk_v_off = 0;   // [chunk_scratch_tokens, Hkv, D] each
   size_t cache_bytes = 0, total = 0;
 };
 
@@ -52,6 +53,13 @@ ArenaPlan plan_arena(const CacheManager& cm, const mixattn_config& cfg) {
   off += align_up((size_t)kWsChunks * cfg.n_q_heads * sizeof(float2));
   pl.status_off = off;
   off += kAlign;
+  if (cfg.chunk_scratch_tokens > 0) {
+    const size_t bytes = align_up((size_t)cfg.chunk_scratch_tokens * ge.n_kv_heads * ge.row_bytes);
+    pl.chunk_k_off = off;
+    off += bytes;
+    pl.chunk_v_off = off;
+    off += bytes;
+  }
   pl.total = off;
   return pl;
 }
@@ -137,6 +145,7 @@ int validate_config(const mixattn_config* cfg, CacheManager* cm, bool allocate =
   if (rc != MIXATTN_OK) return rc;
   if (cfg->softmax_scale < 0.f || !isfinite(cfg->softmax_scale)) return MIXATTN_ERR_INVALID_ARG;
   if (cm->n_full_owners() > 0 && cfg->n_pages < 1) return MIXATTN_ERR_INVALID_ARG;
+  if (cfg->chunk_scratch_tokens < 0) return MIXATTN_ERR_INVALID_ARG;
   return MIXATTN_OK;
 }
 
@@ -462,6 +471,8 @@ int mixattn_prefill(mixattn_ctx* c, int32_t layer, int32_t n_seqs, const int32_t
     int r = 0, mlen = 0;
     for (int j = 0; j < nb; ++j) {
       p.row0[j] = r;
+      p.krow0[j] = r;
+      p.prefix[j] = 0;
       r += seq_lens[i0 + j];
       if (seq_lens[i0 + j] > mlen) mlen = seq_lens[i0 + j];
     }
@@ -480,6 +491,113 @@ int mixattn_prefill(mixattn_ctx* c, int32_t layer, int32_t n_seqs, const int32_t
       return tc ? launch_prefill_tc(p, mlen, c->sm_count, st) : launch_prefill_simple(p, c->cfg.dtype, mlen, st);
     });
     if (e != cudaSuccess) return MIXATTN_ERR_CUDA;
+  }
+  return MIXATTN_OK;
+}
+
+int mixattn_attend_chunk(mixattn_ctx* c, int32_t layer, int32_t n_seqs, const int32_t* seq_ids,
+                         const int32_t* seq_lens, const void* q, const void* k, const void* v,
+                         void* out, void* stream) {
+  if (c == nullptr || !c->cm.valid_layer(layer) || n_seqs < 0) return MIXATTN_ERR_INVALID_ARG;
+  if (n_seqs > 0 && (seq_ids == nullptr || seq_lens == nullptr)) return MIXATTN_ERR_INVALID_ARG;
+  const LayerInfo& li = c->cm.layer(layer);
+  const bool ring = li.kind == MIXATTN_SLIDING;
+  const int scratch = c->cfg.chunk_scratch_tokens;
+  // cached keys each sequence's chunk needs: all of a paged cache, the last window - 1 of a ring
+  std::vector<int32_t> n_prefix(n_seqs > 0 ? n_seqs : 0);
+  {
+    std::vector<char> seen(c->cm.max_seqs(), 0);
+    int64_t total = 0;
+    for (int i = 0; i < n_seqs; ++i) {
+      if (!c->cm.valid_seq(seq_ids[i])) return MIXATTN_ERR_BAD_SEQ;
+      if (seen[seq_ids[i]]) return MIXATTN_ERR_INVALID_ARG;
+      seen[seq_ids[i]] = 1;
+      if (seq_lens[i] < 1) return MIXATTN_ERR_INVALID_ARG;
+      const int64_t n = c->cm.len(layer, seq_ids[i]);
+      if (n + seq_lens[i] > c->cm.max_seq_len()) return MIXATTN_ERR_INVALID_ARG;
+      total += seq_lens[i];
+      n_prefix[i] = (int32_t)(ring ? (n < li.window - 1 ? n : li.window - 1) : n);
+    }
+    if (total > INT32_MAX) return MIXATTN_ERR_INVALID_ARG;
+  }
+  if (scratch <= 0) return MIXATTN_ERR_UNSUPPORTED;
+  for (int i = 0; i < n_seqs; ++i)
+    if ((int64_t)n_prefix[i] + seq_lens[i] > scratch) return MIXATTN_ERR_TOO_LARGE;
+  if (c->host_only || c->sticky_cuda_error) return MIXATTN_ERR_CUDA;
+  if (n_seqs == 0) return MIXATTN_OK;
+  if (q == nullptr || k == nullptr || v == nullptr || out == nullptr) return MIXATTN_ERR_INVALID_ARG;
+  if ((((size_t)k) | ((size_t)v)) & 15) return MIXATTN_ERR_INVALID_ARG;
+  DeviceGuard g(c->device);
+  if (!g.ok) return MIXATTN_ERR_CUDA;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const int Hq = c->cfg.n_q_heads, Hkv = c->cfg.n_kv_heads, D = c->cfg.head_dim;
+  const size_t esz = c->geom.elem_bytes;
+  char* ks = c->arena + c->plan.chunk_k_off;
+  char* vs = c->arena + c->plan.chunk_v_off;
+
+  GatherParams gp;
+  gp.k_out = ks;
+  gp.v_out = vs;
+  gp.pool = c->owner_storage(layer);
+  gp.table = c->dev_table();
+  gp.table_stride = c->cm.max_blocks();
+  gp.is_ring = ring;
+  gp.window = ring ? li.window : 0;
+  gp.ring_pages = ring ? ring_pages_of(li.window) : 0;
+  gp.geom = c->geom;
+  PrefillParams p;
+  p.n_q_heads = Hq;
+  p.n_kv_heads = Hkv;
+  p.head_dim = D;
+  p.window = ring ? li.window : 0;
+  p.scale_log2e = c->scale * 1.4426950408889634f;
+  p.status = c->dev_status();
+  p.k = ks;
+  p.v = vs;
+
+  // groups of consecutive sequences whose keys fit the scratch together; the stream orders
+  // each group's attention before the next group's copy reuses the scratch
+  int64_t row = 0;   // first chunk row of the group in q / k / v / out
+  for (int i0 = 0; i0 < n_seqs;) {
+    int nb = 0, mlen = 0, max_rows = 0;
+    int32_t krow = 0, qrow = 0;
+    while (i0 + nb < n_seqs && nb < kMaxCallSeqs) {
+      const int i = i0 + nb;
+      const int rows = n_prefix[i] + seq_lens[i];
+      if (krow + rows > scratch) break;
+      GatherEntry& e = gp.e[nb];
+      e.seq = seq_ids[i];
+      e.n_prefix = n_prefix[i];
+      e.pos0 = c->cm.len(layer, seq_ids[i]) - n_prefix[i];
+      e.n_chunk = seq_lens[i];
+      e.src_row0 = qrow;
+      e.dst_row0 = krow;
+      p.row0[nb] = qrow;
+      p.krow0[nb] = krow;
+      p.prefix[nb] = n_prefix[i];
+      krow += rows;
+      qrow += seq_lens[i];
+      if (seq_lens[i] > mlen) mlen = seq_lens[i];
+      if (rows > max_rows) max_rows = rows;
+      ++nb;
+    }
+    p.row0[nb] = qrow;
+    p.n_seqs = nb;
+    gp.n_entries = nb;
+    gp.k_chunk = static_cast<const char*>(k) + (size_t)row * Hkv * D * esz;
+    gp.v_chunk = static_cast<const char*>(v) + (size_t)row * Hkv * D * esz;
+    p.q = static_cast<const char*>(q) + (size_t)row * Hq * D * esz;
+    p.out = static_cast<char*>(out) + (size_t)row * Hq * D * esz;
+    cudaError_t e = launch_recorded(c, MIXATTN_K_GATHER, st, [&] { return launch_gather(gp, max_rows, st); });
+    if (e != cudaSuccess) return MIXATTN_ERR_CUDA;
+    const int cls = p.window ? MIXATTN_K_PREFILL_SLIDING : MIXATTN_K_PREFILL_FULL;
+    const bool tc = prefill_tc_supported(c->cfg.dtype, D, p.q, p.k, p.v) && (((size_t)p.out) & 15) == 0;
+    e = launch_recorded(c, cls, st, [&] {
+      return tc ? launch_prefill_tc(p, mlen, c->sm_count, st) : launch_prefill_simple(p, c->cfg.dtype, mlen, st);
+    });
+    if (e != cudaSuccess) return MIXATTN_ERR_CUDA;
+    row += qrow;
+    i0 += nb;
   }
   return MIXATTN_OK;
 }

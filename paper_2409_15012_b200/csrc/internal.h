@@ -114,7 +114,37 @@ struct PrefillParams {
   float scale_log2e;
   int32_t n_seqs;
   int32_t* status;
-  int32_t row0[kMaxCallSeqs + 1];  // first row of each sequence in the packed tensors
+  int32_t row0[kMaxCallSeqs + 1];   // first row of each sequence in q / out (packed)
+  int32_t krow0[kMaxCallSeqs];      // first row of each sequence in k / v
+  int32_t prefix[kMaxCallSeqs];     // key rows of the sequence that precede its first query:
+                                    // k / v hold prefix + (row0[b + 1] - row0[b]) rows for sequence b
+};
+
+// Copies the cached keys a chunk of queries needs, followed by the chunk's own keys, into
+// plain [rows, Hkv, D] tensors (the layout the prompt kernels read).
+struct GatherEntry {
+  int32_t seq;        // sequence slot
+  int32_t pos0;       // position of the first cached token copied
+  int32_t n_prefix;   // cached tokens copied (positions pos0 .. pos0 + n_prefix - 1)
+  int32_t n_chunk;    // tokens taken from the chunk tensors after them
+  int32_t src_row0;   // first row of the chunk in k_chunk / v_chunk
+  int32_t dst_row0;   // first row written in k_out / v_out
+};
+
+struct GatherParams {
+  const void* k_chunk;
+  const void* v_chunk;
+  void* k_out;
+  void* v_out;
+  const char* pool;
+  const int32_t* table;
+  int32_t table_stride;
+  int32_t is_ring;
+  int32_t window;
+  int32_t ring_pages;
+  KvGeom geom;
+  int32_t n_entries;
+  GatherEntry e[kMaxCallSeqs];
 };
 
 // device status codes written to the status word
@@ -122,6 +152,7 @@ enum { kDevOk = 0, kDevWaitTimeout = 1 };
 
 // launchers (each returns the cudaError_t of its launch)
 cudaError_t launch_append(const AppendParams& p, int max_n_new, cudaStream_t st);
+cudaError_t launch_gather(const GatherParams& p, int max_rows, cudaStream_t st);
 cudaError_t prepare_decode_bf16();
 cudaError_t launch_decode_split_bf16(const DecodeParams& p, int sm_count, cudaStream_t st);
 cudaError_t launch_decode_split_f32(const DecodeParams& p, cudaStream_t st);

@@ -2,7 +2,9 @@
 //
 // Paper, Section 3 with the causal order of Section 1: query i attends to keys j <= i
 // (standard layer) or i - window < j <= i (sliding window).  This is the fp32-mode
-// prefill and the fallback for shapes the tensor-core kernel does not take.
+// prefill and the fallback for shapes the tensor-core kernel does not take.  A sequence's
+// queries may sit behind `prefix` keys that earlier calls cached: query row r then has
+// position prefix + r among the sequence's prefix + S key rows.
 // Flash-attention tiling (32 queries x 32 keys per step, online softmax in base 2); key
 // tiles outside the band are skipped.
 #include <cuda_bf16.h>
@@ -33,7 +35,8 @@ __global__ void __launch_bounds__(kThreads) prefill_simple_kernel(const __grid_c
   const int i0 = blockIdx.x * kBM;
   if (i0 >= S) return;
   const int g = h / (p.n_q_heads / p.n_kv_heads);
-  const int64_t base = p.row0[b];
+  const int64_t base = p.row0[b], kbase = p.krow0[b];
+  const int P = p.prefix[b];            // key rows before the first query
   const T* q = reinterpret_cast<const T*>(p.q);
   const T* k = reinterpret_cast<const T*>(p.k);
   const T* v = reinterpret_cast<const T*>(p.v);
@@ -47,18 +50,20 @@ __global__ void __launch_bounds__(kThreads) prefill_simple_kernel(const __grid_c
 #pragma unroll
   for (int e = 0; e < D / 4; ++e) o[e] = 0.f;
   float m = -INFINITY, l = 0.f;
-  const int i = i0 + r;  // this thread's query position
+  const int i = P + i0 + r;  // this thread's query position
+  const bool row_ok = i0 + r < S;
 
-  const int i_last = min(S, i0 + kBM) - 1;
+  const int n_keys = P + S;
+  const int i_last = P + min(S, i0 + kBM) - 1;
   int j_lo = 0;
-  if (p.window > 0) j_lo = max(0, i0 - p.window + 1) / kBN * kBN;
+  if (p.window > 0) j_lo = max(0, P + i0 - p.window + 1) / kBN * kBN;
   for (int j0 = j_lo; j0 <= i_last; j0 += kBN) {
     __syncthreads();
     for (int e = tid; e < kBN * D; e += kThreads) {
       const int jj = e / D, d = e - jj * D;
-      const bool in = j0 + jj < S;
-      Ks[jj * (D + 1) + d] = in ? to_f32(k[((base + j0 + jj) * p.n_kv_heads + g) * D + d]) : 0.f;
-      Vs[jj * D + d] = in ? to_f32(v[((base + j0 + jj) * p.n_kv_heads + g) * D + d]) : 0.f;
+      const bool in = j0 + jj < n_keys;
+      Ks[jj * (D + 1) + d] = in ? to_f32(k[((kbase + j0 + jj) * p.n_kv_heads + g) * D + d]) : 0.f;
+      Vs[jj * D + d] = in ? to_f32(v[((kbase + j0 + jj) * p.n_kv_heads + g) * D + d]) : 0.f;
     }
     __syncthreads();
     float s[kBN / 4];
@@ -68,7 +73,7 @@ __global__ void __launch_bounds__(kThreads) prefill_simple_kernel(const __grid_c
       const int j = j0 + c + 4 * jj;
       float acc = 0.f;
       for (int d = 0; d < D; ++d) acc = fmaf(Qs[r * (D + 1) + d], Ks[(c + 4 * jj) * (D + 1) + d], acc);
-      const bool seen = j <= i && i < S && (p.window == 0 || i - j < p.window);
+      const bool seen = j <= i && row_ok && (p.window == 0 || i - j < p.window);
       s[jj] = seen ? acc * p.scale_log2e : -INFINITY;
       mx = fmaxf(mx, s[jj]);
     }
@@ -97,8 +102,8 @@ __global__ void __launch_bounds__(kThreads) prefill_simple_kernel(const __grid_c
       for (int e = 0; e < D / 4; ++e) o[e] = fmaf(pe, Vs[jj * D + c + 4 * e], o[e]);
     }
   }
-  if (i < S) {
-    T* out = reinterpret_cast<T*>(p.out) + ((base + i) * p.n_q_heads + h) * D;
+  if (row_ok) {
+    T* out = reinterpret_cast<T*>(p.out) + ((base + i0 + r) * p.n_q_heads + h) * D;
     const float inv = 1.f / l;
 #pragma unroll
     for (int e = 0; e < D / 4; ++e) store_out(out + c + 4 * e, o[e] * inv);

@@ -3,7 +3,9 @@
 // Paper, Section 3 with the causal order of Section 1: query i attends to keys j <= i
 // (standard layer) or i - window < j <= i (sliding window).  Flash-attention forward:
 // one CTA owns a 128-query tile of one (sequence, head) and walks the 128-key tiles that
-// intersect its band; tiles wholly outside the band are never loaded.
+// intersect its band; tiles wholly outside the band are never loaded.  A sequence's queries
+// may sit behind a prefix of keys cached by earlier calls (k / v then hold prefix + S rows):
+// query row r has position prefix + r.
 //
 //   warp 0     TMA producer: Q once, then K and V tiles (3 / 2 stages) as 128B-swizzled
 //              [128 x 64] boxes straight from the caller's tensors
@@ -76,7 +78,9 @@ struct TcParams {
   float scale_log2e;
   int32_t* status;
   __nv_bfloat16* out;
-  int32_t row0[kMaxCallSeqs + 1];
+  int32_t row0[kMaxCallSeqs + 1];   // first q / out row of each sequence
+  int32_t krow0[kMaxCallSeqs];      // first k / v row of each sequence
+  int32_t prefix[kMaxCallSeqs];     // key rows before the sequence's first query
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -215,7 +219,7 @@ __host__ __device__ constexpr uint32_t idesc_bf16(int b_mn) {
 // in L2 (a pass over all sequences at once re-read K/V from HBM 5x), heaviest tiles first,
 // and the heads of a KV group, which read the same K/V tiles, run at the same time.
 struct WorkItem {
-  int h, g, row_base, S, i0, jt_lo, n_tiles;
+  int h, g, row_base, krow_base, S, i0, pos0, jt_lo, n_tiles;   // pos0 = position of query row i0 among the keys
   bool valid;
 };
 __device__ __forceinline__ WorkItem get_item(const TcParams& p, int id) {
@@ -227,12 +231,14 @@ __device__ __forceinline__ WorkItem get_item(const TcParams& p, int id) {
   w.h = rem - qt_rev * p.n_q_heads;
   w.g = w.h / p.group;
   w.row_base = p.row0[b];
+  w.krow_base = p.krow0[b];
   w.S = p.row0[b + 1] - p.row0[b];
   const int qt = (w.S + kBM - 1) / kBM - 1 - qt_rev;
   w.valid = qt >= 0;
   w.i0 = qt * kBM;
-  const int key_hi = min(w.i0 + kBM - 1, w.S - 1);
-  const int key_lo = p.window > 0 ? max(0, w.i0 - p.window + 1) : 0;
+  w.pos0 = p.prefix[b] + w.i0;
+  const int key_hi = p.prefix[b] + min(w.i0 + kBM - 1, w.S - 1);
+  const int key_lo = p.window > 0 ? max(0, w.pos0 - p.window + 1) : 0;
   w.jt_lo = key_lo / kBN;
   w.n_tiles = key_hi / kBN - w.jt_lo + 1;
   return w;
@@ -309,7 +315,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
           ++q_issued;
           for (int j = 0; j < w.n_tiles && ok; ++j) {
             const int Gj = G + j;
-            const int row = w.row_base + (w.jt_lo + j) * kBN;
+            const int row = w.krow_base + (w.jt_lo + j) * kBN;
             const int ks = Gj % kKStages, ku = Gj / kKStages;
             if (ku > 0) ok = mbar_wait(BAR(B_KE + ks), (ku - 1) & 1, abort_flag);
             if (!ok) break;
@@ -488,7 +494,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     for (int id = blockIdx.x; id < n_ids && ok; id += gridDim.x) {
       const WorkItem w = get_item(p, id);
       if (!w.valid) continue;
-      const int i = w.i0 + r;             // query position
+      const int i = w.pos0 + r;           // query position among the sequence's keys
       float m_ref = -INFINITY, l = 0.f;
       uint32_t sv[64];
       {
@@ -504,7 +510,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         const int j0 = (w.jt_lo + j) * kBN + hs * 64;   // first key of this stream's columns
         const uint32_t s_addr = lane_base + kColS + sb * 128 + hs * 64;
         // band edges: causal (keys after the query) and window (keys older than i - window)
-        const bool edge = (j0 + 63 > w.i0) || (p.window > 0 && j0 <= w.i0 + kBM - 1 - p.window);
+        const bool edge = (j0 + 63 > w.pos0) || (p.window > 0 && j0 <= w.pos0 + kBM - 1 - p.window);
         auto mask_edges = [&]() {
           const int k_max = i - j0;                                      // columns <= k_max are causal-visible
           const int k_min = p.window > 0 ? i - p.window + 1 - j0 : 0;    // columns >= k_min are inside the window
@@ -666,9 +672,14 @@ cudaError_t prepare_prefill_tc() {
 cudaError_t launch_prefill_tc(const PrefillParams& pp, int max_len, int sm_count, cudaStream_t st) {
   if (pp.n_seqs <= 0 || max_len <= 0) return cudaSuccess;
   const int64_t rows = pp.row0[pp.n_seqs];
+  int64_t k_rows = 0;   // k / v hold prefix + S rows per sequence
+  for (int i = 0; i < pp.n_seqs; ++i) {
+    const int64_t end = (int64_t)pp.krow0[i] + pp.prefix[i] + (pp.row0[i + 1] - pp.row0[i]);
+    if (end > k_rows) k_rows = end;
+  }
   CUtensorMap tq, tk, tv;
-  if (!make_map(&tq, pp.q, rows, pp.n_q_heads) || !make_map(&tk, pp.k, rows, pp.n_kv_heads) ||
-      !make_map(&tv, pp.v, rows, pp.n_kv_heads))
+  if (!make_map(&tq, pp.q, rows, pp.n_q_heads) || !make_map(&tk, pp.k, k_rows, pp.n_kv_heads) ||
+      !make_map(&tv, pp.v, k_rows, pp.n_kv_heads))
     return cudaErrorInvalidValue;
   TcParams p;
   p.n_q_heads = pp.n_q_heads;
@@ -679,6 +690,10 @@ cudaError_t launch_prefill_tc(const PrefillParams& pp, int max_len, int sm_count
   p.status = pp.status;
   p.out = static_cast<__nv_bfloat16*>(pp.out);
   for (int i = 0; i <= pp.n_seqs; ++i) p.row0[i] = pp.row0[i];
+  for (int i = 0; i < pp.n_seqs; ++i) {
+    p.krow0[i] = pp.krow0[i];
+    p.prefix[i] = pp.prefix[i];
+  }
   p.max_qt = (max_len + kBM - 1) / kBM;
   const int64_t n_ids = (int64_t)p.max_qt * pp.n_seqs * pp.n_q_heads;
   const int grid = (int)(n_ids < sm_count ? n_ids : sm_count);   // persistent: one CTA per SM

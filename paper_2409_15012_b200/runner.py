@@ -29,7 +29,7 @@ class Session:
 
     def __init__(self, wl: cf.Workload, lengths: Optional[Sequence[int]] = None, device: int = 0,
                  headroom_tokens: int = 0, free_order=None, n_pages: Optional[int] = None,
-                 mirror=None):
+                 mirror=None, chunk_scratch_tokens: int = 0):
         self.wl = wl
         self.device = device
         self.dev = torch.device(f"cuda:{device}")
@@ -50,7 +50,8 @@ class Session:
         self.free_order = free_order
         self.mirror = mirror
         self.ctx = mx.Context(wl.layout, wl.n_q_heads, wl.n_kv_heads, wl.head_dim, wl.dtype, B,
-                              n_pages, max_seq_len=max(max_len, 1), free_order=free_order, device=device)
+                              n_pages, max_seq_len=max(max_len, 1), free_order=free_order, device=device,
+                              chunk_scratch_tokens=chunk_scratch_tokens)
 
     def close(self):
         self.ctx.close()

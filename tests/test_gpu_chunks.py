@@ -1,0 +1,129 @@
+"""Chunks of new tokens behind a cached prefix (chunked prompts, multi-token decode
+steps) on a B200 against the CPU checker: every chunk of every layer element by element,
+the cache state bit for bit after the appends that follow, and a decode step at the end."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import mixattn_oracle as mo
+from synth import configs as cf
+from synth import inputs as si
+
+from gpu_common import check_close, check_stored_bits, compare_state, load_lib, ref_decode, torch_dt
+
+pytestmark = pytest.mark.gpu
+
+
+def run_chunked(wl: cf.Workload, schedule, scratch: int, rows_per_chunk=None):
+    """schedule[b] = chunk lengths of sequence b (0 = the sequence sits that round out)."""
+    mx, runner = load_lib()
+    B = wl.batch
+    totals = [sum(s) for s in schedule]
+    sess = runner.Session(wl, totals, headroom_tokens=2, chunk_scratch_tokens=scratch)
+    ph = mo.PhysicalCache(wl.layout, wl.n_kv_heads, wl.head_dim, B, sess.n_pages, store_values=False)
+    dt = torch_dt(wl.dtype)
+    pos = [0] * B
+    try:
+        for rnd in range(max(len(s) for s in schedule)):
+            ids = [b for b in range(B) if rnd < len(schedule[b]) and schedule[b][rnd] > 0]
+            lens = [schedule[b][rnd] for b in ids]
+            if not ids:
+                continue
+            for l, (kind, W, owner) in enumerate(wl.layout):
+                q = torch.cat([si.q_tokens(wl.seed, l, b, pos[b], n, wl.n_q_heads, wl.head_dim, dt)
+                               for b, n in zip(ids, lens)])
+                kv = [si.kv_tokens(wl.seed, owner, b, pos[b], n, wl.n_kv_heads, wl.head_dim, dt)
+                      for b, n in zip(ids, lens)]
+                k, v = torch.cat([a for a, _ in kv]), torch.cat([c for _, c in kv])
+                out = torch.full_like(q, float("nan"), device="cuda")
+                sess.ctx.attend_chunk(l, ids, lens, q.cuda(), k.cuda(), v.cuda(), out)
+                torch.cuda.synchronize()
+                got = out.float().cpu().double().numpy()
+                row = 0
+                for b, n in zip(ids, lens):
+                    # the checker gets the whole history regenerated from the seed
+                    Kh, Vh = si.kv_tokens(wl.seed, owner, b, 0, pos[b] + n, wl.n_kv_heads, wl.head_dim, dt)
+                    rows = None
+                    if rows_per_chunk is not None and n > rows_per_chunk:
+                        rows = sorted(set(np.linspace(0, n - 1, rows_per_chunk).astype(int).tolist()))
+                    ref = mo.prefill_attention(q[row:row + n], Kh, Vh, kind, W, prefix_len=pos[b], rows=rows)
+                    g = got[row:row + n] if rows is None else got[row:row + n][rows]
+                    check_close(g, ref, wl.dtype, f"round {rnd} layer {l} seq {b} prefix {pos[b]} chunk {n}")
+                    row += n
+            # every layer has seen the chunk: now the owners store it
+            for o in cf.owners_of(wl.layout):
+                kv = [si.kv_tokens(wl.seed, o, b, pos[b], n, wl.n_kv_heads, wl.head_dim, dt)
+                      for b, n in zip(ids, lens)]
+                k, v = torch.cat([a for a, _ in kv]).cuda(), torch.cat([c for _, c in kv]).cuda()
+                sess.ctx.append_kv(o, ids, lens, k, v)
+                ph.append(o, ids, lens)
+            for b, n in zip(ids, lens):
+                pos[b] += n
+            torch.cuda.synchronize()
+            compare_state(sess.ctx, ph, wl)
+        assert sess.ctx.get_device_status() == 0
+        sess.pos[:] = pos
+        for l, (kind, W, owner) in enumerate(wl.layout):
+            for b in range(B):
+                lo = 0 if kind == cf.FULL else max(0, pos[b] - W)
+                check_stored_bits(sess.ctx, ph, wl, l, b, sorted({lo, pos[b] - 1, (lo + pos[b]) // 2}))
+        inputs = sess.step_inputs()
+        outs = sess.alloc_outputs()
+        sess.decode_step(inputs, outs)
+        torch.cuda.synchronize()
+        got = outs.float().cpu().double().numpy()
+        for l in range(len(wl.layout)):
+            for b in range(B):
+                check_close(got[l, b], ref_decode(wl, l, b, pos[b] + 1), wl.dtype, f"decode after chunks {l}/{b}")
+    finally:
+        sess.close()
+
+
+def test_chunks_fp32_tiny_layout():
+    # window 64: chunks shorter than, equal to and longer than the window, single tokens, a
+    # sequence that joins late, and a scratch that only holds one sequence's keys at the end
+    wl = cf.tiny_decode().scaled(batch=3, context=0)
+    schedule = [[100, 1, 37, 64, 200, 1], [5, 64, 129, 3, 0, 70], [0, 0, 300, 1, 1, 33]]
+    run_chunked(wl, schedule, scratch=640)
+
+
+def test_chunks_bf16_tensor_core_path():
+    # head_dim 128, bf16: the tcgen05 kernel with a key prefix that is not a multiple of the
+    # tile (diagonal inside tiles), window 256 shared by a reader, several query tiles
+    wl = cf.prefill_chunk().scaled(layout=cf.layout_tiny(256), batch=2, seq_len=0)
+    schedule = [[300, 129, 1, 500, 77], [50, 700, 128, 4, 256]]
+    run_chunked(wl, schedule, scratch=2600)
+
+
+def test_chunks_bf16_mid_layout_sampled_rows():
+    # the 24-layer layout (two shared rings of 1024, one shared paged cache), longer prefixes
+    wl = cf.prefill_chunk().scaled(batch=2, seq_len=0)
+    schedule = [[1500, 1100, 130], [900, 2048, 1]]
+    run_chunked(wl, schedule, scratch=6000, rows_per_chunk=24)
+
+
+def test_chunk_errors():
+    mx, runner = load_lib()
+    wl = cf.tiny_decode().scaled(batch=2, context=0)
+    q = torch.zeros(8, wl.n_q_heads, wl.head_dim, device="cuda")
+    kv = torch.zeros(8, wl.n_kv_heads, wl.head_dim, device="cuda")
+    out = torch.full_like(q, 7.0)
+    sess = runner.Session(wl, [40, 40], headroom_tokens=2)                      # no scratch
+    try:
+        assert sess.ctx.rc_attend_chunk(0, [0], [8], q, kv, kv, out) == mx.ERR_UNSUPPORTED
+    finally:
+        sess.close()
+    sess = runner.Session(wl, [40, 40], headroom_tokens=2, chunk_scratch_tokens=16)
+    try:
+        sess.fill()
+        assert sess.ctx.rc_attend_chunk(0, [0], [2], q, kv, kv, out) == mx.ERR_TOO_LARGE   # 40 cached + 2 > 16
+        assert sess.ctx.rc_attend_chunk(1, [0], [2], q, kv, kv, out) == mx.ERR_TOO_LARGE   # ring (window 64): 40 + 2 too
+        assert sess.ctx.rc_attend_chunk(0, [0, 0], [1, 1], q, kv, kv, out) == mx.ERR_INVALID_ARG
+        assert sess.ctx.rc_attend_chunk(0, [0], [0], q, kv, kv, out) == mx.ERR_INVALID_ARG
+        assert sess.ctx.rc_attend_chunk(0, [2], [1], q, kv, kv, out) == mx.ERR_BAD_SEQ
+        assert sess.ctx.rc_attend_chunk(0, [0], [3], q, kv, kv, out) == mx.ERR_INVALID_ARG  # beyond max_seq_len
+        torch.cuda.synchronize()
+        assert (out == 7.0).all()
+        assert sess.ctx.get_len(0, 0) == 40                                             # nothing stored
+    finally:
+        sess.close()
