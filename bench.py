@@ -232,6 +232,46 @@ def prefill_figures(mx, runner, peaks, device):
     return res
 
 
+def chunk_figures(mx, runner, peaks, device, prefix=6144, chunk=2048):
+    """The last chunk of the prefill configuration's prompts served in chunks: `chunk` new
+    tokens per sequence behind `prefix` cached ones (gather of the cached keys + attention)."""
+    wl = cf.prefill_chunk().scaled(seq_len=0)
+    B, D, Hq, W = wl.batch, wl.head_dim, wl.n_q_heads, 1024
+    sess = runner.Session(wl, [prefix] * B, device=device, headroom_tokens=chunk,
+                          chunk_scratch_tokens=B * (prefix + chunk))
+    res = {}
+    try:
+        sess.fill(2048)
+        ids, lens = list(range(B)), [chunk] * B
+        pairs_full = sum(prefix + r + 1 for r in range(chunk))
+        pairs_slide = sum(min(prefix + r + 1, W) for r in range(chunk))
+        for name, layer, pairs, cls in (("full", 12, pairs_full, mx.K_PREFILL_FULL),
+                                        ("sliding", 2, pairs_slide, mx.K_PREFILL_SLIDING)):
+            owner = wl.layout[layer][2]
+            q = si.q_tokens_multi(wl.seed, layer, ids, [prefix] * B, chunk, Hq, D, sess.dt,
+                                  sess.dev).reshape(-1, Hq, D)
+            K, V = si.kv_tokens_multi(wl.seed, owner, ids, [prefix] * B, chunk, wl.n_kv_heads, D, sess.dt, sess.dev)
+            K, V = K.reshape(-1, wl.n_kv_heads, D), V.reshape(-1, wl.n_kv_heads, D)
+            out = torch.empty_like(q)
+            reps = 3
+            sess.ctx.attend_chunk(layer, ids, lens, q, K, V, out)
+            torch.cuda.synchronize()
+            sess.ctx.profile_enable(True)
+            for _ in range(reps):
+                sess.ctx.attend_chunk(layer, ids, lens, q, K, V, out)
+            n, ms = sess.ctx.profile_read(cls)
+            ng, msg = sess.ctx.profile_read(mx.K_GATHER)
+            sess.ctx.profile_enable(False)
+            flops = 4.0 * D * pairs * Hq * B
+            t = (ms / n + msg / ng) * 1e-3
+            res[name] = {"ms_attention": ms / n, "ms_gather": msg / ng, "tflops": flops / t / 1e12,
+                         "frac_of_bf16_peak": flops / t / 1e12 / peaks["bf16_tflops"], "useful_flop": flops}
+        res["config"] = {"workload": wl.name, "batch": B, "cached_prefix": prefix, "chunk": chunk, "window": W}
+    finally:
+        sess.close()
+    return res
+
+
 def reduce_over_ranks(dist, times, work, device):
     """Replicas-only aggregation: times -> max over ranks, work -> sum over ranks.
     (No data-path collective exists; this is the only communication of a run.)"""
@@ -403,6 +443,7 @@ def run_gpu_arm(args, wl):
     if not args.no_prefill:
         sess.close()
         prefill = prefill_figures(mx, runner, peaks, local)
+        prefill["chunked"] = chunk_figures(mx, runner, peaks, local)
 
     line = {
         "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": K, "warmup": Wm,
