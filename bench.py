@@ -472,6 +472,36 @@ def run_gpu_arm(args, wl):
         dist.destroy_process_group()
 
 
+def run_trace_arm(args):
+    """Attention-only serving of requests shaped like the paper's benchmark (Section 5.4: prompts of
+    31000 tokens, then generated tokens; 12 query / 3 KV heads), one wave of concurrent requests, for
+    the standard layout (every layer its own full cache), MixAttention and its pairs variant."""
+    from paper_2409_15012_b200 import build as mbuild
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU path")
+    mbuild.build()
+    from paper_2409_15012_b200 import runner
+    torch.cuda.set_device(0)
+    layouts = {"standard (24 full caches)": cf.layout_all_full(24),
+               "mixattention (1 full cache + 2 shared rings)": cf.layout_mid(1024),
+               "mixattention pairs (1 full cache + 12 rings)": cf.layout_pairs(1024)}
+    res = {}
+    for name, lay in layouts.items():
+        res[name] = runner.serve_trace(lay, 12, 3, 128, args.trace_requests, args.trace_prompt, args.trace_gen, 2048)
+    base = res["standard (24 full caches)"]
+    ma = res["mixattention (1 full cache + 2 shared rings)"]
+    line = {"metric": "attention-only serving throughput on a paper-shaped trace", "value": ma["tokens_per_s"],
+            "unit": "tokens/s", "n_gpus": 1, "higher_is_better": True, "dtype": "bf16", "data": "synthetic",
+            "vs_baseline": None,
+            "config": {"workload": "serving_trace", "requests": args.trace_requests, "prompt_len": args.trace_prompt,
+                       "gen_len": args.trace_gen, "chunk": 2048, "heads": "12/3x128", "layers": 24, "window": 1024,
+                       "timing": "sum of the library's kernel times (CUDA events around every launch)"},
+            "speedup_over_standard_layout": ma["tokens_per_s"] / base["tokens_per_s"],
+            "cache_bytes_ratio_standard_over_mixattention": base["cache_bytes"] / ma["cache_bytes"],
+            "layouts": res}
+    print(json.dumps(line), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -484,6 +514,10 @@ def main():
                     help="override the batch size (smaller cases for profiler captures; not a bench value)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-prefill", action="store_true")
+    ap.add_argument("--trace", action="store_true", help="paper-shaped serving trace instead of the decode step")
+    ap.add_argument("--trace-requests", type=int, default=8)
+    ap.add_argument("--trace-prompt", type=int, default=31000)
+    ap.add_argument("--trace-gen", type=int, default=100)
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
@@ -492,6 +526,8 @@ def main():
         wl = wl.scaled(batch=args.batch, name=f"{wl.name}_batch{args.batch}")
     if args.impl == "reference":
         run_reference_arm(args, wl)
+    elif args.trace:
+        run_trace_arm(args)
     else:
         run_gpu_arm(args, wl)
 

@@ -122,6 +122,49 @@ class Session:
             self.pos += 1
 
     # ------------------------------------------------------------------
+    def prefill_in_chunks(self, chunk: int, stream=None):
+        """Serves what is left of every sequence's prompt (target - pos tokens) in rounds of at
+        most `chunk` tokens per sequence: every layer attends the round's chunk behind the cached
+        prefix (attend_chunk stores nothing), then every owner appends the round's K/V.  Returns
+        the last round's outputs [layers][rows, Hq, D] (sequences back to back)."""
+        wl = self.wl
+        B, Hq, Hkv, D = wl.batch, wl.n_q_heads, wl.n_kv_heads, wl.head_dim
+        outs = None
+        while ((self.target - self.pos) > 0).any():
+            ids = [b for b in range(B) if self.target[b] > self.pos[b]]
+            lens = [int(min(chunk, self.target[b] - self.pos[b])) for b in ids]
+            starts = [int(self.pos[b]) for b in ids]
+            same = len(set(lens)) == 1
+
+            def q_of(layer):
+                if same:
+                    return si.q_tokens_multi(wl.seed, layer, ids, starts, lens[0], Hq, D, self.dt,
+                                             self.dev).reshape(-1, Hq, D)
+                return torch.cat([si.q_tokens(wl.seed, layer, b, p0, n, Hq, D, self.dt, self.dev)
+                                  for b, p0, n in zip(ids, starts, lens)])
+
+            def kv_of(owner):
+                if same:
+                    K, V = si.kv_tokens_multi(wl.seed, owner, ids, starts, lens[0], Hkv, D, self.dt, self.dev)
+                    return K.reshape(-1, Hkv, D), V.reshape(-1, Hkv, D)
+                kv = [si.kv_tokens(wl.seed, owner, b, p0, n, Hkv, D, self.dt, self.dev)
+                      for b, p0, n in zip(ids, starts, lens)]
+                return torch.cat([a for a, _ in kv]), torch.cat([c for _, c in kv])
+
+            kv = {o: kv_of(o) for o in self.owners}
+            outs = []
+            for l, (_, _, owner) in enumerate(wl.layout):
+                q = q_of(l)
+                out = torch.empty_like(q)
+                self.ctx.attend_chunk(l, ids, lens, q, kv[owner][0], kv[owner][1], out, stream)
+                outs.append(out)
+            for o in self.owners:
+                self._append(o, ids, lens, kv[o][0], kv[o][1], stream)
+            for b, n in zip(ids, lens):
+                self.pos[b] += n
+        return outs
+
+    # ------------------------------------------------------------------
     def prefill_inputs(self, layer: int, device=None):
         """Packed Q, K, V of the prompts (length wl.seq_len each) for `layer`;
         K/V are the owner's."""
@@ -155,3 +198,37 @@ def kv_bytes_per_step(wl: cf.Workload, lengths_after: Sequence[int]) -> int:
         for n in lengths_after:
             total += (min(int(n), window) if kind == cf.SLIDING else int(n)) * per_tok
     return total
+
+
+def serve_trace(layout, n_q_heads: int, n_kv_heads: int, head_dim: int, n_requests: int, prompt_len: int,
+                gen_len: int, chunk: int, device: int = 0, seed: int = 7, dtype: int = cf.BF16) -> Dict:
+    """Attention-only serving of `n_requests` concurrent requests shaped like the paper's
+    benchmark (Section 5.4: long prompts, then generated tokens): the prompts in chunks
+    through attend_chunk + append_kv, then `gen_len` decode steps.  Times are the sums of the
+    library's own kernel times (its profile hooks), so input generation is excluded."""
+    wl = cf.Workload("serving_trace", list(layout), n_q_heads, n_kv_heads, head_dim, dtype, n_requests, 0, seed)
+    sess = Session(wl, [prompt_len] * n_requests, device=device, headroom_tokens=gen_len + 1,
+                   chunk_scratch_tokens=n_requests * (prompt_len + chunk))
+    try:
+        classes = (mx.K_APPEND, mx.K_DECODE_FULL, mx.K_DECODE_SLIDING, mx.K_COMBINE, mx.K_PREFILL_FULL,
+                   mx.K_PREFILL_SLIDING, mx.K_GATHER)
+        sess.ctx.profile_enable(True)
+        sess.prefill_in_chunks(chunk)
+        torch.cuda.synchronize(sess.dev)
+        prefill_ms = sum(sess.ctx.profile_read(c)[1] for c in classes)
+        outs = sess.alloc_outputs()
+        for _ in range(gen_len):
+            sess.decode_step(sess.step_inputs(), outs)
+        torch.cuda.synchronize(sess.dev)
+        decode_ms = sum(sess.ctx.profile_read(c)[1] for c in classes) - prefill_ms   # the records accumulate
+        sess.ctx.profile_enable(False)
+        status = sess.ctx.get_device_status()
+        cache = mx.cache_bytes(sess.ctx.cfg)
+    finally:
+        sess.close()
+    tokens = n_requests * (prompt_len + gen_len)
+    return {"requests": n_requests, "prompt_len": prompt_len, "gen_len": gen_len, "chunk": chunk,
+            "prefill_kernel_ms": prefill_ms, "decode_kernel_ms": decode_ms,
+            "tokens_per_s": tokens / ((prefill_ms + decode_ms) * 1e-3),
+            "decode_tokens_per_s": n_requests * gen_len / (decode_ms * 1e-3) if decode_ms > 0 else None,
+            "cache_bytes": cache, "device_status": status}

@@ -127,3 +127,41 @@ def test_chunk_errors():
         assert sess.ctx.get_len(0, 0) == 40                                             # nothing stored
     finally:
         sess.close()
+
+
+def test_serving_trace_small():
+    # prompts of different lengths served in chunks, then decode steps, through the runner's
+    # helpers; the cache state and the last step's outputs against the checker
+    mx, runner = load_lib()
+    wl = cf.mid_decode().scaled(layout=cf.layout_mid(128, 6), batch=3, context=0, n_q_heads=12, n_kv_heads=3)
+    prompts = [700, 333, 129]
+    sess = runner.Session(wl, prompts, headroom_tokens=6, chunk_scratch_tokens=3 * (700 + 256))
+    ph = mo.PhysicalCache(wl.layout, wl.n_kv_heads, wl.head_dim, wl.batch, sess.n_pages, store_values=False)
+    sess.mirror = ph
+    try:
+        outs = sess.prefill_in_chunks(256)
+        torch.cuda.synchronize()
+        compare_state(sess.ctx, ph, wl)
+        assert [int(p) for p in sess.pos] == prompts
+        # the last round held only sequence 0's final 188 tokens: check its last row in every layer
+        dt = torch_dt(wl.dtype)
+        for l, (kind, W, owner) in enumerate(wl.layout):
+            q = si.q_tokens(wl.seed, l, 0, 699, 1, wl.n_q_heads, wl.head_dim, dt)
+            Kh, Vh = si.kv_tokens(wl.seed, owner, 0, 0, 700, wl.n_kv_heads, wl.head_dim, dt)
+            ref = mo.prefill_attention(q, Kh, Vh, kind, W, prefix_len=699)
+            check_close(outs[l][-1:].float().cpu().double().numpy(), ref, wl.dtype, f"last prompt row, layer {l}")
+        got = None
+        for _ in range(5):
+            o = sess.alloc_outputs()
+            sess.decode_step(sess.step_inputs(), o)
+            got = o
+        torch.cuda.synchronize()
+        compare_state(sess.ctx, ph, wl)
+        g = got.float().cpu().double().numpy()
+        for l in range(len(wl.layout)):
+            for b in range(wl.batch):
+                check_close(g[l, b], ref_decode(wl, l, b, prompts[b] + 5), wl.dtype, f"decode {l}/{b}")
+        res = runner.serve_trace(wl.layout, 12, 3, 128, 2, 300, 3, 128)
+        assert res["device_status"] == 0 and res["prefill_kernel_ms"] > 0 and res["decode_kernel_ms"] > 0
+    finally:
+        sess.close()
