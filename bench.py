@@ -482,22 +482,23 @@ def run_trace_arm(args):
     mbuild.build()
     from paper_2409_15012_b200 import runner
     torch.cuda.set_device(0)
-    layouts = {"standard (24 full caches)": cf.layout_all_full(24),
-               "mixattention (1 full cache + 2 shared rings)": cf.layout_mid(1024),
-               "mixattention pairs (1 full cache + 12 rings)": cf.layout_pairs(1024)}
+    layouts = {"standard": cf.layout_all_full(24), "sliding_window": cf.layout_all_sliding(24, 1024),
+               "mid-decode layout (1 full cache + 2 shared rings)": cf.layout_mid(1024)}
+    for name in ("MA", "MA-EndSlide", "MA-Offset", "MA-Pairs", "MA-Offset-SlideShare", "MA-Pairs-SlideShare"):
+        layouts[name] = cf.PAPER_VARIANTS[name]()     # the paper's named variants (layer indices: see synth/configs.py)
     res = {}
     for name, lay in layouts.items():
         res[name] = runner.serve_trace(lay, 12, 3, 128, args.trace_requests, args.trace_prompt, args.trace_gen, 2048)
-    base = res["standard (24 full caches)"]
-    ma = res["mixattention (1 full cache + 2 shared rings)"]
+        res[name]["speedup_over_standard"] = res[name]["tokens_per_s"] / res["standard"]["tokens_per_s"]
+        res[name]["cache_bytes_vs_standard"] = res[name]["cache_bytes"] / res["standard"]["cache_bytes"]
+    ma = res["MA-Offset"]
     line = {"metric": "attention-only serving throughput on a paper-shaped trace", "value": ma["tokens_per_s"],
             "unit": "tokens/s", "n_gpus": 1, "higher_is_better": True, "dtype": "bf16", "data": "synthetic",
             "vs_baseline": None,
-            "config": {"workload": "serving_trace", "requests": args.trace_requests, "prompt_len": args.trace_prompt,
-                       "gen_len": args.trace_gen, "chunk": 2048, "heads": "12/3x128", "layers": 24, "window": 1024,
+            "config": {"workload": "serving_trace", "layout": "MA-Offset", "requests": args.trace_requests,
+                       "prompt_len": args.trace_prompt, "gen_len": args.trace_gen, "chunk": 2048, "heads": "12/3x128",
+                       "layers": 24, "window": 1024,
                        "timing": "sum of the library's kernel times (CUDA events around every launch)"},
-            "speedup_over_standard_layout": ma["tokens_per_s"] / base["tokens_per_s"],
-            "cache_bytes_ratio_standard_over_mixattention": base["cache_bytes"] / ma["cache_bytes"],
             "layouts": res}
     print(json.dumps(line), flush=True)
 

@@ -67,6 +67,107 @@ def owners_of(layout: List[Layer]) -> List[int]:
     return [l for l, (_, _, o) in enumerate(layout) if o == l]
 
 
+# ---------------------------------------------------------------------------
+# The paper's named variants (Section 4).  The text fixes, per variant, how many standard
+# attention caches there are, which layer computes them and who shares them; the figures
+# that drew the exact layer indices are not part of the text.  What the text leaves open is
+# a parameter here, with defaults that follow the pattern it cites (a standard layer every
+# sixth layer, sliding-window layers sharing a ring in groups of two or three).
+# ---------------------------------------------------------------------------
+
+def layout_from_roles(n_layers: int, window: int, full_layers, full_owner_of, ring_groups=(3, 2)) -> List[Layer]:
+    """Standard layers at `full_layers`, each reading the cache of full_owner_of[layer]
+    (itself = it computes its own); every run of sliding layers between them is cut into
+    ring-sharing groups of the sizes in `ring_groups`, repeated."""
+    full = set(full_layers)
+    out: List[Layer] = [None] * n_layers
+    group_start, group_left, gi = None, 0, 0
+    for l in range(n_layers):
+        if l in full:
+            out[l] = (FULL, 0, full_owner_of[l])
+            group_left = 0           # a standard layer ends the running ring group
+            continue
+        if group_left == 0:
+            group_start, group_left = l, ring_groups[gi % len(ring_groups)]
+            gi += 1
+        out[l] = (SLIDING, window, group_start)
+        group_left -= 1
+    return out
+
+
+def _every(n_layers: int, first: int, step: int):
+    return list(range(first, n_layers, step))
+
+
+def layout_ma(n_layers: int = 24, window: int = 1024, step: int = 6, ring_groups=(3, 2)) -> List[Layer]:
+    """MA: one standard cache, computed by the first layer; every other standard layer
+    (every `step`-th layer and the last one) reads it."""
+    full = sorted(set(_every(n_layers, 0, step) + [n_layers - 1]))
+    return layout_from_roles(n_layers, window, full, {l: 0 for l in full}, ring_groups)
+
+
+def layout_ma_endslide(n_layers: int = 24, window: int = 1024, step: int = 6, ring_groups=(3, 2)) -> List[Layer]:
+    """MA-EndSlide: MA with a sliding-window layer last."""
+    full = _every(n_layers, 0, step)
+    if full[-1] == n_layers - 1:
+        full = full[:-1]
+    return layout_from_roles(n_layers, window, full, {l: 0 for l in full}, ring_groups)
+
+
+def layout_ma_offset(n_layers: int = 24, window: int = 1024, offset: int = 2, step: int = 6,
+                     ring_groups=(3, 2)) -> List[Layer]:
+    """MA-Offset: the first standard layer (which computes the one standard cache) sits
+    `offset` layers in, after a few sliding-window layers."""
+    full = sorted(set(_every(n_layers, offset, step) + [n_layers - 1]))
+    return layout_from_roles(n_layers, window, full, {l: offset for l in full}, ring_groups)
+
+
+def layout_ma_pairs(n_layers: int = 24, window: int = 1024, reader_distance: int = 6, ring_groups=(3, 2)) -> List[Layer]:
+    """MA-Pairs: two standard caches, computed at the first and the thirteenth layer, each
+    shared with one more standard layer `reader_distance` layers later."""
+    a, b = 0, 12
+    own = {a: a, a + reader_distance: a, b: b, min(b + reader_distance, n_layers - 1): b}
+    return layout_from_roles(n_layers, window, sorted(own), own, ring_groups)
+
+
+def layout_slideshare(base: List[Layer]) -> List[Layer]:
+    """-SlideShare: more sharing among the sliding-window layers: every run of sliding layers
+    between two standard layers shares one ring."""
+    out: List[Layer] = []
+    run_owner = None
+    for l, (kind, w, owner) in enumerate(base):
+        if kind == FULL:
+            out.append((kind, w, owner))
+            run_owner = None
+        else:
+            if run_owner is None:
+                run_owner = l
+            out.append((kind, w, run_owner))
+    return out
+
+
+def layout_noshare(n_layers: int = 24, window: int = 1024, n_full: int = 1, offset: int = 0, step: int = 6,
+                   ring_groups=(3, 2)) -> List[Layer]:
+    """MA-NoShare-k: k standard layers, each with a cache of its own (no standard cache is shared)."""
+    full = _every(n_layers, offset, step)[:n_full]
+    return layout_from_roles(n_layers, window, full, {l: l for l in full}, ring_groups)
+
+
+PAPER_VARIANTS = {
+    "standard": lambda: layout_all_full(24),
+    "sliding_window": lambda: layout_all_sliding(24, 1024),
+    "MA": layout_ma,
+    "MA-EndSlide": layout_ma_endslide,
+    "MA-Offset": layout_ma_offset,
+    "MA-Pairs": layout_ma_pairs,
+    "MA-Offset-SlideShare": lambda: layout_slideshare(layout_ma_offset()),
+    "MA-Pairs-SlideShare": lambda: layout_slideshare(layout_ma_pairs()),
+    "MA-NoShare-1": lambda: layout_noshare(n_full=1),
+    "MA-NoShare-2": lambda: layout_noshare(n_full=2, offset=2, step=12),
+    "MA-NoShare-3": lambda: layout_noshare(n_full=3, offset=2, step=8),
+}
+
+
 @dataclass(frozen=True)
 class Workload:
     name: str

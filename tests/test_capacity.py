@@ -33,3 +33,42 @@ def test_capacity_matches_closed_form_and_sharing_law():
     # one shared full cache instead of 24 private ones: 1/24 of the full-attention bytes
     assert tab["standard"][0] == 24 * (tab["mix"][0] - 2 * W * per_tok)
     assert tab["mix"][1] > 20 * tab["standard"][1]
+
+
+def test_named_variants_have_the_properties_the_paper_states():
+    # Section 4 fixes these facts in words; the exact layer indices (figures) are parameters
+    V = {k: f() for k, f in cf.PAPER_VARIANTS.items()}
+    for name, lay in V.items():
+        assert len(lay) == 24
+        mo.validate_layout(lay)
+        ctx = mx.Context(lay, 12, 3, 128, mx.BF16, 2, 8, device=-1)      # the library accepts it too
+        ctx.close()
+    full_owners = lambda lay: [l for l, (k, _, o) in enumerate(lay) if k == cf.FULL and o == l]
+    full_layers = lambda lay: [l for l, (k, _, o) in enumerate(lay) if k == cf.FULL]
+    # MA: a single standard cache, the first layer's; all other standard layers share it
+    assert full_owners(V["MA"]) == [0] and len(full_layers(V["MA"])) > 2
+    assert V["MA"][23][0] == cf.FULL
+    # MA-EndSlide: the same, but the last layer is a sliding-window layer
+    assert full_owners(V["MA-EndSlide"]) == [0] and V["MA-EndSlide"][23][0] == cf.SLIDING
+    assert full_layers(V["MA-EndSlide"]) == [l for l in full_layers(V["MA"]) if l != 23]
+    # MA-Offset: one standard cache, computed a few layers in, after sliding-window layers
+    off = full_owners(V["MA-Offset"])
+    assert len(off) == 1 and off[0] > 0 and all(V["MA-Offset"][l][0] == cf.SLIDING for l in range(off[0]))
+    # MA-Pairs: two standard caches, at the first and the thirteenth layer, each shared with one more layer
+    assert full_owners(V["MA-Pairs"]) == [0, 12]
+    for o in (0, 12):
+        assert sum(1 for l, (k, _, ow) in enumerate(V["MA-Pairs"]) if k == cf.FULL and ow == o and l != o) == 1
+    # -SlideShare: strictly fewer rings than the base variant, same standard layers
+    rings = lambda lay: len([l for l, (k, _, o) in enumerate(lay) if k == cf.SLIDING and o == l])
+    for base in ("MA-Offset", "MA-Pairs"):
+        assert rings(V[base + "-SlideShare"]) < rings(V[base])
+        assert full_layers(V[base + "-SlideShare"]) == full_layers(V[base])
+    # NoShare-k: k standard layers, none shared
+    for k in (1, 2, 3):
+        lay = V[f"MA-NoShare-{k}"]
+        assert full_owners(lay) == full_layers(lay) and len(full_layers(lay)) == k
+    # cache bytes: every MixAttention variant is far below the standard model at 32K tokens
+    tab = capacity.capacity_table(V, 12, 3, 128, mx.BF16, 32000, 80 * 10**9)
+    for name in V:
+        if name.startswith("MA"):
+            assert tab[name][0] * 5 < tab["standard"][0]
