@@ -354,22 +354,71 @@ def run_gpu_arm(args, wl):
     assert sess.ctx.get_device_status() == 0, "a kernel reported a wait time-out"
 
     # ---- end-to-end pass: host inputs, host outputs ----
-    host_inputs = []
+    # Each step's inputs sit in one pinned host buffer and travel in two pieces on a copy
+    # stream (the first layers' inputs, then the rest, while the first layers already run);
+    # the outputs go back in pieces on a third stream while later layers run (only the last
+    # layer's output is copied after the step's last kernel).  Every step ends with a host wait for its complete result.
     pos_save = sess.pos.copy()
+    n_layers = len(wl.layout)
+    order = [(l, k) for l in range(n_layers) for k in ("q", "k", "v") if k in step_inputs[0][l]]
+    offs, total = {}, 0
+    for l, k in order:
+        t = step_inputs[0][l][k]
+        offs[(l, k)] = total
+        total += -(-t.numel() * t.element_size() // 256) * 256
+    cut_layer = 2                                          # layers before this one travel first
+    cut = offs[(cut_layer, "q")]
+    host_flat = [torch.empty(total, dtype=torch.uint8).pin_memory() for _ in range(kRing)]
+    dev_flat = torch.empty(total, dtype=torch.uint8, device=sess.dev)
+
+    def views(flat):
+        out = {}
+        for l, k in order:
+            t = step_inputs[0][l][k]
+            n = t.numel() * t.element_size()
+            out.setdefault(l, {})[k] = flat[offs[(l, k)]:offs[(l, k)] + n].view(t.dtype).view(t.shape)
+        return out
+
     for s in range(kRing):
-        host_inputs.append({l: {k: t.cpu().pin_memory() for k, t in d.items()} for l, d in step_inputs[s].items()})
-    dev_buf = {l: {k: torch.empty_like(t, device=sess.dev) for k, t in d.items()} for l, d in host_inputs[0].items()}
+        hv = views(host_flat[s])
+        for l, k in order:
+            hv[l][k].copy_(step_inputs[s][l][k])
+    dev_buf = views(dev_flat)
     host_out = torch.empty(outs.shape, dtype=outs.dtype).pin_memory()
-    h2d = sum(t.numel() * t.element_size() for d in host_inputs[0].values() for t in d.values())
+    h2d = sum(t.numel() * t.element_size() for d in step_inputs[0].values() for t in d.values())
     d2h = outs.numel() * outs.element_size()
+    h2d_stream, d2h_stream = torch.cuda.Stream(device=sess.dev), torch.cuda.Stream(device=sess.dev)
+    ev_in = [torch.cuda.Event() for _ in range(2)]
+    d2h_cuts = sorted({n_layers // 2, (5 * n_layers) // 6, n_layers - 1} - {0, n_layers})   # outputs leave in pieces
+    ev_out = [torch.cuda.Event() for _ in d2h_cuts]
+    ids_all = list(range(wl.batch))
 
     def e2e_step(s):
-        for l, d in host_inputs[s % kRing].items():
-            for k, t in d.items():
-                dev_buf[l][k].copy_(t, non_blocking=True)
-        sess.decode_step(dev_buf, outs, stream)
-        host_out.copy_(outs, non_blocking=True)
+        src = host_flat[s % kRing]
+        with torch.cuda.stream(h2d_stream):
+            dev_flat[:cut].copy_(src[:cut], non_blocking=True)
+            ev_in[0].record(h2d_stream)
+            dev_flat[cut:].copy_(src[cut:], non_blocking=True)
+            ev_in[1].record(h2d_stream)
+        for l in range(n_layers):
+            if l == 0 or l == cut_layer:
+                stream.wait_event(ev_in[0 if l == 0 else 1])
+            ent = dev_buf[l]
+            if "k" in ent:
+                sess.ctx.append_kv(l, ids_all, None, ent["k"], ent["v"], stream)
+            sess.ctx.decode(l, ids_all, ent["q"], outs[l], stream)
+            if l + 1 in d2h_cuts:
+                i = d2h_cuts.index(l + 1)
+                lo = d2h_cuts[i - 1] if i > 0 else 0
+                ev_out[i].record(stream)
+                d2h_stream.wait_event(ev_out[i])
+                with torch.cuda.stream(d2h_stream):
+                    host_out[lo:l + 1].copy_(outs[lo:l + 1], non_blocking=True)
+        sess.pos += 1
+        with torch.cuda.stream(stream):
+            host_out[d2h_cuts[-1]:].copy_(outs[d2h_cuts[-1]:], non_blocking=True)
         stream.synchronize()
+        d2h_stream.synchronize()
 
     for s in range(Wm):
         e2e_step(s)
