@@ -16,6 +16,8 @@ namespace {
 constexpr size_t kAlign = 256;
 constexpr int kSplitTokens = 4096;    // automatic split length of long caches (keys)
 constexpr int kMinSplitTokens = 1024; // single-wave splitting never makes splits shorter than this
+constexpr double kL2FitsShare = 0.55;  // a re-read ring up to this share of the L2 is cached whole
+constexpr double kL2KeepShare = 0.45;  // of a larger one, this share of the L2 is kept
 
 inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
@@ -80,6 +82,7 @@ struct mixattn_ctx {
   bool host_only = true;
   int device = -1;
   int sm_count = 148;
+  int64_t l2_bytes = 0;
   float scale = 0.f;
   int32_t split_tokens = 0;
   int64_t launches = 0;
@@ -270,6 +273,7 @@ int mixattn_create(const mixattn_config* cfg, mixattn_ctx** out) {
     cudaDeviceProp prop;
     if (!g.ok || cudaGetDeviceProperties(&prop, c->device) != cudaSuccess) { delete c; return MIXATTN_ERR_CUDA; }
     c->sm_count = prop.multiProcessorCount;
+    c->l2_bytes = prop.l2CacheSize;
     if (prepare_decode_bf16() != cudaSuccess || prepare_prefill_tc() != cudaSuccess) { delete c; return MIXATTN_ERR_CUDA; }
     if (cudaMemsetAsync(c->arena, 0, c->plan.total, 0) != cudaSuccess ||
         cudaStreamSynchronize(0) != cudaSuccess) {
@@ -325,6 +329,28 @@ int mixattn_append_kv(mixattn_ctx* c, int32_t layer, int32_t n_seqs, const int32
                         static_cast<cudaStream_t>(stream));
 }
 
+// L2 policy of a decode launch (see l2_policy_of in decode_bf16.cu).  Only a ring that a later
+// layer reads again (Section 3's cache sharing makes consecutive layers read the same bytes) is
+// worth keeping: the leading part of its storage, up to a share of the L2 that a cyclic scan was
+// measured to keep resident.  The last layer that reads the ring lets go of it.
+static void set_l2_policy(const mixattn_ctx* c, int layer, DecodeParams* p) {
+  p->l2_keep_bytes = 0;
+  p->l2_pool_bytes = 0;
+  const LayerInfo& li = c->cm.layer(layer);
+  if (li.kind != MIXATTN_SLIDING || c->l2_bytes <= 0) return;
+  bool read_again = false;
+  for (int l = layer + 1; l < c->cfg.n_layers; ++l) read_again = read_again || c->cm.layer(l).owner == li.owner;
+  if (!read_again) return;
+  const uint64_t pool = c->plan.owner_bytes[li.owner_slot];
+  // (measured on a 126 MB L2: a 67 MB ring stays resident under plain LRU, a 134 MB ring does not
+  // at all; keeping 0.4-0.5 of the L2 of it gave the shortest step)
+  const uint64_t fits = (uint64_t)(kL2FitsShare * (double)c->l2_bytes);
+  const uint64_t room = (uint64_t)(kL2KeepShare * (double)c->l2_bytes);
+  const uint64_t window = pool < 0xFFFFFF00ull ? pool : 0xFFFFFF00ull;   // the policy's sizes are 32-bit
+  p->l2_pool_bytes = (uint32_t)window;
+  p->l2_keep_bytes = (uint32_t)(window <= fits ? window : room);
+}
+
 int mixattn_decode(mixattn_ctx* c, int32_t layer, int32_t n_seqs, const int32_t* seq_ids,
                    const void* q, void* out, void* stream) {
   if (c == nullptr || !c->cm.valid_layer(layer) || n_seqs < 0) return MIXATTN_ERR_INVALID_ARG;
@@ -359,6 +385,7 @@ int mixattn_decode(mixattn_ctx* c, int32_t layer, int32_t n_seqs, const int32_t*
   p.part_o = reinterpret_cast<float*>(c->arena + c->plan.part_o_off);
   p.part_ml = reinterpret_cast<float2*>(c->arena + c->plan.part_ml_off);
   p.status = c->dev_status();
+  set_l2_policy(c, layer, &p);
 
   for (int i0 = 0; i0 < n_seqs; i0 += kMaxCallSeqs) {
     const int nb = n_seqs - i0 < kMaxCallSeqs ? n_seqs - i0 : kMaxCallSeqs;
@@ -839,6 +866,7 @@ int mixattn_decode_static_scratch(mixattn_ctx* c, int32_t layer, int32_t n_seqs,
   p.geom = c->geom;
   p.n_q_heads = Hq;
   p.scale_log2e = c->scale * 1.4426950408889634f;
+  set_l2_policy(c, layer, &p);
   // every partial slot that the combine pass reads is written by the split pass of the
   // same call first, so nothing in the array has to start at zero
   p.part_o = reinterpret_cast<float*>(scratch);

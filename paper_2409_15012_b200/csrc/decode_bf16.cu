@@ -75,11 +75,25 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     }
   }
 }
-__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar,
+                                         uint64_t l2_policy) {
   asm volatile(
-      "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
-      "l"(src), "r"(bytes), "r"(bar)
+      "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
+      ::"r"(dst), "l"(src), "r"(bytes), "r"(bar), "l"(l2_policy)
       : "memory");
+}
+// L2 eviction policy of a launch's K/V stream.  A ring shared by several layers is read again
+// by the next launch, but a plain LRU keeps nothing of a cyclic scan larger than the cache: the
+// leading part of the ring storage (as much as fits the L2) is cached normally and the rest,
+// like a paged cache that is read once per step, is marked evict-first so that it passes through.
+__device__ __forceinline__ uint64_t l2_policy_of(const char* pool, uint32_t keep_bytes, uint32_t pool_bytes) {
+  uint64_t pol;
+  if (keep_bytes > 0)
+    asm volatile("createpolicy.range.global.L2::evict_normal.L2::evict_first.b64 %0, [%1], %2, %3;"
+                 : "=l"(pol) : "l"(pool), "r"(keep_bytes), "r"(pool_bytes));
+  else
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+  return pol;
 }
 __device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2,
                                         uint32_t& r3) {
@@ -199,6 +213,7 @@ decode_split_bf16_kernel(const __grid_constant__ DecodeParams p, const int n_sta
     // ------------------------------ producer ------------------------------
     int K = 0;  // tiles issued by this CTA so far
     bool ok = true;
+    const uint64_t l2_policy = l2_policy_of(p.pool, p.l2_keep_bytes, p.l2_pool_bytes);
     for (int it = blockIdx.x; ok && it < p.total_items; it += gridDim.x) {
       const Item x = decode_item(p, it);
       const int seq = p.seq_id[x.i];
@@ -230,7 +245,7 @@ decode_split_bf16_kernel(const __grid_constant__ DecodeParams p, const int n_sta
           const int64_t phys = tbl ? (int64_t)my_id : ring_page0 + pg + lane;
           const char* src = p.pool + phys * ge.page_bytes + (int64_t)x.g * kBlkBytes;
           bulk_g2s(smem_u32(stages + (size_t)s * kStageBytes + lane * kBlkBytes), src, kBlkBytes,
-                   full0 + 8 * s);
+                   full0 + 8 * s, l2_policy);
         }
       }
     }

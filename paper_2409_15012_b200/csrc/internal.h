@@ -93,6 +93,9 @@ struct DecodeParams {
   int32_t group;          // query heads per KV head
   int32_t head_chunks;    // ceil(group / 8)
   float scale_log2e;      // softmax scale * log2(e)
+  uint32_t l2_keep_bytes; // leading bytes of `pool` whose lines are cached normally (a ring that later
+  uint32_t l2_pool_bytes; // layers re-read); the rest of the pool's l2_pool_bytes, and everything when
+                          // l2_keep_bytes is 0, is marked evict-first (read once)
   float* part_o;          // [chunks, Hq, D] unnormalised partial outputs
   float2* part_ml;        // [chunks, Hq] running max (log2 units) and sum
   int32_t* status;        // device error word (0 = fine)
