@@ -149,3 +149,45 @@ def test_prefill_full_size_sampled_rows():
             check_stored_bits(sess.ctx, ph, wl, l, 2, [lo, (lo + S) // 2, S - 1])
     finally:
         sess.close()
+
+
+def test_prefill_served_in_chunks_full_size_sampled_rows():
+    # the prefill configuration's prompts (batch 4 x 8192) served in chunks of 2048 behind the cached
+    # prefix, in the launch configuration bench.py times; sampled rows of sampled heads per round
+    mx, runner = load_lib()
+    wl = cf.prefill_chunk().scaled(seq_len=0)
+    S, C, W = 8192, 2048, 1024
+    sess = runner.Session(wl, [S] * wl.batch, headroom_tokens=1, chunk_scratch_tokens=wl.batch * S)
+    ph = mo.PhysicalCache(wl.layout, wl.n_kv_heads, wl.head_dim, wl.batch, sess.n_pages, store_values=False)
+    sess.mirror = ph
+    G = wl.n_q_heads // wl.n_kv_heads
+    hist = HeadHistory(wl)
+    rng = np.random.default_rng(wl.seed + 1)
+    dt = torch_dt(wl.dtype)
+    try:
+        for rnd in range(S // C):
+            P = rnd * C
+            sess.target[:] = P + C
+            outs = sess.prefill_in_chunks(C)
+            torch.cuda.synchronize()
+            rows = sorted({0, 1, 127, 128, C - 1} | set(int(x) for x in rng.integers(0, C, 8)))
+            for l in (0, 1, 12, 13, 23):
+                kind, Wl, owner = wl.layout[l]
+                got = outs[l].view(wl.batch, C, wl.n_q_heads, wl.head_dim)
+                for b, h in ((0, 1), (wl.batch - 1, 30)):
+                    K, V = hist.get(owner, b, h // G, S)
+                    qc = si.q_tokens(wl.seed, l, b, P, C, wl.n_q_heads, wl.head_dim, dt)[:, h].double().numpy()
+                    ref = np.empty((len(rows), wl.head_dim))
+                    for a, i in enumerate(rows):
+                        lo, hi = mo.key_range(kind, Wl, P + i)
+                        ref[a] = mo.softmax_attend(qc[i], K[lo:hi], V[lo:hi], 1.0 / np.sqrt(wl.head_dim))
+                    g = got[b, rows, h].float().cpu().double().numpy()
+                    check_close(g, ref, wl.dtype, f"round {rnd} layer {l} seq {b} head {h}")
+        assert sess.ctx.get_device_status() == 0
+        compare_state(sess.ctx, ph, wl)
+        for l in (0, 1, 13):
+            kind, Wl, _ = wl.layout[l]
+            lo = 0 if kind == cf.FULL else S - Wl
+            check_stored_bits(sess.ctx, ph, wl, l, 2, [lo, (lo + S) // 2, S - 1])
+    finally:
+        sess.close()
