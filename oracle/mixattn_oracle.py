@@ -94,6 +94,24 @@ def key_range(kind: int, window: int, i: int) -> Tuple[int, int]:
     return lo, hi
 
 
+def rope_rotate(x, positions, theta: float) -> np.ndarray:
+    """Rotary position embedding as defined by the RoFormer paper the method cites
+    (Section 4: "We used RoPE positional embeddings"): channel pairs (2i, 2i+1) of a
+    head vector at position m are rotated by the angle m * theta^(-2i/d).
+
+    x [n, heads, d] (d even), positions [n] integers.  float64 throughout."""
+    x = _as64(x)
+    n, _, d = x.shape
+    pos = np.asarray(positions, dtype=np.float64).reshape(n, 1, 1)
+    i = np.arange(d // 2, dtype=np.float64).reshape(1, 1, d // 2)
+    ang = pos * np.power(float(theta), -2.0 * i / d)
+    c, s = np.cos(ang), np.sin(ang)
+    out = np.empty_like(x)
+    out[..., 0::2] = x[..., 0::2] * c - x[..., 1::2] * s
+    out[..., 1::2] = x[..., 0::2] * s + x[..., 1::2] * c
+    return out
+
+
 # --------------------------------------------------------------------------
 # logical half: attention by definition, float64
 # --------------------------------------------------------------------------

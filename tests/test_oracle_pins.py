@@ -394,3 +394,43 @@ def test_chunk_needs_every_key_up_to_its_last_query():
     q, K = rnd(rng, 3, 2, 4), rnd(rng, 9, 2, 4)
     with pytest.raises(mo.OracleError):
         mo.prefill_attention(q, K, K, FULL, 0, prefix_len=5)
+
+
+# --------------------------------------------------------------------------
+# rotary position embedding
+# --------------------------------------------------------------------------
+
+def test_rope_is_complex_multiplication_by_unit_phases():
+    # the same definition written with complex numbers: (x_2i + j x_2i+1) * exp(j m theta^(-2i/d))
+    rng = np.random.default_rng(3)
+    n, H, d, theta = 9, 2, 16, 10000.0
+    x = rnd(rng, n, H, d)
+    pos = np.array([0, 1, 2, 7, 100, 4095, 31999, 131071, 5])
+    z = x[..., 0::2] + 1j * x[..., 1::2]
+    freq = theta ** (-np.arange(0, d, 2) / d)
+    zr = z * np.exp(1j * pos[:, None, None] * freq[None, None, :])
+    got = mo.rope_rotate(x, pos, theta)
+    np.testing.assert_allclose(got[..., 0::2], zr.real, rtol=0, atol=1e-9)
+    np.testing.assert_allclose(got[..., 1::2], zr.imag, rtol=0, atol=1e-9)
+
+
+def test_rope_closed_forms_and_relative_position_property():
+    rng = np.random.default_rng(4)
+    d, theta = 8, 500000.0
+    q, k = rnd(rng, 1, 1, d), rnd(rng, 1, 1, d)
+    # position 0 is the identity; the first pair turns by exactly m radians (theta^0 = 1)
+    np.testing.assert_allclose(mo.rope_rotate(q, [0], theta), q, rtol=0, atol=0)
+    e = np.zeros((1, 1, d)); e[0, 0, 0] = 1.0
+    r = mo.rope_rotate(e, [3], theta)
+    assert abs(r[0, 0, 0] - math.cos(3.0)) < 1e-15 and abs(r[0, 0, 1] - math.sin(3.0)) < 1e-15
+    # the last pair turns by m * theta^(-(d-2)/d)
+    e = np.zeros((1, 1, d)); e[0, 0, d - 2] = 1.0
+    r = mo.rope_rotate(e, [1000], theta)
+    a = 1000.0 * theta ** (-(d - 2) / d)
+    assert abs(r[0, 0, d - 2] - math.cos(a)) < 1e-12 and abs(r[0, 0, d - 1] - math.sin(a)) < 1e-12
+    # norms of pairs are kept; scores depend on the position difference only
+    for m, n_ in ((5, 2), (1000, 997), (70000, 69997)):
+        qm, kn = mo.rope_rotate(q, [m], theta), mo.rope_rotate(k, [n_], theta)
+        np.testing.assert_allclose(np.hypot(qm[..., 0::2], qm[..., 1::2]), np.hypot(q[..., 0::2], q[..., 1::2]), atol=1e-12)
+        ref = float((mo.rope_rotate(q, [m - n_], theta) * k).sum())
+        assert abs(float((qm * kn).sum()) - ref) < 1e-9
