@@ -126,6 +126,19 @@ int mixattn_seq_reset(mixattn_ctx* ctx, int32_t seq);
 int mixattn_append_kv(mixattn_ctx* ctx, int32_t layer, int32_t n_seqs, const int32_t* seq_ids,
                       const int32_t* n_new, const void* k, const void* v, void* stream);
 
+/* mixattn_append_kv with the rotary position embedding fused into the copy
+ * (Section 4: the models use RoPE, with a base theta that grows with the
+ * context length; the embedding is RoFormer's): before a key row is stored,
+ * its channel pairs (2i, 2i+1) are rotated by the angle t * theta^(-2i/d),
+ * t the token's position in the sequence and d = head_dim.  Values are stored
+ * unchanged.  Angles are reduced in double precision, the rotation runs in
+ * fp32 and bf16 rows are rounded once.  (Queries are the caller's: they are
+ * never stored.)  rope_theta must be finite and > 1, else INVALID_ARG; all
+ * else as mixattn_append_kv. */
+int mixattn_append_kv_rope(mixattn_ctx* ctx, int32_t layer, int32_t n_seqs, const int32_t* seq_ids,
+                           const int32_t* n_new, const void* k, const void* v, float rope_theta,
+                           void* stream);
+
 /* One decode step of `layer` for n_seqs sequences (Section 3).  With n the
  * number of tokens in the cache the layer reads (its owner's, after this
  * step's append) the query sits at position n-1 and attends to keys

@@ -72,6 +72,7 @@ def _load() -> C.CDLL:
         "mixattn_destroy": [vp],
         "mixattn_seq_reset": [vp, i32],
         "mixattn_append_kv": [vp, i32, i32, p32, p32, vp, vp, vp],
+        "mixattn_append_kv_rope": [vp, i32, i32, p32, p32, vp, vp, C.c_float, vp],
         "mixattn_decode": [vp, i32, i32, p32, vp, vp, vp],
         "mixattn_decode_static_scratch": [vp, i32, i32, p32, vp, vp, vp],
         "mixattn_attend_chunk": [vp, i32, i32, p32, p32, vp, vp, vp, vp, vp],
@@ -100,7 +101,7 @@ def _load() -> C.CDLL:
 lib = _load()
 EXPORTS = [
     "mixattn_arena_bytes", "mixattn_cache_bytes", "mixattn_create", "mixattn_destroy",
-    "mixattn_seq_reset", "mixattn_append_kv", "mixattn_decode", "mixattn_decode_static_scratch", "mixattn_prefill",
+    "mixattn_seq_reset", "mixattn_append_kv", "mixattn_append_kv_rope", "mixattn_decode", "mixattn_decode_static_scratch", "mixattn_prefill",
     "mixattn_attend_chunk",
     "mixattn_get_len", "mixattn_get_block_table", "mixattn_get_n_free_pages",
     "mixattn_get_ring_state", "mixattn_locate", "mixattn_debug_read_kv",
@@ -216,6 +217,17 @@ class Context:
         rc = self.rc_append_kv(layer, seq_ids, n_new, k, v, stream)
         if rc:
             raise MixAttnError(rc, "mixattn_append_kv")
+
+    def rc_append_kv_rope(self, layer, seq_ids, n_new, k, v, rope_theta, stream=None) -> int:
+        s = _i32(seq_ids)
+        n = None if n_new is None else _i32(n_new)
+        return lib.mixattn_append_kv_rope(self.h, layer, len(s), _p32(s), _p32(n), _dev(k), _dev(v),
+                                          float(rope_theta), _stream(stream))
+
+    def append_kv_rope(self, layer, seq_ids, n_new, k, v, rope_theta, stream=None):
+        rc = self.rc_append_kv_rope(layer, seq_ids, n_new, k, v, rope_theta, stream)
+        if rc:
+            raise MixAttnError(rc, "mixattn_append_kv_rope")
 
     def rc_decode(self, layer, seq_ids, q, out, stream=None) -> int:
         s = _i32(seq_ids)

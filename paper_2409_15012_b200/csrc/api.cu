@@ -156,7 +156,7 @@ int validate_config(const mixattn_config* cfg, CacheManager* cm, bool allocate =
 int enqueue_append(mixattn_ctx* c, int layer, int n_seqs, const int32_t* seq_ids,
                    const int32_t* n_new, const std::vector<int32_t>& start_pos,
                    const std::vector<PageGrant>& grants, const void* k, const void* v,
-                   cudaStream_t st) {
+                   cudaStream_t st, double rope_log2_theta = 0.0) {
   const LayerInfo& li = c->cm.layer(layer);
   const bool ring = li.kind == MIXATTN_SLIDING;
   bool single = true;
@@ -188,6 +188,7 @@ int enqueue_append(mixattn_ctx* c, int layer, int n_seqs, const int32_t* seq_ids
   p.window = ring ? li.window : 0;
   p.ring_pages = ring ? ring_pages_of(li.window) : 0;
   p.geom = c->geom;
+  p.rope_log2_theta = rope_log2_theta;
   int row = 0;
   size_t gi = 0;
   for (int i0 = 0; i0 < n_seqs; i0 += kMaxCallSeqs) {
@@ -306,8 +307,8 @@ int mixattn_seq_reset(mixattn_ctx* c, int32_t seq) {
   return MIXATTN_OK;
 }
 
-int mixattn_append_kv(mixattn_ctx* c, int32_t layer, int32_t n_seqs, const int32_t* seq_ids,
-                      const int32_t* n_new, const void* k, const void* v, void* stream) {
+static int append_impl(mixattn_ctx* c, int32_t layer, int32_t n_seqs, const int32_t* seq_ids,
+                       const int32_t* n_new, const void* k, const void* v, void* stream, double rope_log2_theta) {
   if (c == nullptr) return MIXATTN_ERR_INVALID_ARG;
   int rc = c->cm.check_append(layer, n_seqs, seq_ids, n_new);
   if (rc != MIXATTN_OK) return rc;
@@ -326,7 +327,19 @@ int mixattn_append_kv(mixattn_ctx* c, int32_t layer, int32_t n_seqs, const int32
   DeviceGuard g(c->device);
   if (!g.ok) return MIXATTN_ERR_CUDA;
   return enqueue_append(c, layer, n_seqs, seq_ids, n_new, start, grants, k, v,
-                        static_cast<cudaStream_t>(stream));
+                        static_cast<cudaStream_t>(stream), rope_log2_theta);
+}
+
+int mixattn_append_kv(mixattn_ctx* c, int32_t layer, int32_t n_seqs, const int32_t* seq_ids,
+                      const int32_t* n_new, const void* k, const void* v, void* stream) {
+  return append_impl(c, layer, n_seqs, seq_ids, n_new, k, v, stream, 0.0);
+}
+
+int mixattn_append_kv_rope(mixattn_ctx* c, int32_t layer, int32_t n_seqs, const int32_t* seq_ids,
+                           const int32_t* n_new, const void* k, const void* v, float rope_theta,
+                           void* stream) {
+  if (!(rope_theta > 1.f) || !isfinite(rope_theta)) return MIXATTN_ERR_INVALID_ARG;
+  return append_impl(c, layer, n_seqs, seq_ids, n_new, k, v, stream, log2((double)rope_theta));
 }
 
 // L2 policy of a decode launch (see l2_policy_of in decode_bf16.cu).  Only a ring that a later

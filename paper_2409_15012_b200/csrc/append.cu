@@ -3,6 +3,8 @@
 //
 // Paper, Section 1 (keys/values of earlier tokens are cached) and Section 3 (a window-s
 // cache keeps the past s tokens).  HBM-bound copy; 16-byte vector accesses.
+#include <cuda_bf16.h>
+
 #include "internal.h"
 
 namespace mixattn {
@@ -11,6 +13,40 @@ namespace {
 
 constexpr int kThreads = 256;
 constexpr int kTokensPerBlock = 8;
+
+// Rotary position embedding of one 16-byte chunk of a key row (RoFormer's definition, which
+// Section 4 of the paper cites): channel pair (2i, 2i+1) at position m turns by the angle
+// m * theta^(-2i/d).  The angle is formed and reduced modulo 2 pi in double precision
+// (positions reach 10^5 and the first pairs turn by about a radian per position), the
+// rotation itself runs in fp32, and bf16 rows are rounded once.
+__device__ __forceinline__ void rope_pair(float& a, float& b, int pair, int pos, int head_dim, double log2_theta) {
+  const double freq = exp2(-2.0 * (double)pair / (double)head_dim * log2_theta);
+  double ang = (double)pos * freq;
+  ang -= 6.283185307179586476925 * rint(ang * 0.15915494309189533577);
+  float sn, cs;
+  sincosf((float)ang, &sn, &cs);
+  const float x = a, y = b;
+  a = x * cs - y * sn;
+  b = x * sn + y * cs;
+}
+__device__ __forceinline__ int4 rope_chunk(int4 v, const KvGeom& ge, int chunk, int pos, double log2_theta) {
+  if (ge.elem_bytes == 4) {   // 4 fp32 = pairs 2 chunk, 2 chunk + 1
+    float f[4] = {__int_as_float(v.x), __int_as_float(v.y), __int_as_float(v.z), __int_as_float(v.w)};
+    rope_pair(f[0], f[1], 2 * chunk, pos, ge.head_dim, log2_theta);
+    rope_pair(f[2], f[3], 2 * chunk + 1, pos, ge.head_dim, log2_theta);
+    return make_int4(__float_as_int(f[0]), __float_as_int(f[1]), __float_as_int(f[2]), __float_as_int(f[3]));
+  }
+  int w[4] = {v.x, v.y, v.z, v.w};   // 8 bf16 = pairs 4 chunk .. 4 chunk + 3, one pair per word
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    __nv_bfloat162 h = *reinterpret_cast<__nv_bfloat162*>(&w[i]);
+    float a = __low2float(h), b = __high2float(h);
+    rope_pair(a, b, 4 * chunk + i, pos, ge.head_dim, log2_theta);
+    h = __floats2bfloat162_rn(a, b);
+    w[i] = *reinterpret_cast<int*>(&h);
+  }
+  return make_int4(w[0], w[1], w[2], w[3]);
+}
 
 __global__ void __launch_bounds__(kThreads) append_kernel(const __grid_constant__ AppendParams p) {
   const AppendEntry& e = p.e[blockIdx.y];
@@ -47,7 +83,9 @@ __global__ void __launch_bounds__(kThreads) append_kernel(const __grid_constant_
     const char* src = (const char*)(which ? p.v : p.k) +
                       ((int64_t)(e.src_row0 + t) * ge.n_kv_heads + g) * ge.row_bytes + chunk * 16;
     char* dst = p.pool + kv_chunk_offset(ge, page, g, which, slot, chunk);
-    *reinterpret_cast<int4*>(dst) = *reinterpret_cast<const int4*>(src);
+    int4 val = *reinterpret_cast<const int4*>(src);
+    if (p.rope_log2_theta > 0.0 && which == 0) val = rope_chunk(val, ge, chunk, pos, p.rope_log2_theta);
+    *reinterpret_cast<int4*>(dst) = val;
   }
 }
 

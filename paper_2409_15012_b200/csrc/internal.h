@@ -77,6 +77,7 @@ struct AppendParams {
   int32_t window;
   int32_t ring_pages;    // pages per sequence in a ring
   KvGeom geom;
+  double rope_log2_theta;  // > 0: K rows are rotated (rotary embedding, base theta) at their positions
   int32_t n_entries;
   AppendEntry e[kMaxCallSeqs];
 };
