@@ -151,3 +151,31 @@ def test_cache_bytes_follow_the_sharing_law():
             ph = mo.PhysicalCache(lay, Hkv, D, B, n_pages, store_values=False)
             assert mx.cache_bytes(cfg) == ph.cache_bytes(e)
             assert mx.arena_bytes(cfg) > mx.cache_bytes(cfg)
+
+
+def test_chunk_and_rope_calls_on_a_host_only_context():
+    # argument checks run on the host before anything else; a host-only context keeps the
+    # bookkeeping of a rope append (k / v ignored) and cannot attend
+    layout = cf.layout_tiny(8)
+    ph = mo.PhysicalCache(layout, 2, 64, 2, 6, store_values=False)
+    ctx = mx.Context(layout, 4, 2, 64, mx.F32, 2, 6, device=-1)
+    assert ctx.rc_attend_chunk(0, [0], [4], None, None, None, None) == mx.ERR_UNSUPPORTED   # no scratch configured
+    ctx.close()
+    ctx = mx.Context(layout, 4, 2, 64, mx.F32, 2, 6, device=-1, chunk_scratch_tokens=32)
+    for o in cf.owners_of(layout):
+        assert ctx.rc_append_kv_rope(o, [0, 1], [20, 3], None, None, 10000.0) == 0
+        ph.append(o, [0, 1], [20, 3])
+    _compare_state(ctx, ph, layout, 2)
+    assert ctx.rc_append_kv_rope(0, [0], [1], None, None, 1.0) == mx.ERR_INVALID_ARG        # theta must exceed 1
+    assert ctx.rc_append_kv_rope(0, [0], [1], None, None, float("inf")) == mx.ERR_INVALID_ARG
+    assert ctx.rc_append_kv_rope(2, [0], [1], None, None, 10000.0) == mx.ERR_NOT_OWNER
+    assert ctx.rc_attend_chunk(0, [0, 0], [1, 1], None, None, None, None) == mx.ERR_INVALID_ARG
+    assert ctx.rc_attend_chunk(0, [5], [1], None, None, None, None) == mx.ERR_BAD_SEQ
+    assert ctx.rc_attend_chunk(0, [0], [0], None, None, None, None) == mx.ERR_INVALID_ARG
+    assert ctx.rc_attend_chunk(7, [0], [1], None, None, None, None) == mx.ERR_INVALID_ARG
+    assert ctx.rc_attend_chunk(0, [0], [13], None, None, None, None) == mx.ERR_TOO_LARGE      # 20 cached + 13 > 32
+    assert ctx.rc_attend_chunk(1, [0], [26], None, None, None, None) == mx.ERR_TOO_LARGE      # ring: 7 cached + 26 > 32
+    assert ctx.rc_attend_chunk(1, [0], [25], None, None, None, None) == mx.ERR_CUDA           # fits; no device
+    assert ctx.rc_attend_chunk(0, [0, 1], [4, 4], None, None, None, None) == mx.ERR_CUDA
+    _compare_state(ctx, ph, layout, 2)                                                        # nothing stored
+    ctx.close()
