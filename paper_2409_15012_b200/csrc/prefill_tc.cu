@@ -67,7 +67,8 @@ enum {
   B_VF = 10, B_VE = 12,          // V stage full / free
   B_SF = 14, B_SR = 16,          // S buffer: scores ready / buffer (with the P in it) consumed by both P V
   B_PF = 18,                     // per stream and S buffer (18 + 2 stream + buffer): P announced
-  B_OF = 22,                     // per stream: P V done
+  B_OF = 22,                     // per stream: the item's last P V done (one phase per item: a parity wait
+                                 // is only valid for the phase right after the last one known complete)
   B_XC = 24, B_OR = 25,          // per item: streams published (reference, sum) / epilogue has read the O accumulators
   B_N = 26
 };
@@ -410,7 +411,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
             for (int ks = 0; ks < 4; ++ks)   // 64 keys = 4 steps of 16
               umma_bf16_ts(tmem + kColO + hs * 128, tmem + kColS + sb * 128 + hs * 64 + ks * 8,
                            vdesc + (uint64_t)(ks * (2048 >> 4)), kIdescPV, (j > 0 || ks > 0) ? 1u : 0u);
-            umma_commit(BAR(B_OF + hs));   // this stream's accumulator is up to date
+            if (j == w.n_tiles - 1) umma_commit(BAR(B_OF + hs));   // this stream's accumulator is complete
             umma_commit(BAR(B_VE + vs));   // V stage free once both streams' P V are done (count 2)
             umma_commit(BAR(B_SR + sb));   // and so is the S buffer
           }
@@ -429,17 +430,16 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     const uint32_t lane_base = tmem + ((uint32_t)(qd * 32) << 16);
     const float2* xchg = reinterpret_cast<const float2*>(gbase + kSmXchg);
     bool ok = true;
-    int G = 0, it = 0;
+    int it = 0;
     for (int id = blockIdx.x; id < n_ids && ok; id += gridDim.x) {
       const WorkItem w = get_item(p, id);
       if (!w.valid) continue;
-      G += w.n_tiles;
       ok = __all_sync(0xffffffffu, mbar_wait(BAR(B_XC), it & 1, abort_flag));
       if (!ok) break;
       const float2 lo = xchg[r], hi = xchg[128 + r];
       // both streams' last P V of the item have landed
-      ok = __all_sync(0xffffffffu, mbar_wait(BAR(B_OF + 0), (G - 1) & 1, abort_flag) &&
-                                   mbar_wait(BAR(B_OF + 1), (G - 1) & 1, abort_flag));
+      ok = __all_sync(0xffffffffu, mbar_wait(BAR(B_OF + 0), it & 1, abort_flag) &&
+                                   mbar_wait(BAR(B_OF + 1), it & 1, abort_flag));
       if (!ok) break;
       tc_fence_after();
       const float m_all = fmaxf(lo.x, hi.x);              // finite for every valid row (key i is visible)
@@ -556,7 +556,9 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
           // they have accumulated, and recompute this tile's weights
           const float alpha = far ? ex2_approx(m_ref - mt) : 1.f;
           if (j > 0) {   // the O row holds earlier tiles: rescale it once this stream's previous P V has landed
-            if (!__all_sync(0xffffffffu, mbar_wait(BAR(B_OF + hs), (Gj - 1) & 1, abort_flag))) { ok = false; break; }
+            // (the S buffer of tile G - 1 is released when both streams' P V of that tile are done;
+            // its previous phase is known complete because the scores of tile G - 1 existed)
+            if (!__all_sync(0xffffffffu, mbar_wait(BAR(B_SR + (sb ^ 1)), ((Gj - 1) >> 1) & 1, abort_flag))) { ok = false; break; }
             tc_fence_after();
 #pragma unroll 1
             for (int c = 0; c < 4; ++c) {

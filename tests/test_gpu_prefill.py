@@ -174,3 +174,38 @@ def test_prefill_scores_that_outrun_the_exponent_reference(gain):
         assert sess.ctx.get_device_status() == 0
     finally:
         sess.close()
+
+
+def test_many_short_prompts_repeated_calls():
+    # 64 prompts of 200 tokens: thousands of work items of one or two key tiles, so the warps that
+    # write finished tiles fall behind the ones that compute them; every repetition must give the
+    # same bits, and those must match the checker (an accumulator read before its last product
+    # has landed shows up here)
+    mx, runner = load_lib()
+    wl = cf.prefill_chunk().scaled(batch=64, seq_len=200)
+    sess = runner.Session(wl, [0] * wl.batch)
+    dt = torch_dt(wl.dtype)
+    S = wl.seq_len
+    try:
+        for l in (12, 2):        # readers of the standard and of a sliding-window cache: repeatable
+            kind, W, owner = wl.layout[l]
+            q, k, v = sess.prefill_inputs(l)
+            first = None
+            for rep in range(12):
+                out = torch.full_like(q, float("nan"))
+                sess.prefill_layer(l, q, k, v, out)
+                torch.cuda.synchronize()
+                if first is None:
+                    first = out
+                else:
+                    assert torch.equal(out.view(torch.int16), first.view(torch.int16)), f"layer {l} repetition {rep}"
+            got = first.float().cpu().double().numpy().reshape(wl.batch, S, wl.n_q_heads, wl.head_dim)
+            for b in (0, 31, 63):
+                qc = si.q_tokens(wl.seed, l, b, 0, S, wl.n_q_heads, wl.head_dim, dt)
+                Kc, Vc = si.kv_tokens(wl.seed, owner, b, 0, S, wl.n_kv_heads, wl.head_dim, dt)
+                rows = [0, 1, 127, 128, 129, 199]
+                ref = mo.prefill_attention(qc, Kc, Vc, kind, W, rows=rows)
+                check_close(got[b][rows], ref, wl.dtype, f"layer {l} seq {b}")
+        assert sess.ctx.get_device_status() == 0
+    finally:
+        sess.close()
