@@ -446,6 +446,10 @@ cudaError_t launch_decode_split_bf16(const DecodeParams& p, int sm_count, cudaSt
   const size_t budget = small ? 110 * 1024 : 220 * 1024;
   int n_stages = kMaxStages;
   while (n_stages > 2 && smem_bytes(D, p.group, n_stages, ncw) > budget) --n_stages;
+  // Two consumer groups take alternate tiles: with an even ring every stage always belongs to the
+  // same group, which then waits for its phases one after the other (a parity wait is only valid
+  // for the phase right after the last one known complete).
+  if (ncw == 8 && (n_stages & 1)) --n_stages;
   const size_t smem = smem_bytes(D, p.group, n_stages, ncw);
   const int slots = small ? 2 * sm_count : sm_count;
   const int grid = p.total_items < slots ? p.total_items : slots;
