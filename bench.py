@@ -189,7 +189,10 @@ def run_reference_arm(args, wl):
         "impl": "reference", "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": secs / args.steps * 1e3,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
-        "data": "synthetic", "config": {"workload": wl.name, "sample": sample},
+        "data": "synthetic",
+        "config": {"workload": wl.name, "batch": wl.batch, "context": wl.context or list(wl.context_range),
+                   "window": 1024, "layers": len(wl.layout), "heads": f"{wl.n_q_heads}/{wl.n_kv_heads}x{wl.head_dim}",
+                   "l2": "host run: no device cache involved", "parallelism": "replicas only", "sample": sample},
         "cpu_baseline": {"value": value, "unit": "GB/s", "cores": threads, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }
