@@ -42,10 +42,10 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 
 # (dram__bytes_read.sum + dram__bytes_write.sum) / algorithmic KV bytes of the dominant kernel, from the
 # ncu capture of a batch-4 launch summarised in profiles/decode_split_bf16_kernel.mid_decode.md
-# (540.64 MB moved for 536.95 MB of keys and values).  DRAM traffic grows in proportion to the keys read,
+# (541.30 MB moved for 536.95 MB of keys and values).  DRAM traffic grows in proportion to the keys read,
 # so the full-size figure is this ratio times the launch's algorithmic bytes.  Set to None when the
 # kernel changes until the counters are taken again.
-DECODE_FULL_TRAFFIC_RATIO = 540.635392 / 536.952832
+DECODE_FULL_TRAFFIC_RATIO = 541.304832 / 536.952832
 
 
 def load_peaks():
