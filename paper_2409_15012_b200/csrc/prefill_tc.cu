@@ -24,7 +24,8 @@
 //              S buffer (tcgen05.st).  The exponent reference of a row is the maximum of the
 //              first tile in which the row saw a key and is only moved (accumulators
 //              rescaled, weights recomputed) when a later score leads it by more than 2^64,
-//              so the exponentials of a tile never wait for the tile maximum.
+//              which is noticed from the sum of the tile's weights: the exponentials of a
+//              tile neither wait for the tile maximum nor compute it.
 //   warps 12-15  epilogue: thread r merges the two accumulators of row r, normalises and
 //              writes the row while the softmax warps are already on the next work item.
 //
@@ -534,7 +535,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         // probe the next tile's scores now; the answer is read after the exponentials
         const bool more = j + 1 < w.n_tiles;
         const bool next_ready = more && mbar_test_wait(BAR(B_SF + (sb ^ 1)), ((Gj + 1) >> 1) & 1);
-        float sum0 = 0.f, sum1 = 0.f, mxa = -INFINITY, mxb = -INFINITY;
+        float sum0 = 0.f, sum1 = 0.f;
         uint32_t pk[32];
 #pragma unroll
         for (int e = 0; e < 64; e += 4) {
@@ -546,14 +547,28 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
           sum1 += p1 + p3;
           pk[e >> 1] = pack_bf16(p0, p1);
           pk[(e >> 1) + 1] = pack_bf16(p2, p3);
-          mxa = fmax3(mxa, __uint_as_float(sv[e]), __uint_as_float(sv[e + 1]));
-          mxb = fmax3(mxb, __uint_as_float(sv[e + 2]), __uint_as_float(sv[e + 3]));
         }
-        const float mt = fmaxf(mxa, mxb) * p.scale_log2e;
-        const bool far = mt > m_ref + kMaxLead;
-        if (__any_sync(0xffffffffu, far)) {
-          // rare: move the reference of the leading rows up to the tile maximum, rescale what
+        // A score that leads the reference by more than 2^kMaxLead shows in the sum of the tile's
+        // weights (64 weights of at most 2^kMaxLead each stay below 2^(kMaxLead + 6); an overflow
+        // gives inf or NaN, which fail the comparison too), so the loop above carries no maximum.
+        const bool big = !(sum0 + sum1 <= 0x1p70f);
+        static_assert(kMaxLead == 64.f, "the bound above is 2^(kMaxLead + 6)");
+        if (__any_sync(0xffffffffu, big)) {
+          // rare: take the tile maximum from the scores, which are still in the S buffer (P has
+          // not been written yet), move the reference of the leading rows up to it, rescale what
           // they have accumulated, and recompute this tile's weights
+          tmem_ld32(s_addr, *reinterpret_cast<uint32_t(*)[32]>(&sv[0]));
+          tmem_ld32(s_addr + 32, *reinterpret_cast<uint32_t(*)[32]>(&sv[32]));
+          tmem_wait_ld_pin(*reinterpret_cast<uint32_t(*)[32]>(&sv[0]), *reinterpret_cast<uint32_t(*)[32]>(&sv[32]));
+          if (edge) mask_edges();
+          float mxa = -INFINITY, mxb = -INFINITY;
+#pragma unroll
+          for (int e = 0; e < 64; e += 4) {
+            mxa = fmax3(mxa, __uint_as_float(sv[e]), __uint_as_float(sv[e + 1]));
+            mxb = fmax3(mxb, __uint_as_float(sv[e + 2]), __uint_as_float(sv[e + 3]));
+          }
+          const float mt = fmaxf(mxa, mxb) * p.scale_log2e;
+          const bool far = mt > m_ref + kMaxLead;
           const float alpha = far ? ex2_approx(m_ref - mt) : 1.f;
           if (j > 0) {   // the O row holds earlier tiles: rescale it once this stream's previous P V has landed
             // (the S buffer of tile G - 1 is released when both streams' P V of that tile are done;
@@ -575,11 +590,6 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
           neg_m = m_ref == -INFINITY ? 0.f : -m_ref;
           sum0 = 0.f;
           sum1 = 0.f;
-          // the scores are still in the S buffer (P has not been written yet)
-          tmem_ld32(s_addr, *reinterpret_cast<uint32_t(*)[32]>(&sv[0]));
-          tmem_ld32(s_addr + 32, *reinterpret_cast<uint32_t(*)[32]>(&sv[32]));
-          tmem_wait_ld_pin(*reinterpret_cast<uint32_t(*)[32]>(&sv[0]), *reinterpret_cast<uint32_t(*)[32]>(&sv[32]));
-          if (edge) mask_edges();
 #pragma unroll
           for (int e = 0; e < 64; e += 2) {
             const float p0 = ex2_approx(fmaf(__uint_as_float(sv[e]), p.scale_log2e, neg_m));
