@@ -269,6 +269,30 @@ def chunk_figures(mx, runner, peaks, device, prefix=6144, chunk=2048):
             t = (ms / n + msg / ng) * 1e-3
             res[name] = {"ms_attention": ms / n, "ms_gather": msg / ng, "tflops": flops / t / 1e12,
                          "frac_of_bf16_peak": flops / t / 1e12 / peaks["bf16_tflops"], "useful_flop": flops}
+        # the same chunk through all 24 layers, each reader handed its owner's K/V, with the copy of
+        # the cached keys shared by the layers that read one cache (4 copies: F, S1, F, S2)
+        sess.ctx.set_chunk_gather_reuse(True)
+        kv = {}
+        for o in sess.owners:
+            K, V = si.kv_tokens_multi(wl.seed, o, ids, [prefix] * B, chunk, wl.n_kv_heads, D, sess.dt, sess.dev)
+            kv[o] = (K.reshape(-1, wl.n_kv_heads, D), V.reshape(-1, wl.n_kv_heads, D))
+        q = si.q_tokens_multi(wl.seed, 0, ids, [prefix] * B, chunk, Hq, D, sess.dt, sess.dev).reshape(-1, Hq, D)
+        out = torch.empty_like(q)
+        flops_pass = 0.0
+        for timed in (False, True):
+            sess.ctx.profile_enable(timed)
+            for layer, (kind, _, owner) in enumerate(wl.layout):
+                sess.ctx.attend_chunk(layer, ids, lens, q, kv[owner][0], kv[owner][1], out)
+                if timed:
+                    flops_pass += 4.0 * D * (pairs_full if kind == cf.FULL else pairs_slide) * Hq * B
+            torch.cuda.synchronize()
+        ms_pass = sum(sess.ctx.profile_read(c)[1] for c in (mx.K_PREFILL_FULL, mx.K_PREFILL_SLIDING, mx.K_GATHER))
+        n_gather = sess.ctx.profile_read(mx.K_GATHER)[0]
+        sess.ctx.profile_enable(False)
+        sess.ctx.set_chunk_gather_reuse(False)
+        res["layout_pass"] = {"layers": len(wl.layout), "gathers": n_gather, "ms": ms_pass,
+                              "tflops": flops_pass / (ms_pass * 1e-3) / 1e12,
+                              "frac_of_bf16_peak": flops_pass / (ms_pass * 1e-3) / 1e12 / peaks["bf16_tflops"]}
         res["config"] = {"workload": wl.name, "batch": B, "cached_prefix": prefix, "chunk": chunk, "window": W}
     finally:
         sess.close()

@@ -192,6 +192,20 @@ int mixattn_attend_chunk(mixattn_ctx* ctx, int32_t layer, int32_t n_seqs, const 
                          const int32_t* seq_lens, const void* q, const void* k, const void* v,
                          void* out, void* stream);
 
+/* One copy for all the layers that share a cache (Section 3: such layers read
+ * the same cached keys, and a layer that reuses a cache is handed its owner's
+ * K/V for the chunk, so consecutive mixattn_attend_chunk calls of these layers
+ * would copy identical rows into the chunk scratch).  With reuse enabled, a
+ * chunk call skips the copy when the previous chunk call on this context read
+ * the same owner's cache for the same seq_ids and seq_lens with the same k and
+ * v pointers on the same stream, fitted the scratch in one piece, and no call
+ * since has changed a cache (append, prefill of an owner, seq_reset).  By
+ * enabling it the caller promises that the contents behind k and v do not
+ * change between such calls.  Off by default; enable = 0 switches it off again
+ * and forgets what the scratch holds.  Results are identical either way.
+ * Errors: INVALID_ARG for a null context. */
+int mixattn_set_chunk_gather_reuse(mixattn_ctx* ctx, int32_t enable);
+
 /* Size of the static device array behind mixattn_decode_static_scratch. */
 #define MIXATTN_STATIC_SCRATCH_BYTES (8u << 20)
 

@@ -85,6 +85,7 @@ def _load() -> C.CDLL:
         "mixattn_debug_read_kv": [vp, i32, i32, i32, vp, vp],
         "mixattn_get_device_status": [vp, p32],
         "mixattn_set_split_tokens": [vp, i32],
+        "mixattn_set_chunk_gather_reuse": [vp, i32],
         "mixattn_profile_enable": [vp, i32],
         "mixattn_profile_read": [vp, i32, p32, C.POINTER(C.c_float)],
         "mixattn_get_launch_count": [vp, C.POINTER(C.c_int64)],
@@ -105,7 +106,8 @@ EXPORTS = [
     "mixattn_attend_chunk",
     "mixattn_get_len", "mixattn_get_block_table", "mixattn_get_n_free_pages",
     "mixattn_get_ring_state", "mixattn_locate", "mixattn_debug_read_kv",
-    "mixattn_get_device_status", "mixattn_set_split_tokens", "mixattn_profile_enable",
+    "mixattn_get_device_status", "mixattn_set_split_tokens", "mixattn_set_chunk_gather_reuse",
+    "mixattn_profile_enable",
     "mixattn_profile_read", "mixattn_get_launch_count", "mixattn_strerror",
 ]
 
@@ -331,6 +333,13 @@ class Context:
         rc = lib.mixattn_set_split_tokens(self.h, tokens)
         if rc:
             raise MixAttnError(rc, "mixattn_set_split_tokens")
+
+    def set_chunk_gather_reuse(self, enable: bool):
+        """Layers that share a cache gather the same rows for a chunk: copy them once per run of
+        such calls (the caller keeps k / v unchanged between them)."""
+        rc = lib.mixattn_set_chunk_gather_reuse(self.h, 1 if enable else 0)
+        if rc:
+            raise MixAttnError(rc, "mixattn_set_chunk_gather_reuse")
 
     def profile_enable(self, enable: bool):
         rc = lib.mixattn_profile_enable(self.h, 1 if enable else 0)

@@ -4,6 +4,7 @@
 #include <string.h>
 
 #include <new>
+#include <algorithm>
 #include <vector>
 
 #include "cache_manager.hpp"
@@ -90,6 +91,19 @@ struct mixattn_ctx {
   std::vector<ProfileRecord> records;
   std::vector<cudaEvent_t> event_pool;
   bool sticky_cuda_error = false;
+  // Chunk calls of layers that share a cache gather the same rows: what the scratch holds is
+  // remembered so that, when the caller has enabled it, the copy runs once per run of such calls.
+  bool chunk_reuse = false;
+  uint64_t cache_epoch = 0;   // bumped by every call that changes a cache
+  struct GatherKey {
+    bool valid = false;
+    int owner = -1;
+    uint64_t epoch = 0;
+    const void* k = nullptr;
+    const void* v = nullptr;
+    cudaStream_t st = nullptr;
+    std::vector<int32_t> ids, lens;
+  } scratch_holds;
 
   char* owner_storage(int layer) const { return arena + plan.owner_off[cm.layer(layer).owner_slot]; }
   int32_t* dev_table() const { return reinterpret_cast<int32_t*>(arena + plan.table_off); }
@@ -304,6 +318,7 @@ int mixattn_seq_reset(mixattn_ctx* c, int32_t seq) {
   if (c == nullptr) return MIXATTN_ERR_INVALID_ARG;
   if (!c->cm.valid_seq(seq)) return MIXATTN_ERR_BAD_SEQ;
   c->cm.seq_reset(seq);
+  ++c->cache_epoch;
   return MIXATTN_OK;
 }
 
@@ -323,6 +338,7 @@ static int append_impl(mixattn_ctx* c, int32_t layer, int32_t n_seqs, const int3
   for (int i = 0; i < n_seqs; ++i) start[i] = c->cm.len(layer, seq_ids[i]);
   std::vector<PageGrant> grants;
   c->cm.apply_append(layer, n_seqs, seq_ids, n_new, &grants);
+  ++c->cache_epoch;
   if (c->host_only) return MIXATTN_OK;
   DeviceGuard g(c->device);
   if (!g.ok) return MIXATTN_ERR_CUDA;
@@ -493,6 +509,7 @@ int mixattn_prefill(mixattn_ctx* c, int32_t layer, int32_t n_seqs, const int32_t
     std::vector<int32_t> start(n_seqs, 0);
     std::vector<PageGrant> grants;
     c->cm.apply_append(layer, n_seqs, seq_ids, seq_lens, &grants);
+    ++c->cache_epoch;
     int rc = enqueue_append(c, layer, n_seqs, seq_ids, seq_lens, start, grants, k, v, st);
     if (rc != MIXATTN_OK) return rc;
   }
@@ -595,6 +612,32 @@ int mixattn_attend_chunk(mixattn_ctx* c, int32_t layer, int32_t n_seqs, const in
   p.k = ks;
   p.v = vs;
 
+  // The rows this call would copy are already in the scratch when the previous chunk call read
+  // the same cache for the same sequences with the same chunk K/V, in one piece, on this stream,
+  // and no cache has changed since (a reader layer right after its owner, or after another reader).
+  bool one_piece = n_seqs <= kMaxCallSeqs;
+  {
+    int64_t rows = 0;
+    for (int i = 0; i < n_seqs; ++i) rows += (int64_t)n_prefix[i] + seq_lens[i];
+    one_piece = one_piece && rows <= scratch;
+  }
+  mixattn_ctx::GatherKey& held = c->scratch_holds;
+  const bool reuse = c->chunk_reuse && one_piece && held.valid && held.owner == li.owner &&
+                     held.epoch == c->cache_epoch && held.k == k && held.v == v && held.st == st &&
+                     held.ids.size() == (size_t)n_seqs &&
+                     std::equal(held.ids.begin(), held.ids.end(), seq_ids) &&
+                     std::equal(held.lens.begin(), held.lens.end(), seq_lens);
+  if (!reuse) {
+    held.valid = false;   // set again below, once the copy of a one-piece call has been issued
+    held.owner = li.owner;
+    held.epoch = c->cache_epoch;
+    held.k = k;
+    held.v = v;
+    held.st = st;
+    held.ids.assign(seq_ids, seq_ids + n_seqs);
+    held.lens.assign(seq_lens, seq_lens + n_seqs);
+  }
+
   // groups of consecutive sequences whose keys fit the scratch together; the stream orders
   // each group's attention before the next group's copy reuses the scratch
   int64_t row = 0;   // first chunk row of the group in q / k / v / out
@@ -628,8 +671,12 @@ int mixattn_attend_chunk(mixattn_ctx* c, int32_t layer, int32_t n_seqs, const in
     gp.v_chunk = static_cast<const char*>(v) + (size_t)row * Hkv * D * esz;
     p.q = static_cast<const char*>(q) + (size_t)row * Hq * D * esz;
     p.out = static_cast<char*>(out) + (size_t)row * Hq * D * esz;
-    cudaError_t e = launch_recorded(c, MIXATTN_K_GATHER, st, [&] { return launch_gather(gp, max_rows, st); });
-    if (e != cudaSuccess) return MIXATTN_ERR_CUDA;
+    cudaError_t e = cudaSuccess;
+    if (!reuse) {
+      e = launch_recorded(c, MIXATTN_K_GATHER, st, [&] { return launch_gather(gp, max_rows, st); });
+      if (e != cudaSuccess) return MIXATTN_ERR_CUDA;
+      held.valid = one_piece;
+    }
     const int cls = p.window ? MIXATTN_K_PREFILL_SLIDING : MIXATTN_K_PREFILL_FULL;
     const bool tc = prefill_tc_supported(c->cfg.dtype, D, p.q, p.k, p.v) && (((size_t)p.out) & 15) == 0;
     e = launch_recorded(c, cls, st, [&] {
@@ -740,6 +787,13 @@ int mixattn_get_device_status(mixattn_ctx* c, int32_t* status) {
 int mixattn_set_split_tokens(mixattn_ctx* c, int32_t tokens) {
   if (c == nullptr || tokens < 0) return MIXATTN_ERR_INVALID_ARG;
   c->split_tokens = tokens;
+  return MIXATTN_OK;
+}
+
+int mixattn_set_chunk_gather_reuse(mixattn_ctx* c, int32_t enable) {
+  if (c == nullptr) return MIXATTN_ERR_INVALID_ARG;
+  c->chunk_reuse = enable != 0;
+  c->scratch_holds.valid = false;
   return MIXATTN_OK;
 }
 

@@ -213,6 +213,9 @@ def serve_trace(layout, n_q_heads: int, n_kv_heads: int, head_dim: int, n_reques
         classes = (mx.K_APPEND, mx.K_DECODE_FULL, mx.K_DECODE_SLIDING, mx.K_COMBINE, mx.K_PREFILL_FULL,
                    mx.K_PREFILL_SLIDING, mx.K_GATHER)
         sess.ctx.profile_enable(True)
+        # prefill_in_chunks hands every reader its owner's K/V tensors, unchanged within a round:
+        # the cached keys of a shared cache are copied once per run of layers that read it
+        sess.ctx.set_chunk_gather_reuse(True)
         sess.prefill_in_chunks(chunk)
         torch.cuda.synchronize(sess.dev)
         prefill_ms = sum(sess.ctx.profile_read(c)[1] for c in classes)

@@ -165,3 +165,42 @@ def test_serving_trace_small():
         assert res["device_status"] == 0 and res["prefill_kernel_ms"] > 0 and res["decode_kernel_ms"] > 0
     finally:
         sess.close()
+
+
+@pytest.mark.parametrize("scratch_seqs", [2, 1])
+def test_gather_reuse_same_outputs_fewer_copies(scratch_seqs):
+    # Layers that share a cache gather the same rows: with reuse enabled the copy runs once per run
+    # of such layers (6-layer layout: standard owner, ring owner, two ring readers, a reader of the
+    # standard cache, a second ring owner = 4 copies per round instead of 6) and every output is
+    # bit-identical.  With a scratch that holds one sequence at a time the call works in two
+    # pieces and must copy every time.
+    mx, runner = load_lib()
+    layout = [(cf.FULL, 0, 0), (cf.SLIDING, 256, 1), (cf.SLIDING, 256, 1), (cf.SLIDING, 256, 1),
+              (cf.FULL, 0, 0), (cf.SLIDING, 256, 5)]
+    wl = cf.prefill_chunk().scaled(layout=layout, batch=2, seq_len=0)
+    total, chunk = 900, 300
+    results = []
+    for reuse in (False, True):
+        sess = runner.Session(wl, [total, total], headroom_tokens=2,
+                              chunk_scratch_tokens=scratch_seqs * total if scratch_seqs == 2 else total + 8)
+        try:
+            sess.ctx.set_chunk_gather_reuse(reuse)
+            sess.ctx.profile_enable(True)
+            outs = sess.prefill_in_chunks(chunk)
+            torch.cuda.synchronize()
+            n_gather = sess.ctx.profile_read(mx.K_GATHER)[0]
+            sess.ctx.profile_enable(False)
+            assert sess.ctx.get_device_status() == 0
+            results.append(([o.clone() for o in outs], n_gather))
+        finally:
+            sess.close()
+    (off, n_off), (on, n_on) = results
+    for a, b in zip(off, on):
+        assert torch.equal(a.view(torch.int16), b.view(torch.int16))
+    rounds = total // chunk
+    if scratch_seqs == 2:
+        assert n_off == 6 * rounds and n_on == 4 * rounds
+    else:
+        # the first round (empty caches, 2 x 300 rows) still fits in one piece; the later rounds
+        # take two pieces per call and copy each time
+        assert n_off == 6 + 12 * (rounds - 1) and n_on == 4 + 12 * (rounds - 1)
