@@ -130,6 +130,19 @@ __device__ __forceinline__ uint32_t movmatrix_t(uint32_t a) {  // transpose an 8
   asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(d) : "r"(a));
   return d;
 }
+// distributed shared memory: the address of the same variable in the first CTA of the cluster
+__device__ __forceinline__ uint32_t map_to_cta0(uint32_t local) {
+  uint32_t remote;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, 0;" : "=r"(remote) : "r"(local));
+  return remote;
+}
+__device__ __forceinline__ void st_cluster_f32(uint32_t addr, float v) {
+  asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(addr), "f"(v) : "memory");
+}
+// all threads of the cluster that have not exited (the producer warps exit on their own)
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
 template <int NCW>
 __device__ __forceinline__ void consumer_bar() {  // the consumer threads only
   asm volatile("bar.sync 1, %0;" ::"n"(NCW * 32) : "memory");
@@ -163,10 +176,24 @@ __device__ __forceinline__ Item decode_item(const DecodeParams& p, int it) {
   return x;
 }
 
+// The part of an item's keys that CTA `crank` of a two-CTA cluster takes: whole stages of
+// kTileKeys keys, the first CTA the larger half (never empty); the second may get none.
+__device__ __forceinline__ void cluster_share(Item& x, int crank) {
+  const int tiles = (x.t1 - x.t0 + kTileKeys - 1) / kTileKeys;   // x.t0 is a multiple of the page size
+  const int mid = min(x.t1, x.t0 + ((tiles + 1) / 2) * kTileKeys);
+  if (crank == 0) x.t1 = mid;
+  else if (mid < x.t1) x.t0 = mid;
+  else x.t0 = x.t1 = 0;   // nothing left for the second CTA: no stage is streamed
+}
+
 // NCW consumer warps: 8 (two groups alternating stages; one CTA per SM with a deep ring, for
 // long key streams) or 4 (one group; two CTAs per SM with short rings, so that a launch with
 // few, short work items keeps every item in flight at once instead of queueing two per SM).
-template <int D, int NCW>
+// CL = 2: a launch of few items runs each item on a thread-block cluster of two CTAs (two SMs),
+// which take halves of the item's keys and merge through distributed shared memory: one CTA
+// ingests K/V at a fixed rate, so a short launch that leaves SMs idle is halved this way
+// without a second launch.  The grid then holds exactly one cluster per item.
+template <int D, int NCW, int CL>
 __global__ void __launch_bounds__((NCW + 1) * 32, NCW == 8 ? 1 : 2)
 decode_split_bf16_kernel(const __grid_constant__ DecodeParams p, const int n_stages) {
   constexpr int kConsumerWarps = NCW;
@@ -183,6 +210,12 @@ decode_split_bf16_kernel(const __grid_constant__ DecodeParams p, const int n_sta
   float* merge_ml = merge + kConsumerWarps * rows_cap * D;            // [warp][row][2]
   uint64_t* bars = reinterpret_cast<uint64_t*>(merge_ml + kConsumerWarps * rows_cap * 2);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + 2 * kMaxStages);
+  // cluster exchange (CL > 1), in the first CTA of the cluster: [CTA][row][D] partial O, then [CTA][row] (max, sum)
+  float* xch = reinterpret_cast<float*>(bars + 2 * kMaxStages + 2);
+  int crank = 0;
+  if constexpr (CL > 1) asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(crank));
+  const int item0 = CL > 1 ? (int)blockIdx.x / CL : (int)blockIdx.x;
+  const int item_stride = CL > 1 ? (int)gridDim.x / CL : (int)gridDim.x;
   const uint32_t full0 = smem_u32(bars);
   const uint32_t empty0 = smem_u32(bars + kMaxStages);
 
@@ -203,6 +236,9 @@ decode_split_bf16_kernel(const __grid_constant__ DecodeParams p, const int n_sta
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   __syncthreads();
+  // every thread of the cluster checks in once; the consumers wait for this phase before their
+  // first access to the other CTA's shared memory, which must be running by then
+  if constexpr (CL > 1) asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
   // ... and do not touch global memory before the kernels ahead in the stream have
   // completed and flushed (a no-op when this kernel was launched the ordinary way)
   asm volatile("griddepcontrol.wait;" ::: "memory");
@@ -214,8 +250,9 @@ decode_split_bf16_kernel(const __grid_constant__ DecodeParams p, const int n_sta
     int K = 0;  // tiles issued by this CTA so far
     bool ok = true;
     const uint64_t l2_policy = l2_policy_of(p.pool, p.l2_keep_bytes, p.l2_pool_bytes);
-    for (int it = blockIdx.x; ok && it < p.total_items; it += gridDim.x) {
-      const Item x = decode_item(p, it);
+    for (int it = item0; ok && it < p.total_items; it += item_stride) {
+      Item x = decode_item(p, it);
+      if constexpr (CL > 1) cluster_share(x, crank);
       const int seq = p.seq_id[x.i];
       const int32_t* tbl = p.table ? p.table + (int64_t)seq * p.table_stride : nullptr;
       const int64_t ring_page0 = (int64_t)seq * p.ring_pages;
@@ -257,6 +294,13 @@ decode_split_bf16_kernel(const __grid_constant__ DecodeParams p, const int n_sta
         mbar_wait(full0 + 8 * (Kb % n_stages), (Kb / n_stages) & 1, abort_flag + 1);
       }
     }
+    if constexpr (CL > 1) {
+      // the producer takes no part in the merge, but the consumers' cluster barrier counts every
+      // thread: check in for it before leaving (after the start-up phase, which is complete as soon
+      // as both CTAs run)
+      __syncwarp();
+      asm volatile("barrier.cluster.wait.acquire.aligned;\n\tbarrier.cluster.arrive.release.aligned;" ::: "memory");
+    }
     return;
   }
 
@@ -276,8 +320,9 @@ decode_split_bf16_kernel(const __grid_constant__ DecodeParams p, const int n_sta
   const int v_tok = (lm >> 1) * 8 + lr, v_chk = lm & 1;   // V^T as A (.trans): (chunk 2jt|2jt+1) x (keys 0-7|8-15)
 
   int K = 0;
-  for (int it = blockIdx.x; it < p.total_items; it += gridDim.x) {
-    const Item x = decode_item(p, it);
+  for (int it = item0; it < p.total_items; it += item_stride) {
+    Item x = decode_item(p, it);
+    if constexpr (CL > 1) cluster_share(x, crank);
     const int rows = min(kMaxGroupRows, p.group - x.hc * kMaxGroupRows);
     const int h0 = x.g * p.group + x.hc * kMaxGroupRows;
 
@@ -387,21 +432,36 @@ decode_split_bf16_kernel(const __grid_constant__ DecodeParams p, const int n_sta
       }
     }
     consumer_bar<NCW>();
-    if (*abort_flag) {  // uniform: set before the barrier by whichever role gave up
-      if (threadIdx.x == 0) atomicExch(p.status, kDevWaitTimeout);
-      return;
-    }
-    for (int e = threadIdx.x; e < rows * D; e += kConsumerWarps * 32) {
+    const bool gave_up = *abort_flag != 0;  // uniform: set before the barrier by whichever role gave up
+    if (gave_up && threadIdx.x == 0) atomicExch(p.status, kDevWaitTimeout);
+    if (CL == 1 && gave_up) return;
+    // (in a cluster every consumer thread goes on to the cluster barrier below, which has no
+    // time-out of its own: the other CTA's threads reach it after at most their own bounded waits)
+    if constexpr (CL > 1) asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+    float* xo = xch;                                   // [CL][rows_cap][D]
+    float* xml = xch + CL * rows_cap * D;              // [CL][rows_cap][2]
+    for (int e = threadIdx.x; e < rows * D && !gave_up; e += kConsumerWarps * 32) {
       const int r = e / D, d = e - r * D;
       float M = -INFINITY;
 #pragma unroll
       for (int w = 0; w < kConsumerWarps; ++w) M = fmaxf(M, merge_ml[(w * rows_cap + r) * 2]);
       float L = 0.f, acc = 0.f;
+      if (M > -INFINITY) {   // (a CTA of a cluster may have had no key at all)
 #pragma unroll
-      for (int w = 0; w < kConsumerWarps; ++w) {
-        const float sc = exp2f(merge_ml[(w * rows_cap + r) * 2] - M);
-        L += merge_ml[(w * rows_cap + r) * 2 + 1] * sc;
-        acc += merge[((size_t)w * rows_cap + r) * D + d] * sc;
+        for (int w = 0; w < kConsumerWarps; ++w) {
+          const float sc = exp2f(merge_ml[(w * rows_cap + r) * 2] - M);
+          L += merge_ml[(w * rows_cap + r) * 2 + 1] * sc;
+          acc += merge[((size_t)w * rows_cap + r) * D + d] * sc;
+        }
+      }
+      if constexpr (CL > 1) {
+        // hand (M, L, acc) to the first CTA of the cluster through its shared memory
+        st_cluster_f32(map_to_cta0(smem_u32(xo + ((size_t)crank * rows_cap + r) * D + d)), acc);
+        if (d == 0) {
+          st_cluster_f32(map_to_cta0(smem_u32(xml + ((size_t)crank * rows_cap + r) * 2)), M);
+          st_cluster_f32(map_to_cta0(smem_u32(xml + ((size_t)crank * rows_cap + r) * 2 + 1)), L);
+        }
+        continue;
       }
       const int h = h0 + r;
       if (x.n_splits == 1) {
@@ -413,23 +473,49 @@ decode_split_bf16_kernel(const __grid_constant__ DecodeParams p, const int n_sta
         if (d == 0) p.part_ml[slot] = make_float2(M, L);
       }
     }
+    if constexpr (CL > 1) {
+      cluster_sync_all();   // both CTAs' partials are in the first CTA's shared memory
+      if (gave_up) return;
+      if (crank == 0) {
+        for (int e = threadIdx.x; e < rows * D; e += kConsumerWarps * 32) {
+          const int r = e / D, d = e - r * D;
+          const float M0 = xml[r * 2], M1 = xml[(rows_cap + r) * 2];
+          const float M = fmaxf(M0, M1);
+          const float s0 = exp2f(M0 - M), s1 = exp2f(M1 - M);   // 2^-inf = 0 for a CTA without keys
+          const float L = xml[r * 2 + 1] * s0 + xml[(rows_cap + r) * 2 + 1] * s1;
+          const float acc = xo[(size_t)r * D + d] * s0 + xo[((size_t)rows_cap + r) * D + d] * s1;
+          const int h = h0 + r;
+          if (x.n_splits == 1) {
+            reinterpret_cast<__nv_bfloat16*>(p.out)[((int64_t)x.i * p.n_q_heads + h) * D + d] =
+                __float2bfloat16_rn(acc / L);
+          } else {
+            const int64_t slot = (int64_t)(p.chunk_base[x.i] + x.c) * p.n_q_heads + h;
+            p.part_o[slot * D + d] = acc;
+            if (d == 0) p.part_ml[slot] = make_float2(M, L);
+          }
+        }
+      }
+    }
     consumer_bar<NCW>();
   }
 }
 
-size_t smem_bytes(int D, int group, int n_stages, int ncw) {
+size_t smem_bytes(int D, int group, int n_stages, int ncw, int cl) {
   const int rows_cap = group < kMaxGroupRows ? group : kMaxGroupRows;
   size_t stage = (size_t)kGroupWarps * 2 * kPage * D * 2;
-  return n_stages * stage + (size_t)ncw * rows_cap * (D + 2) * 4 + 2 * kMaxStages * 8 + 32;
+  const size_t exchange = cl > 1 ? (size_t)cl * rows_cap * (D + 2) * 4 : 0;
+  return n_stages * stage + (size_t)ncw * rows_cap * (D + 2) * 4 + 2 * kMaxStages * 8 + 32 + exchange;
 }
 
 }  // namespace
 
 cudaError_t prepare_decode_bf16() {
-  cudaError_t e = cudaFuncSetAttribute(decode_split_bf16_kernel<128, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(decode_split_bf16_kernel<64, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(decode_split_bf16_kernel<128, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, 113 * 1024);
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(decode_split_bf16_kernel<64, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, 113 * 1024);
+  cudaError_t e = cudaFuncSetAttribute(decode_split_bf16_kernel<128, 8, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(decode_split_bf16_kernel<64, 8, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(decode_split_bf16_kernel<128, 4, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 113 * 1024);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(decode_split_bf16_kernel<64, 4, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 113 * 1024);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(decode_split_bf16_kernel<128, 8, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(decode_split_bf16_kernel<64, 8, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
   return e;
 }
 
@@ -442,17 +528,20 @@ cudaError_t launch_decode_split_bf16(const DecodeParams& p, int sm_count, cudaSt
   int64_t max_keys = 0;
   for (int i = 0; i < p.n_seqs; ++i) max_keys = p.chunk_len[i] > max_keys ? p.chunk_len[i] : max_keys;
   const bool small = p.total_items > sm_count && p.total_items <= 2 * sm_count && max_keys <= 2048;
+  // At most one item per two SMs, and items of several stages: a cluster of two CTAs per item.
+  const bool paired = 2 * p.total_items <= sm_count && max_keys >= 4 * kTileKeys;
+  const int cl = paired ? 2 : 1;
   const int ncw = small ? 4 : 8;
   const size_t budget = small ? 110 * 1024 : 220 * 1024;
   int n_stages = kMaxStages;
-  while (n_stages > 2 && smem_bytes(D, p.group, n_stages, ncw) > budget) --n_stages;
+  while (n_stages > 2 && smem_bytes(D, p.group, n_stages, ncw, cl) > budget) --n_stages;
   // Two consumer groups take alternate tiles: with an even ring every stage always belongs to the
   // same group, which then waits for its phases one after the other (a parity wait is only valid
   // for the phase right after the last one known complete).
   if (ncw == 8 && (n_stages & 1)) --n_stages;
-  const size_t smem = smem_bytes(D, p.group, n_stages, ncw);
+  const size_t smem = smem_bytes(D, p.group, n_stages, ncw, cl);
   const int slots = small ? 2 * sm_count : sm_count;
-  const int grid = p.total_items < slots ? p.total_items : slots;
+  const int grid = paired ? 2 * p.total_items : (p.total_items < slots ? p.total_items : slots);
   // launched with programmatic stream serialization: the kernel's set-up may overlap the
   // tail of the previous kernel in the stream; it waits (griddepcontrol.wait) before its
   // first global access
@@ -461,17 +550,23 @@ cudaError_t launch_decode_split_bf16(const DecodeParams& p, int sm_count, cudaSt
   cfg.blockDim = dim3((ncw + 1) * 32);
   cfg.dynamicSmemBytes = smem;
   cfg.stream = st;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
+  attr[1].id = cudaLaunchAttributeClusterDimension;
+  attr[1].val.clusterDim.x = 2;
+  attr[1].val.clusterDim.y = 1;
+  attr[1].val.clusterDim.z = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = 1;
+  cfg.numAttrs = paired ? 2 : 1;
   if (D == 128) {
-    if (small) return cudaLaunchKernelEx(&cfg, decode_split_bf16_kernel<128, 4>, p, n_stages);
-    return cudaLaunchKernelEx(&cfg, decode_split_bf16_kernel<128, 8>, p, n_stages);
+    if (paired) return cudaLaunchKernelEx(&cfg, decode_split_bf16_kernel<128, 8, 2>, p, n_stages);
+    if (small) return cudaLaunchKernelEx(&cfg, decode_split_bf16_kernel<128, 4, 1>, p, n_stages);
+    return cudaLaunchKernelEx(&cfg, decode_split_bf16_kernel<128, 8, 1>, p, n_stages);
   }
-  if (small) return cudaLaunchKernelEx(&cfg, decode_split_bf16_kernel<64, 4>, p, n_stages);
-  return cudaLaunchKernelEx(&cfg, decode_split_bf16_kernel<64, 8>, p, n_stages);
+  if (paired) return cudaLaunchKernelEx(&cfg, decode_split_bf16_kernel<64, 8, 2>, p, n_stages);
+  if (small) return cudaLaunchKernelEx(&cfg, decode_split_bf16_kernel<64, 4, 1>, p, n_stages);
+  return cudaLaunchKernelEx(&cfg, decode_split_bf16_kernel<64, 8, 1>, p, n_stages);
 }
 
 }  // namespace mixattn
