@@ -159,3 +159,10 @@ def test_repeated_calls_are_bit_identical_and_profile_hooks_count():
             assert torch.equal(a.view(torch.int16), b.view(torch.int16))
     finally:
         sess.close()
+
+
+def test_bf16_few_items_short_and_long_sequences_together():
+    # a launch of few items gives every item two CTAs that halve its keys: a sequence of one
+    # stage or less leaves the second CTA without keys, 65 keys give it a single one
+    wl = cf.mid_decode().scaled(layout=cf.layout_tiny(512), batch=4, context=1000, n_q_heads=16, n_kv_heads=4)
+    run_decode_case(wl, [1000, 4, 63, 64], steps=2, chunk=250)
