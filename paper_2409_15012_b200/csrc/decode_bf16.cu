@@ -20,6 +20,9 @@
 //     (sequence not split) or an unnormalised partial + (max, sum) for the combine pass.
 //     (Combining inside this kernel -- last split to finish, ticket counter -- was
 //     measured slower: the fence before the ticket stalls the consumers per item.)
+//   * a launch with at most one item per two SMs gives each item a cluster of two CTAs,
+//     which stream halves of its keys and merge through distributed shared memory: one
+//     CTA ingests K/V at a bounded rate, so idle SMs are better used than a second launch.
 //
 // Every mbarrier wait is bounded: on time-out the kernel raises a status word and all
 // roles leave.
