@@ -11,7 +11,11 @@
  * Conventions for every call
  *   - returns MIXATTN_OK (0) or a negative MIXATTN_ERR_* code; nothing throws,
  *     aborts or traps.  All validation happens on the host before any launch,
- *     and a failing call changes no state.
+ *     and a call that fails it changes no state.  The one exception is
+ *     MIXATTN_ERR_CUDA from a launch or copy the CUDA runtime refused in the
+ *     middle of a call: the cache bookkeeping may already have moved, so the
+ *     context turns unusable (every later call that would touch the device
+ *     returns MIXATTN_ERR_CUDA); destroy it.
  *   - "host" pointers are read (or written) before the call returns.
  *     "device" pointers are borrowed until `stream` has executed the work the
  *     call enqueued.  `stream` is a cudaStream_t passed as void* (NULL = the
@@ -127,7 +131,7 @@ int mixattn_append_kv(mixattn_ctx* ctx, int32_t layer, int32_t n_seqs, const int
                       const int32_t* n_new, const void* k, const void* v, void* stream);
 
 /* mixattn_append_kv with the rotary position embedding fused into the copy
- * (Section 4: the models use RoPE, with a base theta that grows with the
+ * (Section 3: the models use RoPE, with a base theta that grows with the
  * context length; the embedding is RoFormer's): before a key row is stored,
  * its channel pairs (2i, 2i+1) are rotated by the angle t * theta^(-2i/d),
  * t the token's position in the sequence and d = head_dim.  Values are stored
@@ -232,7 +236,9 @@ int mixattn_set_chunk_gather_reuse(mixattn_ctx* ctx, int32_t enable);
  *     nothing launched;
  *   - the first call on a device looks up the array's device address (a CUDA
  *     runtime query with that device current); make that first call outside
- *     any stream capture;
+ *     any stream capture.  The address is kept for the life of the process;
+ *     after a cudaDeviceReset of that device it is stale and this entry point
+ *     must not be used any more;
  *   - all calls, from every context and stream of the process, share the one
  *     array per device.  Its contents are left over from the previous call;
  *     nothing in it needs to start at zero, since each call overwrites every

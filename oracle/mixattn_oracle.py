@@ -64,8 +64,7 @@ class OracleError(Exception):
 
 def validate_layout(layout: Sequence[Tuple[int, int, int]]) -> None:
     """A reader names an EARLIER layer that computes its own cache (Section 3,
-    "reusing the KV cache computed by a earlier layer"); kind and window of a
-    reader equal its owner's."""
+    paragraph on KV cache reuse); kind and window of a reader equal its owner's."""
     if len(layout) == 0:
         raise OracleError(ERR_INVALID_LAYOUT, "no layers")
     for l, (kind, window, owner) in enumerate(layout):
@@ -96,7 +95,7 @@ def key_range(kind: int, window: int, i: int) -> Tuple[int, int]:
 
 def rope_rotate(x, positions, theta: float) -> np.ndarray:
     """Rotary position embedding as defined by the RoFormer paper the method cites
-    (Section 4: "We used RoPE positional embeddings"): channel pairs (2i, 2i+1) of a
+    (Section 3, last paragraph: the models use rotary embeddings): channel pairs (2i, 2i+1) of a
     head vector at position m are rotated by the angle m * theta^(-2i/d).
 
     x [n, heads, d] (d even), positions [n] integers.  float64 throughout."""

@@ -3,8 +3,9 @@
 #include <math.h>
 #include <string.h>
 
-#include <new>
 #include <algorithm>
+#include <atomic>
+#include <new>
 #include <vector>
 
 #include "cache_manager.hpp"
@@ -177,19 +178,20 @@ int enqueue_append(mixattn_ctx* c, int layer, int n_seqs, const int32_t* seq_ids
   for (int i = 0; i < n_seqs; ++i) single = single && (n_new == nullptr || n_new[i] == 1);
   const int stride = c->cm.max_blocks();
   if (!ring && !single && !grants.empty()) {
-    // bulk append: push each sequence's new table entries, then let the kernel read the table
-    size_t a = 0;
-    while (a < grants.size()) {
-      size_t b = a;
-      while (b + 1 < grants.size() && grants[b + 1].seq == grants[a].seq) ++b;
-      const int32_t* src = c->cm.table_row(grants[a].seq) + grants[a].block;
-      int32_t* dst = c->dev_table() + (size_t)grants[a].seq * stride + grants[a].block;
-      if (cudaMemcpyAsync(dst, src, (b - a + 1) * sizeof(int32_t), cudaMemcpyHostToDevice, st) !=
-          cudaSuccess) {
-        c->sticky_cuda_error = true;
-        return MIXATTN_ERR_CUDA;
+    // bulk append: the new table entries travel in kernel parameters (no host copy that would
+    // wait for the stream or depend on pageable memory) and are set by a small kernel ahead of
+    // the copy kernel, which reads the table
+    TableSetParams tp;
+    tp.table = c->dev_table();
+    for (size_t a = 0; a < grants.size(); a += kTableSetMax) {
+      const size_t n = grants.size() - a < (size_t)kTableSetMax ? grants.size() - a : (size_t)kTableSetMax;
+      for (size_t i = 0; i < n; ++i) {
+        tp.idx[i] = grants[a + i].seq * stride + grants[a + i].block;
+        tp.page[i] = grants[a + i].page;
       }
-      a = b + 1;
+      tp.n = (int32_t)n;
+      cudaError_t e = launch_recorded(c, MIXATTN_K_APPEND, st, [&] { return launch_table_set(tp, st); });
+      if (e != cudaSuccess) return MIXATTN_ERR_CUDA;
     }
   }
   AppendParams p;
@@ -380,6 +382,54 @@ static void set_l2_policy(const mixattn_ctx* c, int layer, DecodeParams* p) {
   p->l2_keep_bytes = (uint32_t)(window <= fits ? window : room);
 }
 
+// Split plan of one decode launch over sequences ids[0 .. nb): fills the per-sequence fields of
+// *p (seq_id, n_eff, chunk_len, chunk_base, n_seqs, total_items; group and head_chunks must be
+// set) and returns the number of split slots the launch writes; *any_split tells whether a
+// combine pass is needed.  Long caches are cut into splits of kSplitTokens keys (large splits
+// keep the per-item epilogue negligible; thousands of items balance over the SMs).  When there
+// are fewer (sequence, KV head) pairs than SMs, short caches are cut further, but only up to one
+// item per SM, so the launch stays a single wave.  Both decode entry points use this one
+// function, so they add the partial results in the same order.
+static int plan_splits(const mixattn_ctx* c, int layer, const int32_t* ids, int nb, DecodeParams* p,
+                       bool* any_split) {
+  const int Hkv = c->cfg.n_kv_heads;
+  int64_t total = 0;
+  for (int j = 0; j < nb; ++j) {
+    p->seq_id[j] = ids[j];
+    p->n_eff[j] = c->cm.n_attended(layer, ids[j]);
+    total += p->n_eff[j];
+  }
+  int64_t T = c->split_tokens > 0 ? (c->split_tokens + kPage - 1) / kPage * kPage : kSplitTokens;
+  int64_t t_min = (total + kWsExtraChunks - 1) / kWsExtraChunks;
+  t_min = (t_min + kPage - 1) / kPage * kPage;
+  if (T < t_min) T = t_min;
+  const int64_t pairs = (int64_t)nb * Hkv * p->head_chunks;
+  int64_t nc_wave = c->split_tokens > 0 ? 1 : c->sm_count / pairs;
+  if (nc_wave > kWsWaveChunks / nb) nc_wave = kWsWaveChunks / nb;   // the workspace bounds the extra splits
+  int base = 0;
+  *any_split = false;
+  for (int j = 0; j < nb; ++j) {
+    const int64_t n = p->n_eff[j];
+    int64_t nc = (n + T - 1) / T;
+    if (nc < nc_wave) {
+      int64_t by_len = n / kMinSplitTokens;
+      nc = by_len < nc_wave ? by_len : nc_wave;
+      if (nc < 1) nc = 1;
+    }
+    int64_t len = (n + nc - 1) / nc;
+    len = (len + kPage - 1) / kPage * kPage;
+    nc = (n + len - 1) / len;
+    p->chunk_base[j] = base;
+    p->chunk_len[j] = (int32_t)len;
+    base += (int)nc;
+    *any_split = *any_split || nc > 1;
+  }
+  p->chunk_base[nb] = base;
+  p->n_seqs = nb;
+  p->total_items = base * Hkv * p->head_chunks;
+  return base;
+}
+
 int mixattn_decode(mixattn_ctx* c, int32_t layer, int32_t n_seqs, const int32_t* seq_ids,
                    const void* q, void* out, void* stream) {
   if (c == nullptr || !c->cm.valid_layer(layer) || n_seqs < 0) return MIXATTN_ERR_INVALID_ARG;
@@ -418,43 +468,9 @@ int mixattn_decode(mixattn_ctx* c, int32_t layer, int32_t n_seqs, const int32_t*
 
   for (int i0 = 0; i0 < n_seqs; i0 += kMaxCallSeqs) {
     const int nb = n_seqs - i0 < kMaxCallSeqs ? n_seqs - i0 : kMaxCallSeqs;
-    int64_t total = 0;
-    for (int j = 0; j < nb; ++j) {
-      p.seq_id[j] = seq_ids[i0 + j];
-      p.n_eff[j] = c->cm.n_attended(layer, p.seq_id[j]);
-      total += p.n_eff[j];
-    }
-    // Split choice.  Long caches are cut into splits of kSplitTokens keys (large splits
-    // keep the per-item epilogue negligible; thousands of items balance over the SMs).
-    // When there are fewer (sequence, KV head) pairs than SMs, short caches are cut
-    // further, but only up to one item per SM, so the launch stays a single wave.
-    int64_t T = c->split_tokens > 0 ? (c->split_tokens + kPage - 1) / kPage * kPage : kSplitTokens;
-    int64_t t_min = (total + kWsExtraChunks - 1) / kWsExtraChunks;
-    t_min = (t_min + kPage - 1) / kPage * kPage;
-    if (T < t_min) T = t_min;
-    const int64_t pairs = (int64_t)nb * Hkv * p.head_chunks;
-    const int64_t nc_wave = c->split_tokens > 0 ? 1 : c->sm_count / pairs;
-    int base = 0;
     bool any_split = false;
-    for (int j = 0; j < nb; ++j) {
-      const int64_t n = p.n_eff[j];
-      int64_t nc = (n + T - 1) / T;
-      if (nc < nc_wave) {
-        int64_t by_len = n / kMinSplitTokens;
-        nc = by_len < nc_wave ? by_len : nc_wave;
-        if (nc < 1) nc = 1;
-      }
-      int64_t len = (n + nc - 1) / nc;
-      len = (len + kPage - 1) / kPage * kPage;
-      nc = (n + len - 1) / len;
-      p.chunk_base[j] = base;
-      p.chunk_len[j] = (int32_t)len;
-      base += (int)nc;
-      any_split = any_split || nc > 1;
-    }
-    p.chunk_base[nb] = base;
-    p.n_seqs = nb;
-    p.total_items = base * Hkv * p.head_chunks;
+    const int base = plan_splits(c, layer, seq_ids + i0, nb, &p, &any_split);
+    if (base > kWsChunks) return MIXATTN_ERR_UNSUPPORTED;   // (cannot happen: the plan is bounded by the workspace)
     p.q = static_cast<const char*>(q) + (size_t)i0 * Hq * D * esz;
     p.out = static_cast<char*>(out) + (size_t)i0 * Hq * D * esz;
     const int cls = ring ? MIXATTN_K_DECODE_SLIDING : MIXATTN_K_DECODE_FULL;
@@ -505,14 +521,6 @@ int mixattn_prefill(mixattn_ctx* c, int32_t layer, int32_t n_seqs, const int32_t
   DeviceGuard g(c->device);
   if (!g.ok) return MIXATTN_ERR_CUDA;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  if (owner) {
-    std::vector<int32_t> start(n_seqs, 0);
-    std::vector<PageGrant> grants;
-    c->cm.apply_append(layer, n_seqs, seq_ids, seq_lens, &grants);
-    ++c->cache_epoch;
-    int rc = enqueue_append(c, layer, n_seqs, seq_ids, seq_lens, start, grants, k, v, st);
-    if (rc != MIXATTN_OK) return rc;
-  }
   const int Hq = c->cfg.n_q_heads, Hkv = c->cfg.n_kv_heads, D = c->cfg.head_dim;
   const size_t esz = c->geom.elem_bytes;
   PrefillParams p;
@@ -548,6 +556,17 @@ int mixattn_prefill(mixattn_ctx* c, int32_t layer, int32_t n_seqs, const int32_t
       return tc ? launch_prefill_tc(p, mlen, c->sm_count, st) : launch_prefill_simple(p, c->cfg.dtype, mlen, st);
     });
     if (e != cudaSuccess) return MIXATTN_ERR_CUDA;
+  }
+  // The attention reads the caller's tensors, not the cache, so the cache is written after it:
+  // the bookkeeping moves only once every attention launch (tensor maps included) has been
+  // accepted.  A CUDA failure past this point leaves the context unusable (see the header).
+  if (owner) {
+    std::vector<int32_t> start(n_seqs, 0);
+    std::vector<PageGrant> grants;
+    c->cm.apply_append(layer, n_seqs, seq_ids, seq_lens, &grants);
+    ++c->cache_epoch;
+    int rc = enqueue_append(c, layer, n_seqs, seq_ids, seq_lens, start, grants, k, v, st);
+    if (rc != MIXATTN_OK) return rc;
   }
   return MIXATTN_OK;
 }
@@ -844,16 +863,19 @@ static __device__ __align__(256) unsigned char g_decode_scratch[kStaticScratchBy
 // Device address of g_decode_scratch per device ordinal.  In host code the array's name
 // is only a handle for the runtime; the address a kernel can use comes from
 // cudaGetSymbolAddress, asked once per device with that device current.
-void* g_decode_scratch_ptr[kMaxDevices] = {};
+// Contexts on several threads may make their first call at once: the slots are atomic (every
+// thread that asks gets the same address, so a relaxed load / store is enough).  The address is
+// kept until the process exits; it does not survive a cudaDeviceReset of that device.
+std::atomic<void*> g_decode_scratch_ptr[kMaxDevices];
 
 int static_scratch_for_current_device(int device, void** out) {
   if (device < 0 || device >= kMaxDevices) return MIXATTN_ERR_INVALID_ARG;
-  if (g_decode_scratch_ptr[device] == nullptr) {
-    void* ptr = nullptr;
+  void* ptr = g_decode_scratch_ptr[device].load(std::memory_order_relaxed);
+  if (ptr == nullptr) {
     if (cudaGetSymbolAddress(&ptr, g_decode_scratch) != cudaSuccess || ptr == nullptr) return MIXATTN_ERR_CUDA;
-    g_decode_scratch_ptr[device] = ptr;
+    g_decode_scratch_ptr[device].store(ptr, std::memory_order_relaxed);
   }
-  *out = g_decode_scratch_ptr[device];
+  *out = ptr;
   return MIXATTN_OK;
 }
 
@@ -880,38 +902,10 @@ int mixattn_decode_static_scratch(mixattn_ctx* c, int32_t layer, int32_t n_seqs,
   DecodeParams p;
   p.group = Hq / Hkv;
   p.head_chunks = (p.group + kMaxGroupRows - 1) / kMaxGroupRows;
-  // same split plan as mixattn_decode, so both calls add the partial results in the same order
-  int64_t total = 0;
-  for (int j = 0; j < n_seqs; ++j) {
-    p.seq_id[j] = seq_ids[j];
-    p.n_eff[j] = c->cm.n_attended(layer, p.seq_id[j]);
-    total += p.n_eff[j];
-  }
-  int64_t T = c->split_tokens > 0 ? (c->split_tokens + kPage - 1) / kPage * kPage : kSplitTokens;
-  int64_t t_min = (total + kWsExtraChunks - 1) / kWsExtraChunks;
-  t_min = (t_min + kPage - 1) / kPage * kPage;
-  if (T < t_min) T = t_min;
-  const int64_t pairs = (int64_t)n_seqs * Hkv * p.head_chunks;
-  const int64_t nc_wave = c->split_tokens > 0 ? 1 : c->sm_count / pairs;
-  int base = 0;
+  // the split plan of mixattn_decode (one function), so both calls add the partial results in
+  // the same order and give the same bits
   bool any_split = false;
-  for (int j = 0; j < n_seqs; ++j) {
-    const int64_t n = p.n_eff[j];
-    int64_t nc = (n + T - 1) / T;
-    if (nc < nc_wave) {
-      int64_t by_len = n / kMinSplitTokens;
-      nc = by_len < nc_wave ? by_len : nc_wave;
-      if (nc < 1) nc = 1;
-    }
-    int64_t len = (n + nc - 1) / nc;
-    len = (len + kPage - 1) / kPage * kPage;
-    nc = (n + len - 1) / len;
-    p.chunk_base[j] = base;
-    p.chunk_len[j] = (int32_t)len;
-    base += (int)nc;
-    any_split = any_split || nc > 1;
-  }
-  p.chunk_base[n_seqs] = base;
+  const int base = plan_splits(c, layer, seq_ids, n_seqs, &p, &any_split);
   // scratch needed: per split and query head, D partial outputs + (max, sum)
   const size_t part_o_bytes = align_up((size_t)base * Hq * D * sizeof(float));
   const size_t need = part_o_bytes + (size_t)base * Hq * sizeof(float2);
@@ -939,8 +933,6 @@ int mixattn_decode_static_scratch(mixattn_ctx* c, int32_t layer, int32_t n_seqs,
   p.part_o = reinterpret_cast<float*>(scratch);
   p.part_ml = reinterpret_cast<float2*>(static_cast<char*>(scratch) + part_o_bytes);
   p.status = c->dev_status();
-  p.n_seqs = n_seqs;
-  p.total_items = base * Hkv * p.head_chunks;
   const int cls = ring ? MIXATTN_K_DECODE_SLIDING : MIXATTN_K_DECODE_FULL;
   cudaError_t e = launch_recorded(c, cls, st, [&] {
     return c->cfg.dtype == MIXATTN_BF16 ? launch_decode_split_bf16(p, c->sm_count, st)

@@ -15,7 +15,7 @@ constexpr int kThreads = 256;
 constexpr int kTokensPerBlock = 8;
 
 // Rotary position embedding of one 16-byte chunk of a key row (RoFormer's definition, which
-// Section 4 of the paper cites): channel pair (2i, 2i+1) at position m turns by the angle
+// Section 3 of the paper cites): channel pair (2i, 2i+1) at position m turns by the angle
 // m * theta^(-2i/d).  The angle is formed and reduced modulo 2 pi in double precision
 // (positions reach 10^5 and the first pairs turn by about a radian per position), the
 // rotation itself runs in fp32, and bf16 rows are rounded once.
@@ -89,7 +89,18 @@ __global__ void __launch_bounds__(kThreads) append_kernel(const __grid_constant_
   }
 }
 
+__global__ void __launch_bounds__(kThreads) table_set_kernel(const __grid_constant__ TableSetParams p) {
+  const int i = blockIdx.x * kThreads + threadIdx.x;
+  if (i < p.n) p.table[p.idx[i]] = p.page[i];
+}
+
 }  // namespace
+
+cudaError_t launch_table_set(const TableSetParams& p, cudaStream_t st) {
+  if (p.n <= 0) return cudaSuccess;
+  table_set_kernel<<<(p.n + kThreads - 1) / kThreads, kThreads, 0, st>>>(p);
+  return cudaGetLastError();
+}
 
 cudaError_t launch_append(const AppendParams& p, int max_n_new, cudaStream_t st) {
   if (p.n_entries <= 0) return cudaSuccess;

@@ -72,6 +72,7 @@ class CacheManager {
     if (msl < 1) msl = 1;
     max_seq_len_ = (int32_t)msl;
     max_blocks_ = (max_seq_len_ + kPageSize - 1) / kPageSize;
+    if ((int64_t)max_seqs_ * max_blocks_ > INT32_MAX) return MIXATTN_ERR_INVALID_ARG;   // table entries are indexed in 32 bits
     free_.clear();
     if (cfg.free_order) {
       std::vector<char> seen(cfg.n_pages, 0);

@@ -12,7 +12,8 @@ constexpr int kPage = 16;          // tokens per page (paged pools and rings ali
 constexpr int kMaxCallSeqs = 128;  // sequences per kernel launch (metadata travels in kernel params)
 constexpr int kMaxGroupRows = 8;   // query heads of one KV head handled by one work item
 constexpr int kWsExtraChunks = 1024;                        // splits beyond one per sequence
-constexpr int kWsChunks = kMaxCallSeqs + kWsExtraChunks + 256;  // split slots in the workspace (256: single-wave splits)
+constexpr int kWsWaveChunks = 256;                          // splits added to fill a single wave of SMs
+constexpr int kWsChunks = kMaxCallSeqs + kWsExtraChunks + kWsWaveChunks;  // split slots in the workspace
 
 // ---------------------------------------------------------------------------
 // K/V storage format.
@@ -151,11 +152,21 @@ struct GatherParams {
   GatherEntry e[kMaxCallSeqs];
 };
 
+// Block-table entries a bulk append sets on the device before its copy kernel reads them.
+constexpr int kTableSetMax = 1024;
+struct TableSetParams {
+  int32_t* table;
+  int32_t n;
+  int32_t idx[kTableSetMax];    // entry index: seq * table_stride + logical block
+  int32_t page[kTableSetMax];
+};
+
 // device status codes written to the status word
 enum { kDevOk = 0, kDevWaitTimeout = 1 };
 
 // launchers (each returns the cudaError_t of its launch)
 cudaError_t launch_append(const AppendParams& p, int max_n_new, cudaStream_t st);
+cudaError_t launch_table_set(const TableSetParams& p, cudaStream_t st);
 cudaError_t launch_gather(const GatherParams& p, int max_rows, cudaStream_t st);
 cudaError_t prepare_decode_bf16();
 cudaError_t launch_decode_split_bf16(const DecodeParams& p, int sm_count, cudaStream_t st);

@@ -68,7 +68,7 @@ def owners_of(layout: List[Layer]) -> List[int]:
 
 
 # ---------------------------------------------------------------------------
-# The paper's named variants (Section 4).  The text fixes, per variant, how many standard
+# The paper's named variants (Sections 5.1 and 5.2, Appendix A).  The text fixes, per variant, how many standard
 # attention caches there are, which layer computes them and who shares them; the figures
 # that drew the exact layer indices are not part of the text.  What the text leaves open is
 # a parameter here, with defaults that follow the pattern it cites (a standard layer every
@@ -153,6 +153,23 @@ def layout_noshare(n_layers: int = 24, window: int = 1024, n_full: int = 1, offs
     return layout_from_roles(n_layers, window, full, {l: l for l in full}, ring_groups)
 
 
+def layout_ma_successive(n_layers: int = 24, window: int = 1024, first: int = 0, gap: int = 12, n_pairs: int = 2,
+                         ring_groups=(3, 2)) -> List[Layer]:
+    """MA-Successive-k (Appendix A.1): standard caches shared between CONSECUTIVE layers.  Pair p
+    sits at layers (first + p * gap, first + p * gap + 1): the first computes a standard cache,
+    the next reads it.  The four variants differ in where the pairs sit (`first`) and how far
+    apart they are (`gap`); the figure that drew them is not part of the text, so both are
+    parameters."""
+    own = {}
+    for p in range(n_pairs):
+        a = first + p * gap
+        if a + 1 >= n_layers:
+            raise ValueError("pair does not fit the model")
+        own[a] = a
+        own[a + 1] = a
+    return layout_from_roles(n_layers, window, sorted(own), own, ring_groups)
+
+
 PAPER_VARIANTS = {
     "standard": lambda: layout_all_full(24),
     "sliding_window": lambda: layout_all_sliding(24, 1024),
@@ -165,6 +182,10 @@ PAPER_VARIANTS = {
     "MA-NoShare-1": lambda: layout_noshare(n_full=1),
     "MA-NoShare-2": lambda: layout_noshare(n_full=2, offset=2, step=12),
     "MA-NoShare-3": lambda: layout_noshare(n_full=3, offset=2, step=8),
+    "MA-Successive-1": lambda: layout_ma_successive(first=0, gap=12),
+    "MA-Successive-2": lambda: layout_ma_successive(first=2, gap=12),
+    "MA-Successive-3": lambda: layout_ma_successive(first=2, gap=6),
+    "MA-Successive-4": lambda: layout_ma_successive(first=6, gap=12),
 }
 
 

@@ -36,7 +36,7 @@ def test_capacity_matches_closed_form_and_sharing_law():
 
 
 def test_named_variants_have_the_properties_the_paper_states():
-    # Section 4 fixes these facts in words; the exact layer indices (figures) are parameters
+    # Sections 5.1 and 5.2 fix these facts in words; the exact layer indices (figures) are parameters
     V = {k: f() for k, f in cf.PAPER_VARIANTS.items()}
     for name, lay in V.items():
         assert len(lay) == 24
@@ -67,6 +67,16 @@ def test_named_variants_have_the_properties_the_paper_states():
     for k in (1, 2, 3):
         lay = V[f"MA-NoShare-{k}"]
         assert full_owners(lay) == full_layers(lay) and len(full_layers(lay)) == k
+    # Successive-k (Appendix A.1): standard layers come in consecutive pairs, the second reading the
+    # first's cache; the variants differ in the pairs' positions and distance, MA-Pairs-like otherwise
+    seen = set()
+    for k in (1, 2, 3, 4):
+        lay = V[f"MA-Successive-{k}"]
+        owners, layers = full_owners(lay), full_layers(lay)
+        assert len(owners) == 2 and layers == sorted(owners + [o + 1 for o in owners])
+        assert all(lay[o + 1] == (cf.FULL, 0, o) for o in owners)
+        seen.add((owners[0], owners[1] - owners[0]))
+    assert len(seen) == 4 and len({g for _, g in seen}) > 1 and len({f for f, _ in seen}) > 1
     # cache bytes: every MixAttention variant is far below the standard model at 32K tokens
     tab = capacity.capacity_table(V, 12, 3, 128, mx.BF16, 32000, 80 * 10**9)
     for name in V:

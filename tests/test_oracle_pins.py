@@ -434,3 +434,42 @@ def test_rope_closed_forms_and_relative_position_property():
         np.testing.assert_allclose(np.hypot(qm[..., 0::2], qm[..., 1::2]), np.hypot(q[..., 0::2], q[..., 1::2]), atol=1e-12)
         ref = float((mo.rope_rotate(q, [m - n_], theta) * k).sum())
         assert abs(float((qm * kn).sum()) - ref) < 1e-9
+
+
+def test_logical_cache_prefill_records_for_owners_only():
+    """LogicalCache.prefill: output is the dense masked reference; an owner records the
+    prompt's K/V under ITS OWN layer (a later decode of owner and reader sees prompt + new
+    token), a reader records nothing, and a non-empty owner cache is refused."""
+    rng = np.random.default_rng(21)
+    S, Hq, Hkv, D, W = 19, 4, 2, 8, 5
+    layout = [(FULL, 0, 0), (SLIDING, W, 1), (SLIDING, W, 1), (FULL, 0, 0)]
+    lc = mo.LogicalCache(layout, Hq, Hkv, D)
+    K = {0: rnd(rng, S, Hkv, D), 1: rnd(rng, S, Hkv, D)}
+    V = {0: rnd(rng, S, Hkv, D), 1: rnd(rng, S, Hkv, D)}
+    for layer, (kind, window, owner) in enumerate(layout):
+        q = rnd(rng, S, Hq, D)
+        before = {k: (v[0].shape[0]) for k, v in lc.hist.items()}
+        out = lc.prefill(layer, 0, q, K[owner], V[owner])
+        np.testing.assert_allclose(out, dense_reference(q, K[owner], V[owner], kind, window), rtol=0, atol=1e-12)
+        if owner == layer:
+            assert set(lc.hist) - set(before) == {(layer, 0)}
+            np.testing.assert_array_equal(lc.hist[(layer, 0)][0], K[layer])
+            np.testing.assert_array_equal(lc.hist[(layer, 0)][1], V[layer])
+        else:   # a reader stores nothing
+            assert {k: v[0].shape[0] for k, v in lc.hist.items()} == before
+    # the recorded prompt is what a following decode step sees, for owner and reader alike
+    k1, v1 = rnd(rng, 1, Hkv, D), rnd(rng, 1, Hkv, D)
+    lc.append(1, 0, k1, v1)
+    qd = rnd(rng, Hq, D)
+    Kall, Vall = np.concatenate([K[1], k1]), np.concatenate([V[1], v1])
+    qs = np.zeros((S + 1, Hq, D))
+    qs[S] = qd
+    ref = dense_reference(qs, Kall, Vall, SLIDING, W)[S]
+    for layer in (1, 2):
+        np.testing.assert_allclose(lc.decode(layer, 0, qd), ref, rtol=0, atol=1e-12)
+    # the other sequence slot is untouched; a second prompt into a filled owner is refused
+    assert lc.history(0, 1)[0].shape[0] == 0
+    with pytest.raises(mo.OracleError) as ei:
+        lc.prefill(0, 0, rnd(rng, S, Hq, D), K[0], V[0])
+    assert ei.value.code == mo.ERR_UNSUPPORTED
+    assert lc.history(0, 0)[0].shape[0] == S

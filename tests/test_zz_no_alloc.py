@@ -6,9 +6,12 @@ buffer sized for the caches only, an allocator that must not be re-entered).
 For them the library has a decode entry point whose split-KV partial results
 live in a static device array.  This test drives that entry point through the
 C ABI on a cache with several splits per sequence, twice in a row (the array
-keeps the first call's contents), and requires the same outputs as
-mixattn_decode within the bf16 tolerance of the other GPU tests; it also checks
-that an oversized request is refused without a launch.
+keeps the first call's contents), and requires the outputs of mixattn_decode:
+within the bf16 tolerance of the other GPU tests, and, because both entry
+points share one split planner and so add the partial results in the same
+order, bit for bit.  The device's free-memory figure must be the same before
+and after the call (nothing was allocated), and an oversized request must be
+refused without a launch.
 
 The file name sorts last on purpose: a run that stops at the first failure has
 then already run every other test.
@@ -44,14 +47,19 @@ def test_static_scratch_decode_matches_decode_twice():
                 got = torch.full_like(ref, float("nan"))
                 sess.ctx.decode(l, ids, ent["q"], ref)
                 launches = sess.ctx.get_launch_count()
+                torch.cuda.synchronize()
+                free_before = torch.cuda.mem_get_info()[0]
                 rc = sess.ctx.rc_decode_static_scratch(l, ids, ent["q"], got)
                 assert rc == 0, mx.strerror(rc)
                 assert sess.ctx.get_launch_count() - launches == 2      # split pass + combine pass
                 torch.cuda.synchronize()
+                if call > 0 or l > 0:   # (the very first call may load the kernels' module)
+                    assert torch.cuda.mem_get_info()[0] == free_before, "the call changed the device's free memory"
                 a, b = got.float().cpu().numpy(), ref.float().cpu().numpy()
                 assert np.isfinite(a).all()
                 err = np.abs(a - b)
                 assert err.max() <= tol["max_abs"] and err.mean() <= tol["mean_abs"], (call, l, err.max())
+                assert torch.equal(got.view(torch.int16), ref.view(torch.int16)), (call, l, "bits differ")
             sess.pos += 1
         assert sess.ctx.get_device_status() == 0
 
