@@ -151,6 +151,42 @@ def test_prefill_full_size_sampled_rows():
         sess.close()
 
 
+def test_prefill_full_size_every_row_of_one_sequence():
+    # one standard layer (12) and one sliding-window layer (2) of the prefill configuration,
+    # checked on ALL 8192 query rows of one sequence for one head of each of the eight KV
+    # groups: every work item of the persistent kernel (64 query tiles per head, up to 64 key
+    # tiles per row of tiles) is covered for those heads, not a sample of them
+    mx, runner = load_lib()
+    wl = cf.prefill_chunk()
+    sess = runner.Session(wl, [0] * wl.batch)
+    S = wl.seq_len
+    G = wl.n_q_heads // wl.n_kv_heads
+    hist = HeadHistory(wl)
+    b = 1
+    heads = (0, 5, 10, 15, 17, 22, 27, 31)   # one head of each of the eight KV groups
+    scale = 1.0 / np.sqrt(wl.head_dim)
+    try:
+        for l in (12, 2):
+            kind, Wl, owner = wl.layout[l]
+            assert owner != l          # readers: the call stores nothing
+            q, k, v = sess.prefill_inputs(l)
+            out = torch.full_like(q, float("nan"))
+            sess.prefill_layer(l, q, k, v, out)
+            torch.cuda.synchronize()
+            got = out.view(wl.batch, S, wl.n_q_heads, wl.head_dim)[b].float().cpu().double().numpy()
+            qc = si.q_tokens(wl.seed, l, b, 0, S, wl.n_q_heads, wl.head_dim, torch_dt(wl.dtype)).double().numpy()
+            for h in heads:
+                K, V = hist.get(owner, b, h // G, S)
+                ref = np.empty((S, wl.head_dim))
+                for i in range(S):
+                    lo, hi = mo.key_range(kind, Wl, i)
+                    ref[i] = mo.softmax_attend(qc[i, h], K[lo:hi], V[lo:hi], scale)
+                check_close(got[:, h], ref, wl.dtype, f"prefill layer {l} seq {b} head {h}, all rows")
+        assert sess.ctx.get_device_status() == 0
+    finally:
+        sess.close()
+
+
 def test_prefill_served_in_chunks_full_size_sampled_rows():
     # the prefill configuration's prompts (batch 4 x 8192) served in chunks of 2048 behind the cached
     # prefix, in the launch configuration bench.py times; sampled rows of sampled heads per round

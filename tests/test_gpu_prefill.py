@@ -209,3 +209,42 @@ def test_many_short_prompts_repeated_calls():
         assert sess.ctx.get_device_status() == 0
     finally:
         sess.close()
+
+
+def test_prefill_bf16_error_budget_over_seeds(capsys):
+    # The tensor-core prompt kernel against the checker over several seeds, with the error split
+    # into the part no bf16 kernel can avoid (rounding the exact result to bf16: |bf16(ref) - ref|)
+    # and the kernel's own arithmetic (|got - bf16(ref)|: bf16 weights in the P V product, fp32
+    # accumulation order, approximate exponentials).  The tolerances are the usual ones; the two
+    # parts are printed (run with -s) so that the margin under the absolute bound is on record.
+    mx, runner = load_lib()
+    worst = dict(total=0.0, rounding=0.0, arithmetic=0.0)
+    for seed in (3, 11, 12, 13, 14, 15):
+        wl = cf.prefill_chunk().scaled(layout=cf.layout_tiny(128), batch=2, seq_len=300, seed=seed)
+        sess = runner.Session(wl, [0] * wl.batch, headroom_tokens=2)
+        dt = torch_dt(wl.dtype)
+        S = wl.seq_len
+        try:
+            for l, (kind, W, owner) in enumerate(wl.layout):
+                q, k, v = sess.prefill_inputs(l)
+                out = torch.full_like(q, float("nan"))
+                sess.prefill_layer(l, q, k, v, out)
+                torch.cuda.synchronize()
+                got = out.float().cpu().double().numpy().reshape(wl.batch, S, wl.n_q_heads, wl.head_dim)
+                for b in range(wl.batch):
+                    qc = si.q_tokens(wl.seed, l, b, 0, S, wl.n_q_heads, wl.head_dim, dt)
+                    Kc, Vc = si.kv_tokens(wl.seed, owner, b, 0, S, wl.n_kv_heads, wl.head_dim, dt)
+                    ref = mo.prefill_attention(qc, Kc, Vc, kind, W)
+                    check_close(got[b], ref, wl.dtype, f"seed {seed} layer {l} seq {b}")
+                    ref_bf16 = torch.from_numpy(ref).to(torch.bfloat16).double().numpy()
+                    worst["total"] = max(worst["total"], float(np.abs(got[b] - ref).max()))
+                    worst["rounding"] = max(worst["rounding"], float(np.abs(ref_bf16 - ref).max()))
+                    worst["arithmetic"] = max(worst["arithmetic"], float(np.abs(got[b] - ref_bf16).max()))
+            assert sess.ctx.get_device_status() == 0
+        finally:
+            sess.close()
+    with capsys.disabled():
+        print(f"\nprefill bf16 error budget over 6 seeds: max-abs {worst['total']:.3e} = output rounding "
+              f"{worst['rounding']:.3e} + kernel arithmetic {worst['arithmetic']:.3e} (bound 1e-2)")
+    # rounding the exact result of magnitude 2..4 to bf16 costs up to 2^-7 = 7.8e-3 by itself
+    assert worst["rounding"] <= 2.0 ** -7
