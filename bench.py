@@ -38,13 +38,14 @@ from synth import configs as cf
 from synth import inputs as si
 
 METRIC = "decode attention HBM GB/s (% of peak) & tokens/s; prefill TFLOP/s (% bf16 peak)"
+NOMINAL_BF16_TFLOPS = 2250.0     # dense bf16 datasheet figure of a B200 (context; fractions of it are reported too)
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
-# (dram__bytes_read.sum + dram__bytes_write.sum) / algorithmic KV bytes of the dominant kernel, from the
-# ncu capture of a batch-4 launch summarised in profiles/decode_split_bf16_kernel.mid_decode.md
-# (541.30 MB moved for 536.95 MB of keys and values).  DRAM traffic grows in proportion to the keys read,
-# so the full-size figure is this ratio times the launch's algorithmic bytes.  Set to None when the
-# kernel changes until the counters are taken again.
+# (dram__bytes_read.sum + dram__bytes_write.sum) / algorithmic KV bytes of the dominant kernel, from an
+# ncu capture of one standard-layer launch at batch 4 (541.30 MB moved for 536.95 MB of keys and values;
+# the full-size launch holds too much device memory for a multi-pass capture).  DRAM traffic grows in
+# proportion to the keys read, so the full-size figure is this ratio times the launch's algorithmic
+# bytes.  Set to None when the kernel changes until the counters are taken again.
 DECODE_FULL_TRAFFIC_RATIO = 541.304832 / 536.952832
 
 
@@ -77,7 +78,8 @@ class ClockSampler:
     def __init__(self, index: int):
         self.index = index
         self.proc = None
-        self.lines = []
+        self.lines = []          # (host time, csv line)
+        self.t_lo = self.t_hi = None
 
     def start(self):
         try:
@@ -92,7 +94,13 @@ class ClockSampler:
 
     def _read(self):
         for line in self.proc.stdout:
-            self.lines.append(line.strip())
+            self.lines.append((time.perf_counter(), line.strip()))
+
+    def mark_begin(self):
+        self.t_lo = time.perf_counter()
+
+    def mark_end(self):
+        self.t_hi = time.perf_counter()
 
     def stop(self):
         if self.proc is None:
@@ -102,22 +110,29 @@ class ClockSampler:
             self.proc.wait(timeout=5)
         except Exception:
             self.proc.kill()
-        sm, mx, reasons = [], None, set()
+        sm, sm_all, mx, reasons = [], [], None, set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for ln in self.lines:
+        for t, ln in self.lines:
             parts = [p.strip() for p in ln.split(",")]
             if len(parts) < 6:
                 continue
             try:
-                sm.append(float(parts[0]))
+                mhz = float(parts[0])
                 mx = float(parts[1])
             except ValueError:
                 continue
+            sm_all.append(mhz)
+            # a sample belongs to the timed part when it was read between the two marks (the
+            # query itself takes a few milliseconds, hence the small allowance at the end)
+            if self.t_lo is not None and self.t_hi is not None and not (self.t_lo <= t <= self.t_hi + 0.03):
+                continue
+            sm.append(mhz)
             for nm, val in zip(names, parts[2:6]):
                 if val.lower().startswith("active"):
                     reasons.add(nm)
         return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": mx,
-                "reasons": sorted(reasons), "samples": len(sm)}
+                "reasons": sorted(reasons), "samples": len(sm), "samples_whole_run": len(sm_all),
+                "sm_mhz_whole_run": float(np.median(sm_all)) if sm_all else None}
 
 
 # ---------------------------------------------------------------------------
@@ -215,8 +230,9 @@ def prefill_figures(mx, runner, peaks, device):
                                         ("sliding", 2, pairs_slide, mx.K_PREFILL_SLIDING)):
             q, k, v = sess.prefill_inputs(layer)      # readers: no cache writes, repeatable
             out = torch.empty_like(q)
-            reps = 3
-            sess.prefill_layer(layer, q, k, v, out)
+            reps = 20
+            for _ in range(3):
+                sess.prefill_layer(layer, q, k, v, out)
             torch.cuda.synchronize()
             sess.ctx.profile_enable(True)
             for _ in range(reps):
@@ -226,9 +242,13 @@ def prefill_figures(mx, runner, peaks, device):
             flops = 4.0 * D * pairs * Hq * B
             tf = flops / (ms / n * 1e-3) / 1e12
             res[name] = {"ms_per_layer": ms / n, "tflops": tf, "frac_of_bf16_peak": tf / peaks["bf16_tflops"],
-                         "useful_flop": flops}
+                         "frac_of_nominal_2250": tf / NOMINAL_BF16_TFLOPS, "useful_flop": flops, "launches_timed": n}
         res["config"] = {"workload": wl.name, "batch": B, "seq_len": S, "window": W}
+        # the stated target (sliding-window layer at half the bf16 dense peak) read both ways
+        res["target_half_of_nominal_met"] = res["sliding"]["frac_of_nominal_2250"] >= 0.5
+        res["target_half_of_measured_met"] = res["sliding"]["frac_of_bf16_peak"] >= 0.5
         res["peak_tflops"] = peaks["bf16_tflops"]
+        res["nominal_tflops"] = NOMINAL_BF16_TFLOPS
         res["peak_source"] = peaks["_source"]
     finally:
         sess.close()
@@ -256,8 +276,9 @@ def chunk_figures(mx, runner, peaks, device, prefix=6144, chunk=2048):
             K, V = si.kv_tokens_multi(wl.seed, owner, ids, [prefix] * B, chunk, wl.n_kv_heads, D, sess.dt, sess.dev)
             K, V = K.reshape(-1, wl.n_kv_heads, D), V.reshape(-1, wl.n_kv_heads, D)
             out = torch.empty_like(q)
-            reps = 3
-            sess.ctx.attend_chunk(layer, ids, lens, q, K, V, out)
+            reps = 10
+            for _ in range(2):
+                sess.ctx.attend_chunk(layer, ids, lens, q, K, V, out)
             torch.cuda.synchronize()
             sess.ctx.profile_enable(True)
             for _ in range(reps):
@@ -268,7 +289,8 @@ def chunk_figures(mx, runner, peaks, device, prefix=6144, chunk=2048):
             flops = 4.0 * D * pairs * Hq * B
             t = (ms / n + msg / ng) * 1e-3
             res[name] = {"ms_attention": ms / n, "ms_gather": msg / ng, "tflops": flops / t / 1e12,
-                         "frac_of_bf16_peak": flops / t / 1e12 / peaks["bf16_tflops"], "useful_flop": flops}
+                         "frac_of_bf16_peak": flops / t / 1e12 / peaks["bf16_tflops"],
+                         "frac_of_nominal_2250": flops / t / 1e12 / NOMINAL_BF16_TFLOPS, "useful_flop": flops}
         # the same chunk through all 24 layers, each reader handed its owner's K/V, with the copy of
         # the cached keys shared by the layers that read one cache (4 copies: F, S1, F, S2)
         sess.ctx.set_chunk_gather_reuse(True)
@@ -309,6 +331,116 @@ def reduce_over_ranks(dist, times, work, device):
     return t.tolist(), w.tolist()
 
 
+MIN_TIMED_S = 0.4        # the K-step region is repeated until this much device time has been timed
+MAX_EXTRA_STEPS = 600    # at most this many steps beyond the first region
+
+
+def n_regions_for(region_ms: float, K: int) -> int:
+    """How many K-step regions to time so that the timed part spans at least MIN_TIMED_S (a
+    region of a few tens of milliseconds is shorter than two ticks of the clock sampler)."""
+    if region_ms <= 0:
+        return 1
+    want = int(np.ceil(MIN_TIMED_S * 1e3 / region_ms))
+    return max(1, min(want, 1 + MAX_EXTRA_STEPS // max(K, 1)))
+
+
+def make_session(runner, wl, device, total_steps):
+    """Session with the workload's lengths drawn, its page order permuted if asked, caches filled."""
+    if wl.context_range != (0, 0):
+        lengths = si.draw_lengths(wl.seed, wl.batch, *wl.context_range).tolist()
+    else:
+        lengths = [wl.context] * wl.batch
+    free_order = None
+    if wl.permute_pages:
+        n_pages = sum(-(-(n + total_steps) // wl.page_size) for n in lengths)
+        free_order = si.page_permutation(wl.seed, n_pages)
+    sess = runner.Session(wl, lengths, device=device, headroom_tokens=total_steps, free_order=free_order)
+    sess.fill(1024)
+    return sess, lengths
+
+
+def step_input_ring(sess, n):
+    """n distinct seeded steps' inputs, reused cyclically (the values do not change the work;
+    positions, appends and lengths advance every step as in serving)."""
+    ring = []
+    pos_save = sess.pos.copy()
+    for _ in range(n):
+        ring.append(sess.step_inputs())
+        sess.pos += 1
+    sess.pos[:] = pos_save
+    return ring
+
+
+def device_pass(sess, runner, wl, ring, outs, stream, K, Wm, barrier, sampler=None):
+    """Wm warm-up steps, then regions of exactly K decode steps between CUDA events on the
+    launching stream, inputs resident in HBM.  The first region decides how many more follow
+    (n_regions_for).  Returns (mean ms per region, mean KV bytes per region, regions, launches
+    per region)."""
+    def bytes_next_step():
+        return runner.kv_bytes_per_step(wl, [int(p) + 1 for p in sess.pos])
+
+    step = 0
+    for _ in range(Wm):
+        sess.decode_step(ring[step % len(ring)], outs, stream)
+        step += 1
+    launches0 = sess.ctx.get_launch_count()
+    barrier()
+    if sampler is not None:
+        sampler.mark_begin()
+    events, nbytes = [], []
+
+    def region():
+        nonlocal step
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        b = 0
+        e0.record(stream)
+        for _ in range(K):
+            b += bytes_next_step()
+            sess.decode_step(ring[step % len(ring)], outs, stream)
+            step += 1
+        e1.record(stream)
+        events.append((e0, e1))
+        nbytes.append(b)
+
+    region()
+    torch.cuda.synchronize()
+    more = n_regions_for(events[0][0].elapsed_time(events[0][1]), K) - 1
+    for _ in range(more):
+        region()
+    barrier()
+    if sampler is not None:
+        sampler.mark_end()
+    ms = [a.elapsed_time(b) for a, b in events]
+    launches = (sess.ctx.get_launch_count() - launches0) / len(events)
+    assert sess.ctx.get_device_status() == 0, "a kernel reported a wait time-out"
+    return float(np.mean(ms)), float(np.mean(nbytes)), len(events), launches
+
+
+def other_workload_figures(runner, peaks, device, K, Wm):
+    """The other decode configurations, device-resident, in compact form: long-context decode,
+    its variant with rings shared in pairs, and the mixed serving batch."""
+    res = {}
+    for name in ("long_decode", "long_decode_pairs", "mixed_serving"):
+        wl = get_workload(name)
+        total = Wm + K + MAX_EXTRA_STEPS + 2
+        sess, lengths = make_session(runner, wl, device, total)
+        try:
+            ring = step_input_ring(sess, min(4, Wm + K))
+            outs = sess.alloc_outputs()
+            stream = torch.cuda.current_stream()
+            ms, nbytes, regions, launches = device_pass(sess, runner, wl, ring, outs, stream, K, Wm,
+                                                        torch.cuda.synchronize)
+            gbs = nbytes / (ms * 1e-3) / 1e9
+            res[wl.name] = {"gbs": gbs, "ms_per_step": ms / K, "frac_of_measured_hbm": gbs / peaks["hbm_gbs"],
+                            "frac_of_nominal_8TBs": gbs / 8000.0, "tokens_per_s": wl.batch / (ms / K * 1e-3),
+                            "launches_per_step": launches / K, "steps": K, "regions": regions,
+                            "batch": wl.batch, "context": wl.context or list(wl.context_range),
+                            "kv_gb_per_step": nbytes / K / 1e9}
+        finally:
+            sess.close()
+    return res
+
+
 def run_gpu_arm(args, wl):
     from paper_2409_15012_b200 import build as mbuild
     rank = int(os.environ.get("RANK", "0"))
@@ -327,18 +459,12 @@ def run_gpu_arm(args, wl):
     from paper_2409_15012_b200 import binding as mx, runner
     peaks = load_peaks()
     K, Wm = args.steps, args.warmup
-    total_steps = 2 * (K + Wm) + min(K, 20) + 2       # device-timed pass, e2e pass, profiled pass
-
-    if wl.context_range != (0, 0):
-        lengths = si.draw_lengths(wl.seed, wl.batch, *wl.context_range).tolist()
-    else:
-        lengths = [wl.context] * wl.batch
-    free_order = None
-    if wl.permute_pages:
-        n_pages = sum(-(-(n + total_steps) // wl.page_size) for n in lengths)
-        free_order = si.page_permutation(wl.seed, n_pages)
-    sess = runner.Session(wl, lengths, device=local, headroom_tokens=total_steps, free_order=free_order)
-    sess.fill(1024)
+    # device-timed pass, e2e pass (each up to MAX_EXTRA_STEPS more), profiled pass
+    total_steps = 2 * (K + Wm + MAX_EXTRA_STEPS) + min(K, 20) + 2
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()          # before the fill and the warm-up: the GPU is under load when timing starts
+    sess, lengths = make_session(runner, wl, local, total_steps)
     stream = torch.cuda.current_stream()
     outs = sess.alloc_outputs()
 
@@ -351,34 +477,11 @@ def run_gpu_arm(args, wl):
         return runner.kv_bytes_per_step(wl, [int(p) + 1 for p in sess.pos])
 
     # ---- device-resident pass: `value` ----
-    # step inputs: a ring of kRing distinct seeded steps reused cyclically (the values do not
-    # change the work; positions, appends and lengths advance every step as in serving)
     kRing = min(8, Wm + K)
-    step_inputs = []
-    pos_save = sess.pos.copy()
-    for s in range(kRing):
-        step_inputs.append(sess.step_inputs())
-        sess.pos += 1
-    sess.pos[:] = pos_save
-    for s in range(Wm):
-        sess.decode_step(step_inputs[s % kRing], outs, stream)
-    launches0 = sess.ctx.get_launch_count()
-    sampler = ClockSampler(local)
-    if rank == 0:
-        sampler.start()
-    barrier()
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    kv_bytes = 0
-    ev0.record(stream)
-    for s in range(K):
-        kv_bytes += bytes_next_step()
-        sess.decode_step(step_inputs[(Wm + s) % kRing], outs, stream)
-    ev1.record(stream)
-    barrier()
-    ms = ev0.elapsed_time(ev1)
+    step_inputs = step_input_ring(sess, kRing)
+    ms, kv_bytes, regions, launches = device_pass(sess, runner, wl, step_inputs, outs, stream, K, Wm, barrier,
+                                                  sampler if rank == 0 else None)
     clocks = sampler.stop() if rank == 0 else None
-    launches = sess.ctx.get_launch_count() - launches0
-    assert sess.ctx.get_device_status() == 0, "a kernel reported a wait time-out"
 
     # ---- end-to-end pass: host inputs, host outputs ----
     # Each step's inputs sit in one pinned host buffer and travel in two pieces on a copy
@@ -450,15 +553,26 @@ def run_gpu_arm(args, wl):
     for s in range(Wm):
         e2e_step(s)
     barrier()
-    e2e_bytes = 0
-    t0 = time.perf_counter()
-    ev0.record(stream)
-    for s in range(K):
-        e2e_bytes += bytes_next_step()
-        e2e_step(Wm + s)
-    ev1.record(stream)
+    # as many K-step regions as the device-resident pass timed; each region's time is the larger of
+    # the device time between its events and the host's wall clock around it (every step ends with
+    # a host wait, so the two agree)
+    e2e_ms_all, e2e_bytes_all = [], []
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    step = Wm
+    for _ in range(regions):
+        b = 0
+        t0 = time.perf_counter()
+        ev0.record(stream)
+        for _ in range(K):
+            b += bytes_next_step()
+            e2e_step(step)
+            step += 1
+        ev1.record(stream)
+        torch.cuda.synchronize()
+        e2e_ms_all.append(max(ev0.elapsed_time(ev1), (time.perf_counter() - t0) * 1e3))
+        e2e_bytes_all.append(b)
     barrier()
-    e2e_ms = max(ev0.elapsed_time(ev1), (time.perf_counter() - t0) * 1e3 if world == 1 else 0.0)
+    e2e_ms, e2e_bytes = float(np.mean(e2e_ms_all)), float(np.mean(e2e_bytes_all))
 
     # ---- per-kernel pass: roofline of the dominant kernel (split pass of a standard layer) ----
     full_layers = [l for l, (kind, _, _) in enumerate(wl.layout) if kind == cf.FULL]
@@ -515,11 +629,18 @@ def run_gpu_arm(args, wl):
                          f"heads, context {int(lengths[0])}+1; {reps} passes, {secs:.1f} s",
                "host_cores": os.cpu_count()}
 
-    prefill = None
+    prefill, others = None, None
+    closed = False
     if not args.no_prefill:
         sess.close()
+        closed = True
         prefill = prefill_figures(mx, runner, peaks, local)
         prefill["chunked"] = chunk_figures(mx, runner, peaks, local)
+    if not args.no_other_workloads and world == 1 and args.workload == "mid_decode" and args.batch == 0:
+        if not closed:
+            sess.close()
+            closed = True
+        others = other_workload_figures(runner, peaks, local, min(K, 20), Wm)
 
     line = {
         "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": K, "warmup": Wm,
@@ -535,14 +656,16 @@ def run_gpu_arm(args, wl):
                          "combine": ms_comb / max(n_comb, 1) * 1e3, "append": ms_app / max(n_app, 1) * 1e3},
         "e2e": {"value": e2e_bytes / (e2e_ms * 1e-3) / 1e9, "unit": "GB/s", "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms / K},
-        "gpu_launches": int(launches),
+        "gpu_launches": int(round(launches)),
+        "timed_regions": regions,
         "clocks": clocks,
         "roofline": roofline,
         "cpu_baseline": cpu,
         "prefill": prefill,
+        "other_workloads": others,
     }
     print(json.dumps(line), flush=True)
-    if prefill is None:
+    if not closed:
         sess.close()
     if dist is not None:
         dist.destroy_process_group()
@@ -579,6 +702,34 @@ def run_trace_arm(args):
     print(json.dumps(line), flush=True)
 
 
+def replica_envs(n: int, port: int, base_env=None):
+    """Environment of each of the n replica processes `--gpus n` starts when it was not launched
+    by torchrun: one rank per GPU of this node, rendezvous on the loopback address."""
+    envs = []
+    for r in range(n):
+        e = dict(os.environ if base_env is None else base_env)
+        e.update({"RANK": str(r), "LOCAL_RANK": str(r), "WORLD_SIZE": str(n), "LOCAL_WORLD_SIZE": str(n),
+                  "MASTER_ADDR": "127.0.0.1", "MASTER_PORT": str(port)})
+        envs.append(e)
+    return envs
+
+
+def spawn_replicas(n: int, argv) -> int:
+    """Runs this script once per GPU (independent replicas; NCCL carries only the barrier and the
+    two scalar reductions of the timing).  Rank 0 prints the JSON line.  Returns the worst exit code."""
+    import socket
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        port = sk.getsockname()[1]
+    procs = [subprocess.Popen([sys.executable, os.path.abspath(__file__)] + list(argv), env=e)
+             for e in replica_envs(n, port)]
+    rc = 0
+    for p in procs:
+        p.wait()
+        rc = rc or p.returncode
+    return rc
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -591,6 +742,8 @@ def main():
                     help="override the batch size (smaller cases for profiler captures; not a bench value)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-prefill", action="store_true")
+    ap.add_argument("--no-other-workloads", action="store_true",
+                    help="skip the compact figures of the other decode configurations")
     ap.add_argument("--trace", action="store_true", help="paper-shaped serving trace instead of the decode step")
     ap.add_argument("--trace-requests", type=int, default=8)
     ap.add_argument("--trace-prompt", type=int, default=31000)
@@ -601,6 +754,10 @@ def main():
     wl = get_workload(args.workload)
     if args.batch > 0:
         wl = wl.scaled(batch=args.batch, name=f"{wl.name}_batch{args.batch}")
+    if args.impl == "ours" and not args.trace and args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        if torch.cuda.device_count() < args.gpus:
+            raise SystemExit(f"--gpus {args.gpus}: this node shows {torch.cuda.device_count()} CUDA devices")
+        raise SystemExit(spawn_replicas(args.gpus, sys.argv[1:]))
     if args.impl == "reference":
         run_reference_arm(args, wl)
     elif args.trace:

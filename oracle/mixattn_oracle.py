@@ -23,6 +23,10 @@ a paged cache (16-token pages, FIFO free list, one block table per sequence)
 and of ring buffers (slot = position mod s); attention computed from what the
 physical half still stores must equal the logical half.
 
+Quantised KV storage (FP8 E4M3 elements with a shared power-of-two scale per
+head vector) is a reading of this build, not the paper's: see the section on
+it below and its pins in tests/test_oracle_fp8.py.
+
 Pins (tests/test_oracle_pins.py): dense brute-force masked softmax on tiny
 inputs, torch's scaled_dot_product_attention in float64 for the no-window
 case, closed forms (constant V, zero Q, window 1), needle keys on both sides
@@ -109,6 +113,82 @@ def rope_rotate(x, positions, theta: float) -> np.ndarray:
     out[..., 0::2] = x[..., 0::2] * c - x[..., 1::2] * s
     out[..., 1::2] = x[..., 0::2] * s + x[..., 1::2] * c
     return out
+
+
+# --------------------------------------------------------------------------
+# quantised KV storage (Section 2, "KV Quantization": storing the cached keys and
+# values at reduced precision shrinks the cache and the bytes moved per step; the
+# paper names the technique as compatible and fixes no format)
+#
+# Reading taken here: every head vector (one token, one KV head; K and V apart) is
+# stored as FP8 E4M3 elements with one shared power-of-two scale, the block-scaled
+# layout of the OCP Microscaling formats with the head vector as the block:
+#   * E4M3 (OCP 8-bit floating point): 1 sign, 4 exponent (bias 7), 3 mantissa bits;
+#     exponent field 0 = subnormals m/8 * 2^-6; the largest finite value is 448
+#     (S.1111.110); S.1111.111 is NaN and there is no infinity;
+#   * shared exponent X = floor(log2(max |x|)) - 8 (8 = exponent of E4M3's largest
+#     binade), clamped to [-127, 127]; an all-zero vector takes X = -127;
+#   * element = round-to-nearest-even of x / 2^X onto the E4M3 grid, saturating at
+#     +-448 (a scaled maximum in (448, 512) rounds down to 448).
+# The division by 2^X is exact, so every quantisation decision is a function of exact
+# values: a CUDA implementation must reproduce codes and exponents bit for bit.
+# --------------------------------------------------------------------------
+
+E4M3_MAX = 448.0
+E4M3_EMAX = 8
+
+
+def e4m3_decode(codes) -> np.ndarray:
+    """Value of each 8-bit E4M3 code (float64), from the format definition."""
+    c = np.asarray(codes, dtype=np.uint8).astype(np.int64)
+    sign = np.where(c & 0x80, -1.0, 1.0)
+    e = (c >> 3) & 0xF
+    m = (c & 0x7).astype(np.float64)
+    val = np.where(e == 0, m / 8.0 * 2.0 ** -6, (1.0 + m / 8.0) * np.exp2((e - 7).astype(np.float64)))
+    val = np.where((c & 0x7F) == 0x7F, np.nan, val)
+    return sign * val
+
+
+def e4m3_encode(y) -> np.ndarray:
+    """Round-to-nearest-even of finite float64 values onto the E4M3 grid, saturating at
+    +-448; returns the 8-bit codes.  Written from the grid itself: in the binade
+    [2^e, 2^(e+1)) with e >= -6 the spacing is 2^(e-3); below 2^-6 (subnormals) it is 2^-9."""
+    y = np.asarray(y, dtype=np.float64)
+    a = np.abs(y)
+    e = np.floor(np.log2(np.where(a > 0, a, 1.0)))
+    e = np.maximum(e, -6.0)
+    step = np.exp2(e - 3.0)
+    q = np.rint(a / step) * step            # rint rounds halves to even; a / step is exact
+    q = np.minimum(q, E4M3_MAX)
+    # encode the grid value q (rounding may have carried it into the next binade)
+    e2 = np.floor(np.log2(np.where(q > 0, q, 1.0)))
+    normal = q >= 2.0 ** -6
+    E = np.where(normal, e2 + 7.0, 0.0)
+    M = np.where(normal, q / np.exp2(e2) * 8.0 - 8.0, q / 2.0 ** -9)
+    code = (E.astype(np.int64) << 3) | M.astype(np.int64)
+    code = np.where(np.signbit(y), code | 0x80, code)
+    return code.astype(np.uint8)
+
+
+def quantize_kv(x) -> Tuple[np.ndarray, np.ndarray]:
+    """x [n, heads, d] (K or V rows) -> (codes uint8 [n, heads, d], X int32 [n, heads])."""
+    x = _as64(x)
+    amax = np.abs(x).max(axis=-1)
+    X = np.floor(np.log2(np.where(amax > 0, amax, 1.0))) - E4M3_EMAX
+    X = np.where(amax > 0, X, -127.0)
+    X = np.clip(X, -127.0, 127.0)
+    codes = e4m3_encode(x / np.exp2(X)[..., None])
+    return codes, X.astype(np.int32)
+
+
+def dequantize_kv(codes, X) -> np.ndarray:
+    """Values the quantised cache stands for: element * 2^X (float64, exact)."""
+    return e4m3_decode(codes) * np.exp2(np.asarray(X, dtype=np.float64))[..., None]
+
+
+def kv_roundtrip(x) -> np.ndarray:
+    """dequantize_kv(quantize_kv(x)): what a layer reads back from a quantised cache."""
+    return dequantize_kv(*quantize_kv(x))
 
 
 # --------------------------------------------------------------------------

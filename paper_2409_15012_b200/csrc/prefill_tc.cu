@@ -211,6 +211,12 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   return *reinterpret_cast<uint32_t*>(&t);
 }
 
+// (x, y) -> packed bf16 pair `hi` and the packed bf16 pair `lo` of the rounding residuals
+__device__ __forceinline__ void split_bf16(float x, float y, uint32_t& hi, uint32_t& lo) {
+  hi = pack_bf16(x, y);
+  lo = pack_bf16(x - __uint_as_float(hi << 16), y - __uint_as_float(hi & 0xffff0000u));
+}
+
 // instruction descriptor: D fp32, A/B bf16, M = 128, N = 128; b_mn = 1 for an MN-major B
 __host__ __device__ constexpr uint32_t idesc_bf16(int b_mn) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)b_mn << 16) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
@@ -223,6 +229,7 @@ __host__ __device__ constexpr uint32_t idesc_bf16(int b_mn) {
 struct WorkItem {
   int h, g, row_base, krow_base, S, i0, pos0, jt_lo, n_tiles;   // pos0 = position of query row i0 among the keys
   bool valid;
+  bool lo;   // rows of this tile may see fewer than a tile of keys: P enters P V as two bf16 terms
 };
 __device__ __forceinline__ WorkItem get_item(const TcParams& p, int id) {
   WorkItem w;
@@ -243,6 +250,12 @@ __device__ __forceinline__ WorkItem get_item(const TcParams& p, int id) {
   const int key_lo = p.window > 0 ? max(0, w.pos0 - p.window + 1) : 0;
   w.jt_lo = key_lo / kBN;
   w.n_tiles = key_hi / kBN - w.jt_lo + 1;
+  // A row that sees only a few keys is a mix of a few V rows: its weights' bf16 rounding (2^-9
+  // each) does not average out and, on outputs of magnitude 2..4, would add to the output's own
+  // bf16 rounding.  Such rows (the first query tile of a sequence, or a window shorter than a
+  // tile) carry the rounding residual of P as a second bf16 term, like the decode kernel; all
+  // other tiles, whose rows average over at least a tile of keys, keep the single term.
+  w.lo = w.pos0 < kBM || (p.window > 0 && p.window < kBN);
   return w;
 }
 
@@ -412,6 +425,12 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
             for (int ks = 0; ks < 4; ++ks)   // 64 keys = 4 steps of 16
               umma_bf16_ts(tmem + kColO + hs * 128, tmem + kColS + sb * 128 + hs * 64 + ks * 8,
                            vdesc + (uint64_t)(ks * (2048 >> 4)), kIdescPV, (j > 0 || ks > 0) ? 1u : 0u);
+            if (w.lo) {   // the residual term of P sits in the other 32 of the stream's 64 columns
+#pragma unroll
+              for (int ks = 0; ks < 4; ++ks)
+                umma_bf16_ts(tmem + kColO + hs * 128, tmem + kColS + sb * 128 + hs * 64 + 32 + ks * 8,
+                             vdesc + (uint64_t)(ks * (2048 >> 4)), kIdescPV, 1u);
+            }
             if (j == w.n_tiles - 1) umma_commit(BAR(B_OF + hs));   // this stream's accumulator is complete
             umma_commit(BAR(B_VE + vs));   // V stage free once both streams' P V are done (count 2)
             umma_commit(BAR(B_SR + sb));   // and so is the S buffer
@@ -536,17 +555,28 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         const bool more = j + 1 < w.n_tiles;
         const bool next_ready = more && mbar_test_wait(BAR(B_SF + (sb ^ 1)), ((Gj + 1) >> 1) & 1);
         float sum0 = 0.f, sum1 = 0.f;
-        uint32_t pk[32];
+        uint32_t pk[32], pl[32];   // P as bf16 pairs; pl = rounding residuals (only on w.lo items)
+        if (!w.lo) {
 #pragma unroll
-        for (int e = 0; e < 64; e += 4) {
-          const float p0 = ex2_approx(fmaf(__uint_as_float(sv[e]), p.scale_log2e, neg_m));
-          const float p1 = ex2_approx(fmaf(__uint_as_float(sv[e + 1]), p.scale_log2e, neg_m));
-          const float p2 = ex2_approx(fmaf(__uint_as_float(sv[e + 2]), p.scale_log2e, neg_m));
-          const float p3 = ex2_approx(fmaf(__uint_as_float(sv[e + 3]), p.scale_log2e, neg_m));
-          sum0 += p0 + p2;
-          sum1 += p1 + p3;
-          pk[e >> 1] = pack_bf16(p0, p1);
-          pk[(e >> 1) + 1] = pack_bf16(p2, p3);
+          for (int e = 0; e < 64; e += 4) {
+            const float p0 = ex2_approx(fmaf(__uint_as_float(sv[e]), p.scale_log2e, neg_m));
+            const float p1 = ex2_approx(fmaf(__uint_as_float(sv[e + 1]), p.scale_log2e, neg_m));
+            const float p2 = ex2_approx(fmaf(__uint_as_float(sv[e + 2]), p.scale_log2e, neg_m));
+            const float p3 = ex2_approx(fmaf(__uint_as_float(sv[e + 3]), p.scale_log2e, neg_m));
+            sum0 += p0 + p2;
+            sum1 += p1 + p3;
+            pk[e >> 1] = pack_bf16(p0, p1);
+            pk[(e >> 1) + 1] = pack_bf16(p2, p3);
+          }
+        } else {
+#pragma unroll
+          for (int e = 0; e < 64; e += 2) {
+            const float p0 = ex2_approx(fmaf(__uint_as_float(sv[e]), p.scale_log2e, neg_m));
+            const float p1 = ex2_approx(fmaf(__uint_as_float(sv[e + 1]), p.scale_log2e, neg_m));
+            sum0 += p0;
+            sum1 += p1;
+            split_bf16(p0, p1, pk[e >> 1], pl[e >> 1]);
+          }
         }
         // A score that leads the reference by more than 2^kMaxLead shows in the sum of the tile's
         // weights (64 weights of at most 2^kMaxLead each stay below 2^(kMaxLead + 6); an overflow
@@ -596,12 +626,14 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
             const float p1 = ex2_approx(fmaf(__uint_as_float(sv[e + 1]), p.scale_log2e, neg_m));
             sum0 += p0;
             sum1 += p1;
-            pk[e >> 1] = pack_bf16(p0, p1);
+            split_bf16(p0, p1, pk[e >> 1], pl[e >> 1]);   // (pl is only stored on w.lo items)
           }
         }
         l += sum0 + sum1;
-        // P (bf16 pairs) over the first 32 of this stream's 64 score columns
+        // P (bf16 pairs) over the first 32 of this stream's 64 score columns, the residual
+        // term, where the item carries one, over the other 32
         tmem_st32(s_addr, pk);
+        if (w.lo) tmem_st32(s_addr + 32, pl);
         tmem_wait_st();
         tc_fence_before();
         // (one announcement barrier per S buffer: its next phase cannot complete before the

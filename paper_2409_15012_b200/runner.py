@@ -29,10 +29,14 @@ class Session:
 
     def __init__(self, wl: cf.Workload, lengths: Optional[Sequence[int]] = None, device: int = 0,
                  headroom_tokens: int = 0, free_order=None, n_pages: Optional[int] = None,
-                 mirror=None, chunk_scratch_tokens: int = 0):
+                 mirror=None, chunk_scratch_tokens: int = 0, gen_device=None):
         self.wl = wl
         self.device = device
         self.dev = torch.device(f"cuda:{device}")
+        # where the seeded inputs are generated: on the GPU by default (fast for multi-GiB
+        # caches); "cpu" generates on the host and copies, so that the only kernels a small run
+        # launches are the library's own
+        self.gen_dev = self.dev if gen_device is None else torch.device(gen_device)
         self.dt = torch_dtype(wl.dtype)
         B = wl.batch
         if lengths is None:
@@ -76,9 +80,9 @@ class Session:
             for seqs, n in groups:
                 for o in self.owners:
                     K, V = si.kv_tokens_multi(wl.seed, o, seqs, [self.pos[b] for b in seqs], n,
-                                              wl.n_kv_heads, wl.head_dim, self.dt, self.dev)
-                    K = K.reshape(-1, wl.n_kv_heads, wl.head_dim)
-                    V = V.reshape(-1, wl.n_kv_heads, wl.head_dim)
+                                              wl.n_kv_heads, wl.head_dim, self.dt, self.gen_dev)
+                    K = K.reshape(-1, wl.n_kv_heads, wl.head_dim).to(self.dev)
+                    V = V.reshape(-1, wl.n_kv_heads, wl.head_dim).to(self.dev)
                     self._append(o, seqs, [n] * len(seqs), K, V)
                 for b in seqs:
                     self.pos[b] += n
@@ -90,18 +94,19 @@ class Session:
         """Q for every layer and the new token's K/V for every owner, for the
         decode step that appends position pos[b] to sequence b."""
         wl = self.wl
+        gen = self.gen_dev if device is None else device
         device = self.dev if device is None else device
         out: Dict[int, Dict[str, torch.Tensor]] = {}
         B = wl.batch
         for l in range(len(wl.layout)):
             q = si.q_tokens_multi(wl.seed, l, list(range(B)), [int(p) for p in self.pos], 1, wl.n_q_heads,
-                                  wl.head_dim, self.dt, device)[:, 0].contiguous()
+                                  wl.head_dim, self.dt, gen)[:, 0].contiguous().to(device)
             ent = {"q": q}
             if l in self.owners:
                 K, V = si.kv_tokens_multi(wl.seed, l, list(range(B)), [int(p) for p in self.pos], 1,
-                                          wl.n_kv_heads, wl.head_dim, self.dt, device)
-                ent["k"] = K.reshape(B, wl.n_kv_heads, wl.head_dim)
-                ent["v"] = V.reshape(B, wl.n_kv_heads, wl.head_dim)
+                                          wl.n_kv_heads, wl.head_dim, self.dt, gen)
+                ent["k"] = K.reshape(B, wl.n_kv_heads, wl.head_dim).to(device)
+                ent["v"] = V.reshape(B, wl.n_kv_heads, wl.head_dim).to(device)
             out[l] = ent
         return out
 
@@ -169,14 +174,16 @@ class Session:
         """Packed Q, K, V of the prompts (length wl.seq_len each) for `layer`;
         K/V are the owner's."""
         wl = self.wl
+        gen = self.gen_dev if device is None else device
         device = self.dev if device is None else device
         owner = wl.layout[layer][2]
         S = wl.seq_len
         q = si.q_tokens_multi(wl.seed, layer, list(range(wl.batch)), [0] * wl.batch, S, wl.n_q_heads,
-                              wl.head_dim, self.dt, device).reshape(-1, wl.n_q_heads, wl.head_dim)
+                              wl.head_dim, self.dt, gen).reshape(-1, wl.n_q_heads, wl.head_dim)
         K, V = si.kv_tokens_multi(wl.seed, owner, list(range(wl.batch)), [0] * wl.batch, S,
-                                  wl.n_kv_heads, wl.head_dim, self.dt, device)
-        return q, K.reshape(-1, wl.n_kv_heads, wl.head_dim), V.reshape(-1, wl.n_kv_heads, wl.head_dim)
+                                  wl.n_kv_heads, wl.head_dim, self.dt, gen)
+        return (q.to(device), K.reshape(-1, wl.n_kv_heads, wl.head_dim).to(device),
+                V.reshape(-1, wl.n_kv_heads, wl.head_dim).to(device))
 
     def prefill_layer(self, layer: int, q, k, v, out, stream=None):
         wl = self.wl

@@ -41,3 +41,38 @@ def test_reference_arm_prints_on_rank0_only():
     out = subprocess.run([sys.executable, "bench.py", "--impl", "reference", "--steps", "1"],
                          capture_output=True, text=True, timeout=300, cwd=ROOT, env=env)
     assert out.returncode == 0 and out.stdout.strip() == ""
+
+
+def test_replica_spawner_environment_and_region_count():
+    # `bench.py --gpus N` started without torchrun spawns N replicas itself: one rank per GPU,
+    # loopback rendezvous, every rank told the world size
+    sys.path.insert(0, ROOT)
+    import bench
+    envs = bench.replica_envs(4, 29999, base_env={"PATH": "/usr/bin", "WORLD_SIZE": "stale"})
+    assert [e["RANK"] for e in envs] == ["0", "1", "2", "3"]
+    assert [e["LOCAL_RANK"] for e in envs] == ["0", "1", "2", "3"]
+    assert all(e["WORLD_SIZE"] == "4" and e["MASTER_ADDR"] == "127.0.0.1" and e["MASTER_PORT"] == "29999"
+               and e["PATH"] == "/usr/bin" for e in envs)
+    # a short K-step region is repeated until about MIN_TIMED_S has been timed, within the step cap
+    assert bench.n_regions_for(33.0, 20) == 13
+    assert bench.n_regions_for(330.0, 200) == 2
+    assert bench.n_regions_for(5000.0, 200) == 1
+    assert bench.n_regions_for(0.1, 20) == 1 + bench.MAX_EXTRA_STEPS // 20
+
+
+def test_replica_spawner_runs_one_process_per_rank(tmp_path):
+    # the spawner itself, with a stand-in script: two processes, ranks 0 and 1, worst exit code returned
+    sys.path.insert(0, ROOT)
+    import bench
+    script = tmp_path / "child.py"
+    script.write_text("import os, sys\n"
+                      f"open(os.path.join({str(tmp_path)!r}, 'rank' + os.environ['RANK']), 'w').write(os.environ['WORLD_SIZE'])\n"
+                      "sys.exit(3 if os.environ['RANK'] == '1' else 0)\n")
+    saved = bench.__file__
+    bench.__file__ = str(script)
+    try:
+        rc = bench.spawn_replicas(2, [])
+    finally:
+        bench.__file__ = saved
+    assert rc == 3
+    assert (tmp_path / "rank0").read_text() == "2" and (tmp_path / "rank1").read_text() == "2"
