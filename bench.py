@@ -344,7 +344,7 @@ def n_regions_for(region_ms: float, K: int) -> int:
     return max(1, min(want, 1 + MAX_EXTRA_STEPS // max(K, 1)))
 
 
-def make_session(runner, wl, device, total_steps):
+def make_session(runner, wl, device, total_steps, kv_format=0):
     """Session with the workload's lengths drawn, its page order permuted if asked, caches filled."""
     if wl.context_range != (0, 0):
         lengths = si.draw_lengths(wl.seed, wl.batch, *wl.context_range).tolist()
@@ -354,7 +354,8 @@ def make_session(runner, wl, device, total_steps):
     if wl.permute_pages:
         n_pages = sum(-(-(n + total_steps) // wl.page_size) for n in lengths)
         free_order = si.page_permutation(wl.seed, n_pages)
-    sess = runner.Session(wl, lengths, device=device, headroom_tokens=total_steps, free_order=free_order)
+    sess = runner.Session(wl, lengths, device=device, headroom_tokens=total_steps, free_order=free_order,
+                          kv_format=kv_format)
     sess.fill(1024)
     return sess, lengths
 
@@ -377,7 +378,7 @@ def device_pass(sess, runner, wl, ring, outs, stream, K, Wm, barrier, sampler=No
     (n_regions_for).  Returns (mean ms per region, mean KV bytes per region, regions, launches
     per region)."""
     def bytes_next_step():
-        return runner.kv_bytes_per_step(wl, [int(p) + 1 for p in sess.pos])
+        return runner.kv_bytes_per_step(wl, [int(p) + 1 for p in sess.pos], sess.kv_format)
 
     step = 0
     for _ in range(Wm):
@@ -418,12 +419,17 @@ def device_pass(sess, runner, wl, ring, outs, stream, K, Wm, barrier, sampler=No
 
 def other_workload_figures(runner, peaks, device, K, Wm):
     """The other decode configurations, device-resident, in compact form: long-context decode,
-    its variant with rings shared in pairs, and the mixed serving batch."""
+    its variant with rings shared in pairs, the mixed serving batch, and the mid-decode
+    configuration on a quantised cache (FP8 E4M3 elements: bytes = what that cache holds)."""
+    from paper_2409_15012_b200 import binding as mx
     res = {}
-    for name in ("long_decode", "long_decode_pairs", "mixed_serving"):
+    for name, kvf in (("long_decode", 0), ("long_decode_pairs", 0), ("mixed_serving", 0),
+                      ("mid_decode", mx.KV_FP8_E4M3)):
         wl = get_workload(name)
+        if kvf:
+            wl = wl.scaled(name=wl.name + "_fp8_kv")
         total = Wm + K + MAX_EXTRA_STEPS + 2
-        sess, lengths = make_session(runner, wl, device, total)
+        sess, lengths = make_session(runner, wl, device, total, kvf)
         try:
             ring = step_input_ring(sess, min(4, Wm + K))
             outs = sess.alloc_outputs()

@@ -37,6 +37,11 @@ typedef struct mixattn_ctx mixattn_ctx; /* opaque; owned by the library */
 
 enum { MIXATTN_FULL = 0, MIXATTN_SLIDING = 1 };
 enum { MIXATTN_F32 = 0, MIXATTN_BF16 = 1 };
+/* How cached keys and values are stored (mixattn_config.kv_format). */
+enum {
+  MIXATTN_KV_NATIVE = 0,   /* in the context's dtype                                               */
+  MIXATTN_KV_FP8_E4M3 = 1  /* quantised: see "Quantised KV storage" below                          */
+};
 
 enum {
   MIXATTN_OK = 0,
@@ -81,7 +86,33 @@ typedef struct {
   size_t arena_bytes;               /* >= mixattn_arena_bytes(); the library never frees it         */
   int32_t chunk_scratch_tokens;     /* K/V rows of scratch kept in the arena for
                                        mixattn_attend_chunk; 0 = that call is unavailable           */
+  int32_t kv_format;                /* MIXATTN_KV_NATIVE or MIXATTN_KV_FP8_E4M3                     */
 } mixattn_config;
+
+/* Quantised KV storage (kv_format = MIXATTN_KV_FP8_E4M3).
+ *
+ * Section 2 of the paper ("KV Quantization") names storing the cached keys and
+ * values at reduced precision as a technique that combines with MixAttention:
+ * it shrinks the cache and the bytes a decode step moves, which Section 1
+ * gives as the cost of long-context inference.  The paper fixes no format;
+ * this library stores every head vector (one token, one KV head; K and V
+ * apart) as head_dim FP8 E4M3 elements (OCP 8-bit float: 1 sign, 4 exponent
+ * bits with bias 7, 3 mantissa bits, largest value 448, no infinity) plus one
+ * byte holding a shared power-of-two exponent X (stored as X + 127):
+ *     X       = floor(log2(max |x|)) - 8, clamped to [-127, 127]; -127 for a zero vector
+ *     element = x / 2^X rounded to the nearest E4M3 value, ties to even,
+ *               saturating at +-448
+ * and a reader sees element * 2^X, which is again a bf16 number.  Cached
+ * bytes per token and KV head: 2 * (head_dim + 1) instead of 4 * head_dim.
+ * Requirements: dtype MIXATTN_BF16 and head_dim 128 (else
+ * MIXATTN_ERR_UNSUPPORTED from create).  Q, K, V and out of every call stay
+ * bf16: mixattn_append_kv (and _rope, and the store of mixattn_prefill)
+ * quantise on the way in; mixattn_decode reads the quantised cache, widening
+ * elements exactly to fp16 for the tensor-core products with Q and P converted
+ * to fp16 as well (so |q| must stay below 65504 and max |v| of a row below
+ * 2^23); mixattn_attend_chunk reads the cached part dequantised and the
+ * chunk's own K/V as given.  mixattn_prefill attends over the K/V it is given,
+ * unquantised. */
 
 /* Bytes of device memory a context with this config carves out of `arena`:
  * K/V storage (see mixattn_cache_bytes), the device copy of the block tables
@@ -278,6 +309,14 @@ int mixattn_locate(mixattn_ctx* ctx, int32_t layer, int32_t seq, int32_t pos, in
  * also checks that copy.  For tests. */
 int mixattn_debug_read_kv(mixattn_ctx* ctx, int32_t layer, int32_t seq, int32_t pos, void* k_host,
                           void* v_host);
+
+/* Quantised storage only: the stored bytes of token `pos`: head_dim E4M3 codes per KV head
+ * ([n_kv_heads, head_dim] bytes each for K and V) and the shared exponents X
+ * ([n_kv_heads] int32 each).  UNSUPPORTED on a context with native storage;
+ * all else as mixattn_debug_read_kv, which on a quantised cache returns the
+ * dequantised bf16 values. */
+int mixattn_debug_read_kv_fp8(mixattn_ctx* ctx, int32_t layer, int32_t seq, int32_t pos,
+                              uint8_t* k_codes, int32_t* k_exp, uint8_t* v_codes, int32_t* v_exp);
 
 /* Waits for the device, then reports the status word the kernels share:
  * 0 = fine, 1 = a bounded wait inside a kernel ran out (results invalid). */

@@ -15,6 +15,7 @@ import numpy as np
 
 FULL, SLIDING = 0, 1
 F32, BF16 = 0, 1
+KV_NATIVE, KV_FP8_E4M3 = 0, 1
 
 OK = 0
 ERR_INVALID_ARG = -1
@@ -54,6 +55,7 @@ class Config(C.Structure):
         ("arena", C.c_void_p),
         ("arena_bytes", C.c_size_t),
         ("chunk_scratch_tokens", C.c_int32),
+        ("kv_format", C.c_int32),
     ]
 
 
@@ -83,6 +85,7 @@ def _load() -> C.CDLL:
         "mixattn_get_ring_state": [vp, i32, i32, p32, p32],
         "mixattn_locate": [vp, i32, i32, i32, p32, p32],
         "mixattn_debug_read_kv": [vp, i32, i32, i32, vp, vp],
+        "mixattn_debug_read_kv_fp8": [vp, i32, i32, i32, vp, vp, vp, vp],
         "mixattn_get_device_status": [vp, p32],
         "mixattn_set_split_tokens": [vp, i32],
         "mixattn_set_chunk_gather_reuse": [vp, i32],
@@ -105,7 +108,7 @@ EXPORTS = [
     "mixattn_seq_reset", "mixattn_append_kv", "mixattn_append_kv_rope", "mixattn_decode", "mixattn_decode_static_scratch", "mixattn_prefill",
     "mixattn_attend_chunk",
     "mixattn_get_len", "mixattn_get_block_table", "mixattn_get_n_free_pages",
-    "mixattn_get_ring_state", "mixattn_locate", "mixattn_debug_read_kv",
+    "mixattn_get_ring_state", "mixattn_locate", "mixattn_debug_read_kv", "mixattn_debug_read_kv_fp8",
     "mixattn_get_device_status", "mixattn_set_split_tokens", "mixattn_set_chunk_gather_reuse",
     "mixattn_profile_enable",
     "mixattn_profile_read", "mixattn_get_launch_count", "mixattn_strerror",
@@ -143,7 +146,7 @@ def _stream(stream) -> Optional[int]:
 def make_config(layout: Sequence, n_q_heads: int, n_kv_heads: int, head_dim: int, dtype: int,
                 max_seqs: int, n_pages: int, max_seq_len: int = 0, free_order=None,
                 softmax_scale: float = 0.0, device: int = -1, page_size: int = 16,
-                chunk_scratch_tokens: int = 0):
+                chunk_scratch_tokens: int = 0, kv_format: int = KV_NATIVE):
     """Returns (Config, keepalive): keepalive owns the arrays the struct points to."""
     layers = (LayerDesc * max(1, len(layout)))()
     for i, (kind, window, owner) in enumerate(layout):
@@ -151,7 +154,7 @@ def make_config(layout: Sequence, n_q_heads: int, n_kv_heads: int, head_dim: int
     fo = None if free_order is None else _i32(free_order)
     cfg = Config(len(layout), layers, n_q_heads, n_kv_heads, head_dim, dtype, max_seqs, page_size,
                  n_pages, max_seq_len, _p32(fo), float(softmax_scale), device, None, 0,
-                 int(chunk_scratch_tokens))
+                 int(chunk_scratch_tokens), int(kv_format))
     return cfg, (layers, fo)
 
 
@@ -179,10 +182,11 @@ class Context:
     """
 
     def __init__(self, layout, n_q_heads, n_kv_heads, head_dim, dtype, max_seqs, n_pages,
-                 max_seq_len=0, free_order=None, softmax_scale=0.0, device=-1, chunk_scratch_tokens=0):
+                 max_seq_len=0, free_order=None, softmax_scale=0.0, device=-1, chunk_scratch_tokens=0,
+                 kv_format=KV_NATIVE):
         self.cfg, self._keep = make_config(layout, n_q_heads, n_kv_heads, head_dim, dtype, max_seqs,
                                            n_pages, max_seq_len, free_order, softmax_scale, device,
-                                           chunk_scratch_tokens=chunk_scratch_tokens)
+                                           chunk_scratch_tokens=chunk_scratch_tokens, kv_format=kv_format)
         self.arena = None
         if device >= 0:
             import torch
@@ -321,6 +325,19 @@ class Context:
         if rc:
             raise MixAttnError(rc, "mixattn_debug_read_kv")
         return k, v
+
+    def debug_read_kv_fp8(self, layer, seq, pos):
+        """Quantised storage: (k_codes, k_exp, v_codes, v_exp) as numpy arrays: uint8 [Hkv, D]
+        codes and int32 [Hkv] shared exponents."""
+        kc = np.zeros((self.n_kv_heads, self.head_dim), dtype=np.uint8)
+        vc = np.zeros_like(kc)
+        kx = np.zeros(self.n_kv_heads, dtype=np.int32)
+        vx = np.zeros_like(kx)
+        rc = lib.mixattn_debug_read_kv_fp8(self.h, layer, seq, pos, kc.ctypes.data, kx.ctypes.data,
+                                           vc.ctypes.data, vx.ctypes.data)
+        if rc:
+            raise MixAttnError(rc, "mixattn_debug_read_kv_fp8")
+        return kc, kx, vc, vx
 
     def get_device_status(self) -> int:
         out = C.c_int32()

@@ -36,7 +36,7 @@ int ring_pages_of(int window) { return (window + kPage - 1) / kPage; }
 
 ArenaPlan plan_arena(const CacheManager& cm, const mixattn_config& cfg) {
   ArenaPlan pl;
-  KvGeom ge = make_geom(cfg.n_kv_heads, cfg.head_dim, cfg.dtype);
+  KvGeom ge = make_geom(cfg.n_kv_heads, cfg.head_dim, cfg.dtype, cfg.kv_format);
   size_t off = 0;
   for (int o : cm.owners()) {
     const LayerInfo& li = cm.layer(o);
@@ -164,6 +164,9 @@ int validate_config(const mixattn_config* cfg, CacheManager* cm, bool allocate =
   if (cfg->softmax_scale < 0.f || !isfinite(cfg->softmax_scale)) return MIXATTN_ERR_INVALID_ARG;
   if (cm->n_full_owners() > 0 && cfg->n_pages < 1) return MIXATTN_ERR_INVALID_ARG;
   if (cfg->chunk_scratch_tokens < 0) return MIXATTN_ERR_INVALID_ARG;
+  if (cfg->kv_format != MIXATTN_KV_NATIVE && cfg->kv_format != MIXATTN_KV_FP8_E4M3) return MIXATTN_ERR_INVALID_ARG;
+  if (cfg->kv_format == MIXATTN_KV_FP8_E4M3 && (cfg->dtype != MIXATTN_BF16 || cfg->head_dim != 128))
+    return MIXATTN_ERR_UNSUPPORTED;
   return MIXATTN_OK;
 }
 
@@ -274,7 +277,7 @@ int mixattn_create(const mixattn_config* cfg, mixattn_ctx** out) {
   c->cfg = *cfg;
   c->cfg.layers = nullptr;
   c->cfg.free_order = nullptr;
-  c->geom = make_geom(cfg->n_kv_heads, cfg->head_dim, cfg->dtype);
+  c->geom = make_geom(cfg->n_kv_heads, cfg->head_dim, cfg->dtype, cfg->kv_format);
   c->plan = plan_arena(c->cm, *cfg);
   c->scale = cfg->softmax_scale > 0.f ? cfg->softmax_scale : 1.0f / sqrtf((float)cfg->head_dim);
   c->host_only = cfg->device < 0;
@@ -751,6 +754,60 @@ int mixattn_locate(mixattn_ctx* c, int32_t layer, int32_t seq, int32_t pos, int3
   return c->cm.locate(layer, seq, pos, page, slot) ? MIXATTN_OK : MIXATTN_ERR_INVALID_ARG;
 }
 
+// Physical page (looked up in the DEVICE copy of the block table for a paged cache) and slot
+// within it of a stored token; `slot` comes in as CacheManager::locate returned it.
+static int stored_page_of(mixattn_ctx* c, int layer, int seq, int pos, int64_t* phys, int32_t* slot) {
+  const LayerInfo& li = c->cm.layer(layer);
+  if (li.kind == MIXATTN_FULL) {
+    int32_t dev_page = -1;
+    if (cudaMemcpy(&dev_page, c->dev_table() + (size_t)seq * c->cm.max_blocks() + pos / kPage,
+                   sizeof(int32_t), cudaMemcpyDeviceToHost) != cudaSuccess)
+      return MIXATTN_ERR_CUDA;
+    *phys = dev_page;
+  } else {
+    *phys = (int64_t)seq * ring_pages_of(li.window) + *slot / kPage;
+    *slot = *slot % kPage;
+  }
+  return MIXATTN_OK;
+}
+
+// Copies one stored row (its 16-byte chunks put back in order) to `dst` (st_row_bytes bytes) and,
+// for quantised storage, its shared exponent to *X.
+static int read_stored_row(mixattn_ctx* c, const char* pool, int64_t phys, int gh, int which, int slot,
+                           void* dst, int32_t* X) {
+  const KvGeom& ge = c->geom;
+  unsigned char row[512];
+  if (ge.st_row_bytes > (int)sizeof(row)) return MIXATTN_ERR_UNSUPPORTED;
+  // start of the stored row; its 16-byte chunks are permuted unless the cache is fp32
+  const char* src = pool + phys * ge.page_bytes + (int64_t)gh * ge.blk_bytes +
+                    (int64_t)(which * kPage + slot) * ge.st_row_bytes;
+  if (cudaMemcpy(row, src, ge.st_row_bytes, cudaMemcpyDeviceToHost) != cudaSuccess) return MIXATTN_ERR_CUDA;
+  const int chunks = ge.st_row_bytes / 16;
+  for (int ch = 0; ch < chunks; ++ch) {
+    const int phys_ch = ge.swizzle ? (ch ^ (slot & 7)) : ch;
+    memcpy(static_cast<char*>(dst) + ch * 16, row + phys_ch * 16, 16);
+  }
+  if (ge.fp8 && X != nullptr) {
+    unsigned char xb = 0;
+    if (cudaMemcpy(&xb, pool + kv_exp_offset(ge, phys, gh, which, slot), 1, cudaMemcpyDeviceToHost) != cudaSuccess)
+      return MIXATTN_ERR_CUDA;
+    *X = (int32_t)xb - 127;
+  }
+  return MIXATTN_OK;
+}
+
+// bf16 bit pattern of an E4M3 code times 2^X (host side of the debug read; the format is the
+// OCP 8-bit float: exponent bias 7, subnormals m/8 * 2^-6, no infinity).
+static uint16_t bf16_bits_of_e4m3(unsigned char code, int X) {
+  const int e = (code >> 3) & 0xF, m = code & 7;
+  float v = e == 0 ? ldexpf((float)m, -9) : ldexpf(1.0f + (float)m / 8.0f, e - 7);
+  v = ldexpf(v, X);
+  if (code & 0x80) v = -v;
+  uint32_t bits;
+  memcpy(&bits, &v, 4);
+  return (uint16_t)(bits >> 16);   // exact: four significant bits
+}
+
 int mixattn_debug_read_kv(mixattn_ctx* c, int32_t layer, int32_t seq, int32_t pos, void* k_host, void* v_host) {
   if (c == nullptr || k_host == nullptr || v_host == nullptr || !c->cm.valid_layer(layer))
     return MIXATTN_ERR_INVALID_ARG;
@@ -760,35 +817,49 @@ int mixattn_debug_read_kv(mixattn_ctx* c, int32_t layer, int32_t seq, int32_t po
   if (c->host_only) return MIXATTN_ERR_CUDA;
   DeviceGuard g(c->device);
   if (!g.ok || cudaDeviceSynchronize() != cudaSuccess) return MIXATTN_ERR_CUDA;
-  const LayerInfo& li = c->cm.layer(layer);
   const KvGeom& ge = c->geom;
   int64_t phys;
-  if (li.kind == MIXATTN_FULL) {
-    int32_t dev_page = -1;
-    if (cudaMemcpy(&dev_page, c->dev_table() + (size_t)seq * c->cm.max_blocks() + pos / kPage,
-                   sizeof(int32_t), cudaMemcpyDeviceToHost) != cudaSuccess)
-      return MIXATTN_ERR_CUDA;
-    phys = dev_page;
-  } else {
-    phys = (int64_t)seq * ring_pages_of(li.window) + slot / kPage;
-    slot = slot % kPage;
-  }
+  if (stored_page_of(c, layer, seq, pos, &phys, &slot) != MIXATTN_OK) return MIXATTN_ERR_CUDA;
   const char* pool = c->owner_storage(layer);
-  std::vector<char> row(ge.row_bytes);
-  const int chunks = ge.row_bytes / 16;
+  std::vector<unsigned char> codes(ge.st_row_bytes);
   for (int which = 0; which < 2; ++which) {
     char* dst = static_cast<char*>(which ? v_host : k_host);
     for (int gh = 0; gh < ge.n_kv_heads; ++gh) {
-      // start of the token row; its 16-byte chunks are permuted in bf16 mode
-      const char* src = pool + phys * ge.page_bytes + (int64_t)gh * ge.blk_bytes +
-                        (int64_t)which * kPage * ge.row_bytes + (int64_t)slot * ge.row_bytes;
-      if (cudaMemcpy(row.data(), src, ge.row_bytes, cudaMemcpyDeviceToHost) != cudaSuccess)
-        return MIXATTN_ERR_CUDA;
-      for (int ch = 0; ch < chunks; ++ch) {
-        const int phys_ch = ge.swizzle ? (ch ^ (slot & 7)) : ch;
-        memcpy(dst + (size_t)gh * ge.row_bytes + ch * 16, row.data() + phys_ch * 16, 16);
+      if (!ge.fp8) {
+        if (read_stored_row(c, pool, phys, gh, which, slot, dst + (size_t)gh * ge.row_bytes, nullptr) != MIXATTN_OK)
+          return MIXATTN_ERR_CUDA;
+        continue;
       }
+      // quantised storage: element * 2^X, which is a bf16 number
+      int32_t X = 0;
+      if (read_stored_row(c, pool, phys, gh, which, slot, codes.data(), &X) != MIXATTN_OK) return MIXATTN_ERR_CUDA;
+      uint16_t* out = reinterpret_cast<uint16_t*>(dst + (size_t)gh * ge.row_bytes);
+      for (int d = 0; d < ge.head_dim; ++d) out[d] = bf16_bits_of_e4m3(codes[d], X);
     }
+  }
+  return MIXATTN_OK;
+}
+
+int mixattn_debug_read_kv_fp8(mixattn_ctx* c, int32_t layer, int32_t seq, int32_t pos, uint8_t* k_codes,
+                              int32_t* k_exp, uint8_t* v_codes, int32_t* v_exp) {
+  if (c == nullptr || k_codes == nullptr || k_exp == nullptr || v_codes == nullptr || v_exp == nullptr ||
+      !c->cm.valid_layer(layer))
+    return MIXATTN_ERR_INVALID_ARG;
+  if (!c->cm.valid_seq(seq)) return MIXATTN_ERR_BAD_SEQ;
+  if (!c->geom.fp8) return MIXATTN_ERR_UNSUPPORTED;
+  int32_t page, slot;
+  if (!c->cm.locate(layer, seq, pos, &page, &slot)) return MIXATTN_ERR_INVALID_ARG;
+  if (c->host_only) return MIXATTN_ERR_CUDA;
+  DeviceGuard g(c->device);
+  if (!g.ok || cudaDeviceSynchronize() != cudaSuccess) return MIXATTN_ERR_CUDA;
+  int64_t phys;
+  if (stored_page_of(c, layer, seq, pos, &phys, &slot) != MIXATTN_OK) return MIXATTN_ERR_CUDA;
+  const KvGeom& ge = c->geom;
+  const char* pool = c->owner_storage(layer);
+  for (int gh = 0; gh < ge.n_kv_heads; ++gh) {
+    if (read_stored_row(c, pool, phys, gh, 0, slot, k_codes + (size_t)gh * ge.head_dim, &k_exp[gh]) != MIXATTN_OK ||
+        read_stored_row(c, pool, phys, gh, 1, slot, v_codes + (size_t)gh * ge.head_dim, &v_exp[gh]) != MIXATTN_OK)
+      return MIXATTN_ERR_CUDA;
   }
   return MIXATTN_OK;
 }

@@ -24,9 +24,18 @@
 //     which stream halves of its keys and merge through distributed shared memory: one
 //     CTA ingests K/V at a bounded rate, so idle SMs are better used than a second launch.
 //
+// Quantised cache (paper, Section 2, "KV Quantization"; KV8 instantiations): a (page, head)
+// block holds FP8 E4M3 rows and one shared power-of-two exponent per row, half the bytes per
+// key.  The same stream and the same tile shapes; the elements are widened exactly to fp16
+// after ldmatrix (a 32-bit fragment register then holds four channels of one key, so Q is
+// loaded in the matching channel order), the products run on the fp16 tensor-core path, a K
+// row's exponent multiplies its scores and a V row's exponent is folded into its weight.
+//
 // Every mbarrier wait is bounded: on time-out the kernel raises a status word and all
 // roles leave.
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
+#include <cuda_fp8.h>
 
 #include "internal.h"
 
@@ -118,6 +127,26 @@ __device__ __forceinline__ void mma_bf16(float (&d)[4], const uint32_t (&a)[4], 
       : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
       : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
+__device__ __forceinline__ void mma_f16(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
+      "{%0,%1,%2,%3};"
+      : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+// two E4M3 codes (low 16 bits of x) -> packed fp16 pair, exact
+__device__ __forceinline__ uint32_t e4m3x2_to_f16x2(uint32_t x) {
+  const __half2_raw h = __nv_cvt_fp8x2_to_halfraw2((__nv_fp8x2_storage_t)(x & 0xffffu), __NV_E4M3);
+  return (uint32_t)h.x | ((uint32_t)h.y << 16);
+}
+__device__ __forceinline__ uint32_t pack_f16(float lo, float hi) {
+  const __half2 t = __floats2half2_rn(lo, hi);
+  return *reinterpret_cast<const uint32_t*>(&t);
+}
+// 2^X from the stored exponent byte X + 127 (byte 0 is 2^-127, a subnormal)
+__device__ __forceinline__ float exp_byte_to_float(uint32_t b) {
+  return __int_as_float(b ? (int)(b << 23) : 0x00400000);
+}
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   __nv_bfloat162 t = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<uint32_t*>(&t);
@@ -196,13 +225,14 @@ __device__ __forceinline__ void cluster_share(Item& x, int crank) {
 // which take halves of the item's keys and merge through distributed shared memory: one CTA
 // ingests K/V at a fixed rate, so a short launch that leaves SMs idle is halved this way
 // without a second launch.  The grid then holds exactly one cluster per item.
-template <int D, int NCW, int CL>
+// KV8 = 1: the cache holds FP8 E4M3 rows with shared exponents (see the top of the file).
+template <int D, int NCW, int CL, int KV8>
 __global__ void __launch_bounds__((NCW + 1) * 32, NCW == 8 ? 1 : 2)
 decode_split_bf16_kernel(const __grid_constant__ DecodeParams p, const int n_stages) {
   constexpr int kConsumerWarps = NCW;
   constexpr int kGroups = NCW / kGroupWarps;
-  constexpr int kRowBytes = D * 2;
-  constexpr int kBlkBytes = 2 * kPage * kRowBytes;       // K+V of one (page, head)
+  constexpr int kRowBytes = KV8 ? D : D * 2;
+  constexpr int kBlkBytes = 2 * kPage * kRowBytes + (KV8 ? 2 * kPage : 0);   // K+V (+ exponents) of one (page, head)
   constexpr int kStageBytes = kGroupWarps * kBlkBytes;
   constexpr int kKSteps = D / 16;
 
@@ -331,13 +361,28 @@ decode_split_bf16_kernel(const __grid_constant__ DecodeParams p, const int n_sta
 
     // Q^T fragments (B operand): thread holds head (lane >> 2), channels 16 ks + fcol (+8)
     uint32_t qb[kKSteps][2];
-    {
+    if constexpr (!KV8) {
       const __nv_bfloat16* qp = reinterpret_cast<const __nv_bfloat16*>(p.q) +
                                 ((int64_t)x.i * p.n_q_heads + h0 + frow) * D + fcol;
 #pragma unroll
       for (int ks = 0; ks < kKSteps; ++ks) {
         qb[ks][0] = frow < rows ? *reinterpret_cast<const uint32_t*>(qp + ks * 16) : 0u;
         qb[ks][1] = frow < rows ? *reinterpret_cast<const uint32_t*>(qp + ks * 16 + 8) : 0u;
+      }
+    } else {
+      // A K fragment register holds four consecutive channels of a key (two go to the k index
+      // pair 2t, 2t+1 and two to 2t+8, 2t+9), so this thread's Q values of a 16-channel step
+      // are the four channels 4t .. 4t+3, as fp16
+      const __nv_bfloat16* qp = reinterpret_cast<const __nv_bfloat16*>(p.q) +
+                                ((int64_t)x.i * p.n_q_heads + h0 + frow) * D + 2 * fcol;
+#pragma unroll
+      for (int ks = 0; ks < kKSteps; ++ks) {
+        uint2 w = make_uint2(0u, 0u);
+        if (frow < rows) w = *reinterpret_cast<const uint2*>(qp + ks * 16);
+        const __nv_bfloat162 a = *reinterpret_cast<const __nv_bfloat162*>(&w.x);
+        const __nv_bfloat162 b = *reinterpret_cast<const __nv_bfloat162*>(&w.y);
+        qb[ks][0] = pack_f16(__low2float(a), __high2float(a));
+        qb[ks][1] = pack_f16(__low2float(b), __high2float(b));
       }
     }
     float m[2] = {-INFINITY, -INFINITY};
@@ -358,16 +403,40 @@ decode_split_bf16_kernel(const __grid_constant__ DecodeParams p, const int n_sta
         const uint32_t kb = smem_u32(stages + (size_t)s * kStageBytes + wig * kBlkBytes);
         const uint32_t vb = kb + kPage * kRowBytes;
         float st[4] = {0.f, 0.f, 0.f, 0.f}, st2[4] = {0.f, 0.f, 0.f, 0.f};  // two chains: shorter latency
+        float vscale0 = 1.f, vscale1 = 1.f;   // quantised cache: 2^X of the V rows of keys frow, frow + 8
+        if constexpr (!KV8) {
 #pragma unroll
-        for (int ks = 0; ks < kKSteps; ks += 2) {
-          uint32_t a[4], b[4];
-          ldsm_x4(kb + k_tok * kRowBytes + (((2 * ks + k_chk) ^ (k_tok & 7)) << 4), a[0], a[1], a[2], a[3]);
-          ldsm_x4(kb + k_tok * kRowBytes + (((2 * ks + 2 + k_chk) ^ (k_tok & 7)) << 4), b[0], b[1], b[2], b[3]);
-          mma_bf16(st, a, qb[ks][0], qb[ks][1]);
-          mma_bf16(st2, b, qb[ks + 1][0], qb[ks + 1][1]);
+          for (int ks = 0; ks < kKSteps; ks += 2) {
+            uint32_t a[4], b[4];
+            ldsm_x4(kb + k_tok * kRowBytes + (((2 * ks + k_chk) ^ (k_tok & 7)) << 4), a[0], a[1], a[2], a[3]);
+            ldsm_x4(kb + k_tok * kRowBytes + (((2 * ks + 2 + k_chk) ^ (k_tok & 7)) << 4), b[0], b[1], b[2], b[3]);
+            mma_bf16(st, a, qb[ks][0], qb[ks][1]);
+            mma_bf16(st2, b, qb[ks + 1][0], qb[ks + 1][1]);
+          }
+#pragma unroll
+          for (int e = 0; e < 4; ++e) st[e] = (st[e] + st2[e]) * p.scale_log2e;
+        } else {
+          // one ldmatrix.x4 = (keys 0-7 | 8-15) x (16-byte chunk 2j | 2j+1) = two 16-channel steps
+#pragma unroll
+          for (int j = 0; j < kKSteps / 2; ++j) {
+            uint32_t r[4];
+            ldsm_x4(kb + k_tok * kRowBytes + (((2 * j + k_chk) ^ (k_tok & 7)) << 4), r[0], r[1], r[2], r[3]);
+            const uint32_t a[4] = {e4m3x2_to_f16x2(r[0]), e4m3x2_to_f16x2(r[1]),
+                                   e4m3x2_to_f16x2(r[0] >> 16), e4m3x2_to_f16x2(r[1] >> 16)};
+            const uint32_t b[4] = {e4m3x2_to_f16x2(r[2]), e4m3x2_to_f16x2(r[3]),
+                                   e4m3x2_to_f16x2(r[2] >> 16), e4m3x2_to_f16x2(r[3] >> 16)};
+            mma_f16(st, a, qb[2 * j][0], qb[2 * j][1]);
+            mma_f16(st2, b, qb[2 * j + 1][0], qb[2 * j + 1][1]);
+          }
+          // the shared exponents of the page's rows sit behind its K and V rows
+          const unsigned char* xs = stages + (size_t)s * kStageBytes + wig * kBlkBytes + 2 * kPage * kRowBytes;
+          const float ks0 = exp_byte_to_float(xs[frow]) * p.scale_log2e;
+          const float ks1 = exp_byte_to_float(xs[frow + 8]) * p.scale_log2e;
+          vscale0 = exp_byte_to_float(xs[kPage + frow]);
+          vscale1 = exp_byte_to_float(xs[kPage + frow + 8]);
+          st[0] = (st[0] + st2[0]) * ks0; st[1] = (st[1] + st2[1]) * ks0;
+          st[2] = (st[2] + st2[2]) * ks1; st[3] = (st[3] + st2[3]) * ks1;
         }
-#pragma unroll
-        for (int e = 0; e < 4; ++e) st[e] = (st[e] + st2[e]) * p.scale_log2e;
         if (tok_base + kPage > x.t1) {  // ragged end of the split: keys are rows frow, frow + 8
           const int lim = x.t1 - tok_base;
           if (frow >= lim) st[0] = st[1] = -INFINITY;
@@ -391,23 +460,50 @@ decode_split_bf16_kernel(const __grid_constant__ DecodeParams p, const int n_sta
         // P^T as two bf16 terms (value + rounding residual): the stream leaves tensor
         // time to spare, so P keeps ~16 significant bits; then transpose 8x8 blocks so
         // that keys become the k index of the B operand
-        uint32_t ph0, pl0, ph1, pl1;
-        split_bf16(st[0], st[1], ph0, pl0);   // keys 0-7
-        split_bf16(st[2], st[3], ph1, pl1);   // keys 8-15
-        ph0 = movmatrix_t(ph0); ph1 = movmatrix_t(ph1);
-        pl0 = movmatrix_t(pl0); pl1 = movmatrix_t(pl1);
-        uint32_t va[D / 16][4];
+        if constexpr (!KV8) {
+          uint32_t ph0, pl0, ph1, pl1;
+          split_bf16(st[0], st[1], ph0, pl0);   // keys 0-7
+          split_bf16(st[2], st[3], ph1, pl1);   // keys 8-15
+          ph0 = movmatrix_t(ph0); ph1 = movmatrix_t(ph1);
+          pl0 = movmatrix_t(pl0); pl1 = movmatrix_t(pl1);
+          uint32_t va[D / 16][4];
 #pragma unroll
-        for (int jt = 0; jt < D / 16; ++jt) {
-          ldsm_x4_t(vb + v_tok * kRowBytes + (((2 * jt + v_chk) ^ (v_tok & 7)) << 4), va[jt][0], va[jt][1],
-                    va[jt][2], va[jt][3]);
-          o[jt][0] *= a0; o[jt][1] *= a1;
-          o[jt][2] *= a0; o[jt][3] *= a1;
+          for (int jt = 0; jt < D / 16; ++jt) {
+            ldsm_x4_t(vb + v_tok * kRowBytes + (((2 * jt + v_chk) ^ (v_tok & 7)) << 4), va[jt][0], va[jt][1],
+                      va[jt][2], va[jt][3]);
+            o[jt][0] *= a0; o[jt][1] *= a1;
+            o[jt][2] *= a0; o[jt][3] *= a1;
+          }
+#pragma unroll
+          for (int jt = 0; jt < D / 16; ++jt) mma_bf16(o[jt], va[jt], ph0, ph1);
+#pragma unroll
+          for (int jt = 0; jt < D / 16; ++jt) mma_bf16(o[jt], va[jt], pl0, pl1);
+        } else {
+          // P^T as one fp16 term (11 significant bits against the 4 of the stored V), each
+          // weight already multiplied by its V row's 2^X
+          const uint32_t ph0 = movmatrix_t(pack_f16(st[0] * vscale0, st[1] * vscale0));   // keys 0-7
+          const uint32_t ph1 = movmatrix_t(pack_f16(st[2] * vscale1, st[3] * vscale1));   // keys 8-15
+#pragma unroll
+          for (int jt = 0; jt < D / 16; ++jt) {
+            o[jt][0] *= a0; o[jt][1] *= a1;
+            o[jt][2] *= a0; o[jt][3] *= a1;
+          }
+          // A transposed 8x8 tile of byte pairs gives this thread keys 2t, 2t+1 of the channel
+          // pair 2 frow, 2 frow + 1: the even channel becomes accumulator row frow, the odd one
+          // row frow + 8 (see the merge below)
+#pragma unroll
+          for (int j = 0; j < D / 32; ++j) {
+            uint32_t r[4];
+            ldsm_x4_t(vb + k_tok * kRowBytes + (((2 * j + k_chk) ^ (k_tok & 7)) << 4), r[0], r[1], r[2], r[3]);
+#pragma unroll
+            for (int c = 0; c < 2; ++c) {
+              const uint32_t lo = __byte_perm(r[2 * c], 0u, 0x3120), hi = __byte_perm(r[2 * c + 1], 0u, 0x3120);
+              const uint32_t a[4] = {e4m3x2_to_f16x2(lo), e4m3x2_to_f16x2(lo >> 16),
+                                     e4m3x2_to_f16x2(hi), e4m3x2_to_f16x2(hi >> 16)};
+              mma_f16(o[2 * j + c], a, ph0, ph1);
+            }
+          }
         }
-#pragma unroll
-        for (int jt = 0; jt < D / 16; ++jt) mma_bf16(o[jt], va[jt], ph0, ph1);
-#pragma unroll
-        for (int jt = 0; jt < D / 16; ++jt) mma_bf16(o[jt], va[jt], pl0, pl1);
       }
       __syncwarp();
       if (lane == 0) mbar_arrive(empty0 + 8 * s);
@@ -428,8 +524,13 @@ decode_split_bf16_kernel(const __grid_constant__ DecodeParams p, const int n_sta
       if (r < rows) {
 #pragma unroll
         for (int jt = 0; jt < D / 16; ++jt) {
-          mo[r * D + jt * 16 + frow] = o[jt][e];
-          mo[r * D + jt * 16 + frow + 8] = o[jt][2 + e];
+          if constexpr (!KV8) {
+            mo[r * D + jt * 16 + frow] = o[jt][e];
+            mo[r * D + jt * 16 + frow + 8] = o[jt][2 + e];
+          } else {   // accumulator rows frow / frow + 8 are channels 2 frow / 2 frow + 1 of the block
+            mo[r * D + jt * 16 + 2 * frow] = o[jt][e];
+            mo[r * D + jt * 16 + 2 * frow + 1] = o[jt][2 + e];
+          }
         }
         if (frow == 0) { mml[r * 2] = m[e]; mml[r * 2 + 1] = l[e]; }
       }
@@ -503,9 +604,9 @@ decode_split_bf16_kernel(const __grid_constant__ DecodeParams p, const int n_sta
   }
 }
 
-size_t smem_bytes(int D, int group, int n_stages, int ncw, int cl) {
+size_t smem_bytes(int D, int group, int n_stages, int ncw, int cl, int kv8) {
   const int rows_cap = group < kMaxGroupRows ? group : kMaxGroupRows;
-  size_t stage = (size_t)kGroupWarps * 2 * kPage * D * 2;
+  size_t stage = (size_t)kGroupWarps * (kv8 ? 2 * kPage * D + 2 * kPage : 2 * kPage * D * 2);
   const size_t exchange = cl > 1 ? (size_t)cl * rows_cap * (D + 2) * 4 : 0;
   return n_stages * stage + (size_t)ncw * rows_cap * (D + 2) * 4 + 2 * kMaxStages * 8 + 32 + exchange;
 }
@@ -513,12 +614,16 @@ size_t smem_bytes(int D, int group, int n_stages, int ncw, int cl) {
 }  // namespace
 
 cudaError_t prepare_decode_bf16() {
-  cudaError_t e = cudaFuncSetAttribute(decode_split_bf16_kernel<128, 8, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(decode_split_bf16_kernel<64, 8, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(decode_split_bf16_kernel<128, 4, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 113 * 1024);
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(decode_split_bf16_kernel<64, 4, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 113 * 1024);
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(decode_split_bf16_kernel<128, 8, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(decode_split_bf16_kernel<64, 8, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+  cudaError_t e = cudaFuncSetAttribute(decode_split_bf16_kernel<128, 8, 1, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(decode_split_bf16_kernel<64, 8, 1, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(decode_split_bf16_kernel<128, 4, 1, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, 113 * 1024);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(decode_split_bf16_kernel<64, 4, 1, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, 113 * 1024);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(decode_split_bf16_kernel<128, 8, 2, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(decode_split_bf16_kernel<64, 8, 2, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+  // quantised cache: head_dim 128 only
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(decode_split_bf16_kernel<128, 8, 1, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(decode_split_bf16_kernel<128, 4, 1, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 113 * 1024);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(decode_split_bf16_kernel<128, 8, 2, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
   return e;
 }
 
@@ -536,13 +641,15 @@ cudaError_t launch_decode_split_bf16(const DecodeParams& p, int sm_count, cudaSt
   const int cl = paired ? 2 : 1;
   const int ncw = small ? 4 : 8;
   const size_t budget = small ? 110 * 1024 : 220 * 1024;
+  const int kv8 = p.geom.fp8;
+  if (kv8 && D != 128) return cudaErrorInvalidValue;
   int n_stages = kMaxStages;
-  while (n_stages > 2 && smem_bytes(D, p.group, n_stages, ncw, cl) > budget) --n_stages;
+  while (n_stages > 2 && smem_bytes(D, p.group, n_stages, ncw, cl, kv8) > budget) --n_stages;
   // Two consumer groups take alternate tiles: with an even ring every stage always belongs to the
   // same group, which then waits for its phases one after the other (a parity wait is only valid
   // for the phase right after the last one known complete).
   if (ncw == 8 && (n_stages & 1)) --n_stages;
-  const size_t smem = smem_bytes(D, p.group, n_stages, ncw, cl);
+  const size_t smem = smem_bytes(D, p.group, n_stages, ncw, cl, kv8);
   const int slots = small ? 2 * sm_count : sm_count;
   const int grid = paired ? 2 * p.total_items : (p.total_items < slots ? p.total_items : slots);
   // launched with programmatic stream serialization: the kernel's set-up may overlap the
@@ -562,14 +669,19 @@ cudaError_t launch_decode_split_bf16(const DecodeParams& p, int sm_count, cudaSt
   attr[1].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = paired ? 2 : 1;
-  if (D == 128) {
-    if (paired) return cudaLaunchKernelEx(&cfg, decode_split_bf16_kernel<128, 8, 2>, p, n_stages);
-    if (small) return cudaLaunchKernelEx(&cfg, decode_split_bf16_kernel<128, 4, 1>, p, n_stages);
-    return cudaLaunchKernelEx(&cfg, decode_split_bf16_kernel<128, 8, 1>, p, n_stages);
+  if (kv8) {
+    if (paired) return cudaLaunchKernelEx(&cfg, decode_split_bf16_kernel<128, 8, 2, 1>, p, n_stages);
+    if (small) return cudaLaunchKernelEx(&cfg, decode_split_bf16_kernel<128, 4, 1, 1>, p, n_stages);
+    return cudaLaunchKernelEx(&cfg, decode_split_bf16_kernel<128, 8, 1, 1>, p, n_stages);
   }
-  if (paired) return cudaLaunchKernelEx(&cfg, decode_split_bf16_kernel<64, 8, 2>, p, n_stages);
-  if (small) return cudaLaunchKernelEx(&cfg, decode_split_bf16_kernel<64, 4, 1>, p, n_stages);
-  return cudaLaunchKernelEx(&cfg, decode_split_bf16_kernel<64, 8, 1>, p, n_stages);
+  if (D == 128) {
+    if (paired) return cudaLaunchKernelEx(&cfg, decode_split_bf16_kernel<128, 8, 2, 0>, p, n_stages);
+    if (small) return cudaLaunchKernelEx(&cfg, decode_split_bf16_kernel<128, 4, 1, 0>, p, n_stages);
+    return cudaLaunchKernelEx(&cfg, decode_split_bf16_kernel<128, 8, 1, 0>, p, n_stages);
+  }
+  if (paired) return cudaLaunchKernelEx(&cfg, decode_split_bf16_kernel<64, 8, 2, 0>, p, n_stages);
+  if (small) return cudaLaunchKernelEx(&cfg, decode_split_bf16_kernel<64, 4, 1, 0>, p, n_stages);
+  return cudaLaunchKernelEx(&cfg, decode_split_bf16_kernel<64, 8, 1, 0>, p, n_stages);
 }
 
 }  // namespace mixattn

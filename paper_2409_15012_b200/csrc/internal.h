@@ -24,36 +24,48 @@ constexpr int kWsChunks = kMaxCallSeqs + kWsExtraChunks + kWsWaveChunks;  // spl
 // chunks of a token row are stored XOR-swizzled by (token & 7): the block in HBM is
 // already the bank-conflict-free shared-memory image that ldmatrix wants, and the
 // copy engine needs no tensor map.  fp32 rows are stored unswizzled.
+// Quantised storage (FP8 E4M3 elements, one shared exponent byte per stored row): the rows
+// are D bytes, swizzled the same way, and the block ends with the 16 exponent bytes of its K
+// rows and the 16 of its V rows:  [K: 16 x D B][V: 16 x D B][X_K: 16 B][X_V: 16 B].
 // ---------------------------------------------------------------------------
 struct KvGeom {
   int32_t n_kv_heads;
   int32_t head_dim;
-  int32_t elem_bytes;     // 2 or 4
-  int32_t row_bytes;      // head_dim * elem_bytes
-  int32_t blk_bytes;      // 2 * 16 * row_bytes: K and V of one (page, head)
-  int32_t swizzle;        // 1 in bf16 mode
+  int32_t elem_bytes;     // of Q / K / V / out as the caller passes them: 2 or 4
+  int32_t row_bytes;      // head_dim * elem_bytes: one head vector in the caller's tensors
+  int32_t st_row_bytes;   // one stored head vector: row_bytes, or head_dim for quantised storage
+  int32_t fp8;            // 1: quantised storage
+  int32_t blk_bytes;      // K and V (and exponents) of one (page, head)
+  int32_t swizzle;        // 1 unless fp32
   int64_t page_bytes;     // n_kv_heads * blk_bytes
 };
 
-__host__ __device__ inline KvGeom make_geom(int n_kv_heads, int head_dim, int dtype) {
+__host__ __device__ inline KvGeom make_geom(int n_kv_heads, int head_dim, int dtype, int kv_format) {
   KvGeom g;
   g.n_kv_heads = n_kv_heads;
   g.head_dim = head_dim;
   g.elem_bytes = dtype == MIXATTN_BF16 ? 2 : 4;
   g.row_bytes = head_dim * g.elem_bytes;
-  g.blk_bytes = 2 * kPage * g.row_bytes;
+  g.fp8 = kv_format == MIXATTN_KV_FP8_E4M3 ? 1 : 0;
+  g.st_row_bytes = g.fp8 ? head_dim : g.row_bytes;
+  g.blk_bytes = 2 * kPage * g.st_row_bytes + (g.fp8 ? 2 * kPage : 0);
   g.swizzle = dtype == MIXATTN_BF16 ? 1 : 0;
   g.page_bytes = (int64_t)n_kv_heads * g.blk_bytes;
   return g;
 }
 
-// Byte offset, inside a pool, of 16-byte chunk `chunk` of token slot `tok` (0..15) of
-// page `page`, KV head `g`, which = 0 (K) or 1 (V).
+// Byte offset, inside a pool, of 16-byte chunk `chunk` of the stored row of token slot `tok`
+// (0..15) of page `page`, KV head `g`, which = 0 (K) or 1 (V).
 __host__ __device__ inline int64_t kv_chunk_offset(const KvGeom& ge, int64_t page, int g, int which,
                                                    int tok, int chunk) {
   int c = ge.swizzle ? (chunk ^ (tok & 7)) : chunk;
-  return page * ge.page_bytes + (int64_t)g * ge.blk_bytes + (int64_t)which * kPage * ge.row_bytes +
-         (int64_t)tok * ge.row_bytes + (int64_t)c * 16;
+  return page * ge.page_bytes + (int64_t)g * ge.blk_bytes + (int64_t)which * kPage * ge.st_row_bytes +
+         (int64_t)tok * ge.st_row_bytes + (int64_t)c * 16;
+}
+
+// Quantised storage: byte offset of the shared-exponent byte of that row.
+__host__ __device__ inline int64_t kv_exp_offset(const KvGeom& ge, int64_t page, int g, int which, int tok) {
+  return page * ge.page_bytes + (int64_t)g * ge.blk_bytes + 2 * kPage * ge.st_row_bytes + which * kPage + tok;
 }
 
 // ---------------------------------------------------------------------------
@@ -169,7 +181,7 @@ cudaError_t launch_append(const AppendParams& p, int max_n_new, cudaStream_t st)
 cudaError_t launch_table_set(const TableSetParams& p, cudaStream_t st);
 cudaError_t launch_gather(const GatherParams& p, int max_rows, cudaStream_t st);
 cudaError_t prepare_decode_bf16();
-cudaError_t launch_decode_split_bf16(const DecodeParams& p, int sm_count, cudaStream_t st);
+cudaError_t launch_decode_split_bf16(const DecodeParams& p, int sm_count, cudaStream_t st);   // native or quantised cache
 cudaError_t launch_decode_split_f32(const DecodeParams& p, cudaStream_t st);
 cudaError_t launch_decode_combine(const DecodeParams& p, int dtype, cudaStream_t st);
 cudaError_t launch_prefill_simple(const PrefillParams& p, int dtype, int max_len, cudaStream_t st);

@@ -29,7 +29,7 @@ class Session:
 
     def __init__(self, wl: cf.Workload, lengths: Optional[Sequence[int]] = None, device: int = 0,
                  headroom_tokens: int = 0, free_order=None, n_pages: Optional[int] = None,
-                 mirror=None, chunk_scratch_tokens: int = 0, gen_device=None):
+                 mirror=None, chunk_scratch_tokens: int = 0, gen_device=None, kv_format: int = mx.KV_NATIVE):
         self.wl = wl
         self.device = device
         self.dev = torch.device(f"cuda:{device}")
@@ -55,7 +55,8 @@ class Session:
         self.mirror = mirror
         self.ctx = mx.Context(wl.layout, wl.n_q_heads, wl.n_kv_heads, wl.head_dim, wl.dtype, B,
                               n_pages, max_seq_len=max(max_len, 1), free_order=free_order, device=device,
-                              chunk_scratch_tokens=chunk_scratch_tokens)
+                              chunk_scratch_tokens=chunk_scratch_tokens, kv_format=kv_format)
+        self.kv_format = kv_format
 
     def close(self):
         self.ctx.close()
@@ -194,12 +195,15 @@ class Session:
             self.mirror.append(layer, ids, lens)
 
 
-def kv_bytes_per_step(wl: cf.Workload, lengths_after: Sequence[int]) -> int:
+def kv_bytes_per_step(wl: cf.Workload, lengths_after: Sequence[int], kv_format: int = mx.KV_NATIVE) -> int:
     """KV bytes one decode step reads: per layer and sequence min(n, window)
-    (or n) tokens of 2 * Hkv * D elements; a shared cache counts once per
-    reading layer."""
+    (or n) tokens of 2 * Hkv * D elements (quantised storage: one byte per
+    element plus one exponent byte per head vector); a shared cache counts once
+    per reading layer."""
     e = 2 if wl.dtype == cf.BF16 else 4
     per_tok = 2 * wl.n_kv_heads * wl.head_dim * e
+    if kv_format == mx.KV_FP8_E4M3:
+        per_tok = 2 * wl.n_kv_heads * (wl.head_dim + 1)
     total = 0
     for kind, window, _ in wl.layout:
         for n in lengths_after:

@@ -186,3 +186,24 @@ def test_chunk_and_rope_calls_on_a_host_only_context():
     assert ctx.rc_attend_chunk(1, [0], [25], None, None, None, None) == mx.ERR_CUDA
     ctx.set_chunk_gather_reuse(False)
     ctx.close()
+
+
+def test_quantised_storage_config_rules_and_cache_bytes():
+    # quantised KV storage needs bf16 I/O and head_dim 128; it stores head_dim + 1 bytes per head vector
+    lay = cf.layout_mid(1024)
+    ok = mx.make_config(lay, 32, 8, 128, mx.BF16, 4, 100, kv_format=mx.KV_FP8_E4M3)[0]
+    native = mx.make_config(lay, 32, 8, 128, mx.BF16, 4, 100)[0]
+    assert mx.cache_bytes(ok) * 2 * 128 == mx.cache_bytes(native) * 129
+    for bad in (mx.make_config(lay, 32, 8, 128, mx.F32, 4, 100, kv_format=mx.KV_FP8_E4M3),
+                mx.make_config(lay, 32, 8, 64, mx.BF16, 4, 100, kv_format=mx.KV_FP8_E4M3)):
+        with pytest.raises(mx.MixAttnError) as ei:
+            mx.cache_bytes(bad[0])
+        assert ei.value.code == mx.ERR_UNSUPPORTED
+    with pytest.raises(mx.MixAttnError) as ei:
+        mx.cache_bytes(mx.make_config(lay, 32, 8, 128, mx.BF16, 4, 100, kv_format=7)[0])
+    assert ei.value.code == mx.ERR_INVALID_ARG
+    # a host-only quantised context keeps the same bookkeeping
+    ctx = mx.Context(lay, 32, 8, 128, mx.BF16, 4, 100, device=-1, kv_format=mx.KV_FP8_E4M3)
+    ctx.append_kv(0, [0, 1], [20, 3])
+    assert ctx.get_len(12, 0) == 20 and ctx.get_block_table(0) == [0, 1] and ctx.get_block_table(1) == [2]
+    ctx.close()
