@@ -470,7 +470,8 @@ def run_gpu_arm(args, wl):
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()          # before the fill and the warm-up: the GPU is under load when timing starts
-    sess, lengths = make_session(runner, wl, local, total_steps)
+    kvf = mx.KV_FP8_E4M3 if args.kv_format == "fp8" else mx.KV_NATIVE
+    sess, lengths = make_session(runner, wl, local, total_steps, kvf)
     stream = torch.cuda.current_stream()
     outs = sess.alloc_outputs()
 
@@ -480,7 +481,7 @@ def run_gpu_arm(args, wl):
         torch.cuda.synchronize()
 
     def bytes_next_step():
-        return runner.kv_bytes_per_step(wl, [int(p) + 1 for p in sess.pos])
+        return runner.kv_bytes_per_step(wl, [int(p) + 1 for p in sess.pos], kvf)
 
     # ---- device-resident pass: `value` ----
     kRing = min(8, Wm + K)
@@ -584,7 +585,7 @@ def run_gpu_arm(args, wl):
     full_layers = [l for l, (kind, _, _) in enumerate(wl.layout) if kind == cf.FULL]
     slide_layers = [l for l, (kind, _, _) in enumerate(wl.layout) if kind == cf.SLIDING]
     e = 2 if wl.dtype == cf.BF16 else 4
-    per_tok = 2 * wl.n_kv_heads * wl.head_dim * e
+    per_tok = 2 * wl.n_kv_heads * (wl.head_dim + 1 if kvf else wl.head_dim * e)
     sess.ctx.profile_enable(True)
     full_bytes = 0
     Kp = min(K, 20)
@@ -615,7 +616,7 @@ def run_gpu_arm(args, wl):
         "kernel": "decode_split_bf16_kernel (standard layer)" if wl.dtype == cf.BF16 else "decode_split_f32_kernel",
         "bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
         "frac": achieved / peaks["hbm_gbs"],
-        "traffic": None if DECODE_FULL_TRAFFIC_RATIO is None else DECODE_FULL_TRAFFIC_RATIO * bytes_per_launch,
+        "traffic": None if DECODE_FULL_TRAFFIC_RATIO is None or kvf else DECODE_FULL_TRAFFIC_RATIO * bytes_per_launch,
         "peak_source": f"of {peaks['_source']}", "bytes_per_launch": bytes_per_launch,
         "us_per_launch": sec_per_launch * 1e6, "frac_of_nominal_8TBs": achieved / 8000.0,
     }
@@ -642,7 +643,7 @@ def run_gpu_arm(args, wl):
         closed = True
         prefill = prefill_figures(mx, runner, peaks, local)
         prefill["chunked"] = chunk_figures(mx, runner, peaks, local)
-    if not args.no_other_workloads and world == 1 and args.workload == "mid_decode" and args.batch == 0:
+    if not args.no_other_workloads and world == 1 and args.workload == "mid_decode" and args.batch == 0 and not kvf:
         if not closed:
             sess.close()
             closed = True
@@ -652,7 +653,7 @@ def run_gpu_arm(args, wl):
         "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": K, "warmup": Wm,
         "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16" if wl.dtype == cf.BF16 else "f32", "data": "synthetic",
-        "config": {"workload": wl.name, "batch": wl.batch, "context": wl.context or list(wl.context_range),
+        "config": {"workload": wl.name + ("_fp8_kv" if kvf else ""), "batch": wl.batch, "context": wl.context or list(wl.context_range),
                    "window": 1024, "layers": len(wl.layout), "heads": f"{wl.n_q_heads}/{wl.n_kv_heads}x{wl.head_dim}",
                    "l2": "inputs larger than L2 (KV read per step >> 126 MB)", "parallelism": "replicas only"},
         "tokens_per_s": wl.batch * world / (ms / K * 1e-3),
@@ -750,6 +751,8 @@ def main():
     ap.add_argument("--no-prefill", action="store_true")
     ap.add_argument("--no-other-workloads", action="store_true",
                     help="skip the compact figures of the other decode configurations")
+    ap.add_argument("--kv-format", default="native", choices=["native", "fp8"],
+                    help="fp8: quantised KV storage (FP8 E4M3 elements); bytes counted are the quantised cache's")
     ap.add_argument("--trace", action="store_true", help="paper-shaped serving trace instead of the decode step")
     ap.add_argument("--trace-requests", type=int, default=8)
     ap.add_argument("--trace-prompt", type=int, default=31000)

@@ -776,16 +776,24 @@ static int stored_page_of(mixattn_ctx* c, int layer, int seq, int pos, int64_t* 
 static int read_stored_row(mixattn_ctx* c, const char* pool, int64_t phys, int gh, int which, int slot,
                            void* dst, int32_t* X) {
   const KvGeom& ge = c->geom;
-  unsigned char row[512];
-  if (ge.st_row_bytes > (int)sizeof(row)) return MIXATTN_ERR_UNSUPPORTED;
-  // start of the stored row; its 16-byte chunks are permuted unless the cache is fp32
-  const char* src = pool + phys * ge.page_bytes + (int64_t)gh * ge.blk_bytes +
-                    (int64_t)(which * kPage + slot) * ge.st_row_bytes;
-  if (cudaMemcpy(row, src, ge.st_row_bytes, cudaMemcpyDeviceToHost) != cudaSuccess) return MIXATTN_ERR_CUDA;
-  const int chunks = ge.st_row_bytes / 16;
-  for (int ch = 0; ch < chunks; ++ch) {
-    const int phys_ch = ge.swizzle ? (ch ^ (slot & 7)) : ch;
-    memcpy(static_cast<char*>(dst) + ch * 16, row + phys_ch * 16, 16);
+  if (ge.fp8 && which == 1) {
+    // quantised V is stored transposed: fetch the page's V^T and pick this token's column
+    std::vector<unsigned char> vt((size_t)ge.head_dim * kPage);
+    if (cudaMemcpy(vt.data(), pool + kv_fp8_v_offset(ge, phys, gh, 0, 0), vt.size(), cudaMemcpyDeviceToHost) != cudaSuccess)
+      return MIXATTN_ERR_CUDA;
+    for (int d = 0; d < ge.head_dim; ++d) static_cast<unsigned char*>(dst)[d] = vt[(size_t)d * kPage + slot];
+  } else {
+    unsigned char row[512];
+    if (ge.st_row_bytes > (int)sizeof(row)) return MIXATTN_ERR_UNSUPPORTED;
+    // start of the stored row; its 16-byte chunks are permuted unless the cache is fp32
+    const char* src = pool + phys * ge.page_bytes + (int64_t)gh * ge.blk_bytes +
+                      (int64_t)(which * kPage + slot) * ge.st_row_bytes;
+    if (cudaMemcpy(row, src, ge.st_row_bytes, cudaMemcpyDeviceToHost) != cudaSuccess) return MIXATTN_ERR_CUDA;
+    const int chunks = ge.st_row_bytes / 16;
+    for (int ch = 0; ch < chunks; ++ch) {
+      const int phys_ch = !ge.swizzle ? ch : ge.fp8 ? (ch ^ fp8_k_swizzle(slot)) : (ch ^ (slot & 7));
+      memcpy(static_cast<char*>(dst) + ch * 16, row + phys_ch * 16, 16);
+    }
   }
   if (ge.fp8 && X != nullptr) {
     unsigned char xb = 0;

@@ -151,9 +151,14 @@ __global__ void __launch_bounds__(kThreads) append_fp8_kernel(const __grid_const
       page = e.page_hint >= 0 ? e.page_hint : p.table[(int64_t)e.seq * p.table_stride + pos / kPage];
       slot = pos % kPage;
     }
-    // two lanes share a 16-byte chunk of the stored row
-    char* dst = p.pool + kv_chunk_offset(ge, page, g, which, slot, sub >> 1) + (sub & 1) * 8;
-    *reinterpret_cast<uint2*>(dst) = make_uint2(lo, hi);
+    if (which == 0) {   // K: two lanes share a 16-byte chunk of the stored row
+      char* dst = p.pool + kv_chunk_offset(ge, page, g, 0, slot, sub >> 1) + (sub & 1) * 8;
+      *reinterpret_cast<uint2*>(dst) = make_uint2(lo, hi);
+    } else {            // V is stored transposed: this token's byte of each channel row
+      unsigned char* dst = reinterpret_cast<unsigned char*>(p.pool) + kv_fp8_v_offset(ge, page, g, sub * 8, slot);
+#pragma unroll
+      for (int i = 0; i < 8; ++i) dst[i * kPage] = (unsigned char)((i < 4 ? lo >> (8 * i) : hi >> (8 * (i - 4))) & 0xffu);
+    }
     if (sub == 0) *reinterpret_cast<unsigned char*>(p.pool + kv_exp_offset(ge, page, g, which, slot)) = (unsigned char)(X + 127);
   }
 }

@@ -7,11 +7,14 @@
 //   * persistent CTAs (one per SM) walk a static list of work items
 //     (sequence, split of its keys, KV head); the GQA query heads of that KV head
 //     (up to 16) are the rows of one tensor-core tile, so K/V is read once per group;
-//   * one producer warp streams (page, head) blocks -- 16 keys of K and V, contiguous in
+//   * producer warps stream (page, head) blocks -- 16 keys of K and V, contiguous in
 //     HBM, already in the swizzled shared-memory image -- with one bulk async copy each
 //     into a ring of 64-key stages guarded by full/empty mbarriers; the ring keeps
 //     running across work items, so the next item's keys arrive during this item's
-//     epilogue;
+//     epilogue.  One producer warp needs about 850 cycles per stage (four copy issues, two
+//     barrier operations, the table lookup): enough for 32 KB stages, but the 16 KB stages
+//     of the quantised cache are streamed by four producer warps that take the stages in
+//     turn;
 //   * eight consumer warps, two groups alternating stages, one 16-key page per warp:
 //     S^T = K Q^T and O^T += V^T P^T on mma.sync m16n8k16 (bf16 in, fp32 out) with the
 //     keys as the M dimension and the heads as N = 8, online softmax in base 2, private
@@ -25,11 +28,16 @@
 //     CTA ingests K/V at a bounded rate, so idle SMs are better used than a second launch.
 //
 // Quantised cache (paper, Section 2, "KV Quantization"; KV8 instantiations): a (page, head)
-// block holds FP8 E4M3 rows and one shared power-of-two exponent per row, half the bytes per
-// key.  The same stream and the same tile shapes; the elements are widened exactly to fp16
-// after ldmatrix (a 32-bit fragment register then holds four channels of one key, so Q is
-// loaded in the matching channel order), the products run on the fp16 tensor-core path, a K
-// row's exponent multiplies its scores and a V row's exponent is folded into its weight.
+// block holds FP8 E4M3 elements and one shared power-of-two exponent per head vector, half
+// the bytes per key, so the arithmetic per byte doubles and the instruction count per page is
+// what has to stay small.  The same stream and tile shapes; the elements are widened exactly
+// to fp16 right after ldmatrix (two conversions per 32-bit fragment register, nothing else)
+// and the products run on the fp16 tensor-core path.  A fragment register holds four
+// consecutive bytes: four channels of a key for K, four keys of a channel for V, which is
+// stored transposed.  Q is therefore loaded in the matching channel order, and the 16 keys of
+// a page take the tile rows in the order 0 1 4 5 8 9 12 13 | 2 3 6 7 10 11 14 15, which is
+// the key order the transposed weights then have in the second product.  A K row's exponent
+// multiplies its scores; a V row's exponent is folded into its weight.
 //
 // Every mbarrier wait is bounded: on time-out the kernel raises a status word and all
 // roles leave.
@@ -45,7 +53,7 @@ namespace {
 
 constexpr int kGroupWarps = 4;                      // warps (= pages) per stage
 constexpr int kTileKeys = kGroupWarps * kPage;      // 64 keys per stage
-constexpr int kMaxStages = 8;
+constexpr int kMaxStages = 12;
 constexpr long long kWaitLimitCycles = 4000000000ll;   // about two seconds of SM clock
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
@@ -134,19 +142,26 @@ __device__ __forceinline__ void mma_f16(float (&d)[4], const uint32_t (&a)[4], u
       : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
       : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
-// two E4M3 codes (low 16 bits of x) -> packed fp16 pair, exact
-__device__ __forceinline__ uint32_t e4m3x2_to_f16x2(uint32_t x) {
-  const __half2_raw h = __nv_cvt_fp8x2_to_halfraw2((__nv_fp8x2_storage_t)(x & 0xffffu), __NV_E4M3);
-  return (uint32_t)h.x | ((uint32_t)h.y << 16);
+// four E4M3 codes -> two packed fp16 pairs (bytes 0, 1 and bytes 2, 3), exact
+__device__ __forceinline__ void e4m3x4_to_f16x2x2(uint32_t x, uint32_t& lo, uint32_t& hi) {
+  asm("{\n\t.reg .b16 l, h;\n\t"
+      "mov.b32 {l, h}, %2;\n\t"
+      "cvt.rn.f16x2.e4m3x2 %0, l;\n\t"
+      "cvt.rn.f16x2.e4m3x2 %1, h;\n\t}"
+      : "=r"(lo), "=r"(hi) : "r"(x));
+}
+__device__ __forceinline__ float ex2_ftz(float x) {   // 2^x, one MUFU op; 2^-inf = 0
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
 }
 __device__ __forceinline__ uint32_t pack_f16(float lo, float hi) {
   const __half2 t = __floats2half2_rn(lo, hi);
   return *reinterpret_cast<const uint32_t*>(&t);
 }
-// 2^X from the stored exponent byte X + 127 (byte 0 is 2^-127, a subnormal)
-__device__ __forceinline__ float exp_byte_to_float(uint32_t b) {
-  return __int_as_float(b ? (int)(b << 23) : 0x00400000);
-}
+// 2^X from the stored exponent byte X + 127.  Byte 0 (X = -127: a zero vector, or one whose
+// largest element is below 2^-118) reads as 0 instead of 2^-127.
+__device__ __forceinline__ float exp_byte_to_float(uint32_t b) { return __int_as_float((int)(b << 23)); }
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   __nv_bfloat162 t = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<uint32_t*>(&t);
@@ -226,10 +241,17 @@ __device__ __forceinline__ void cluster_share(Item& x, int crank) {
 // ingests K/V at a fixed rate, so a short launch that leaves SMs idle is halved this way
 // without a second launch.  The grid then holds exactly one cluster per item.
 // KV8 = 1: the cache holds FP8 E4M3 rows with shared exponents (see the top of the file).
+// Producer warps of a variant.  With more than one, the ring length must be a multiple of their
+// number (checked by the launcher): a stage then always belongs to the same producer, whose
+// program order keeps its waits on that stage's barriers one phase apart.  (A producer that
+// waited for a phase two ahead of the barrier's would be answered "complete" by the parity test.)
+__host__ __device__ constexpr int producer_warps(int ncw, int kv8) { return (kv8 && ncw == 8) ? 4 : 1; }
+
 template <int D, int NCW, int CL, int KV8>
-__global__ void __launch_bounds__((NCW + 1) * 32, NCW == 8 ? 1 : 2)
+__global__ void __launch_bounds__((NCW + producer_warps(NCW, KV8)) * 32, NCW == 4 ? 2 : 1)
 decode_split_bf16_kernel(const __grid_constant__ DecodeParams p, const int n_stages) {
   constexpr int kConsumerWarps = NCW;
+  constexpr int kProducerWarps = producer_warps(NCW, KV8);
   constexpr int kGroups = NCW / kGroupWarps;
   constexpr int kRowBytes = KV8 ? D : D * 2;
   constexpr int kBlkBytes = 2 * kPage * kRowBytes + (KV8 ? 2 * kPage : 0);   // K+V (+ exponents) of one (page, head)
@@ -278,9 +300,12 @@ decode_split_bf16_kernel(const __grid_constant__ DecodeParams p, const int n_sta
 
   const KvGeom& ge = p.geom;
 
-  if (warp == kConsumerWarps) {
-    // ------------------------------ producer ------------------------------
-    int K = 0;  // tiles issued by this CTA so far
+  if (warp >= kConsumerWarps) {
+    // ------------------------------ producers ------------------------------
+    // every producer warp walks the whole tile sequence and issues the tiles K with
+    // K % kProducerWarps == pw
+    const int pw = warp - kConsumerWarps;
+    int K = 0;  // tiles of this CTA so far (all producers)
     bool ok = true;
     const uint64_t l2_policy = l2_policy_of(p.pool, p.l2_keep_bytes, p.l2_pool_bytes);
     for (int it = item0; ok && it < p.total_items; it += item_stride) {
@@ -302,6 +327,7 @@ decode_split_bf16_kernel(const __grid_constant__ DecodeParams p, const int n_sta
           ids = ids_next;
           if (tbl && pg + 32 + lane < page_hi) ids_next = tbl[pg + 32 + lane];
         }
+        if (kProducerWarps > 1 && K % kProducerWarps != pw) continue;
         const int s = K % n_stages;
         if (K >= n_stages) {  // lane 0 waits; the verdict is made warp-uniform
           int w = 1;
@@ -324,7 +350,7 @@ decode_split_bf16_kernel(const __grid_constant__ DecodeParams p, const int n_sta
       atomicExch(p.status, kDevWaitTimeout);
       for (int back = 1; back <= n_stages && K - back >= 0; ++back) {
         const int Kb = K - back;
-        mbar_wait(full0 + 8 * (Kb % n_stages), (Kb / n_stages) & 1, abort_flag + 1);
+        if (Kb % kProducerWarps == pw) mbar_wait(full0 + 8 * (Kb % n_stages), (Kb / n_stages) & 1, abort_flag + 1);
       }
     }
     if constexpr (CL > 1) {
@@ -351,6 +377,9 @@ decode_split_bf16_kernel(const __grid_constant__ DecodeParams p, const int n_sta
   const int lm = lane >> 3, lr = lane & 7;
   const int k_tok = (lm & 1) * 8 + lr, k_chk = lm >> 1;   // K as A: (keys 0-7|8-15) x (chunk 2ks|2ks+1)
   const int v_tok = (lm >> 1) * 8 + lr, v_chk = lm & 1;   // V^T as A (.trans): (chunk 2jt|2jt+1) x (keys 0-7|8-15)
+  // quantised cache: tile row r of a page is key 4 (r >> 1) + (r & 1) for r < 8 and that + 2 for r - 8
+  const int k8_tok = 4 * (lr >> 1) + (lr & 1) + 2 * (lm & 1);   // key whose K row this lane addresses
+  const int key0 = 4 * (frow >> 1) + (frow & 1);                // this thread's score rows: keys key0 and key0 + 2
 
   int K = 0;
   for (int it = item0; it < p.total_items; it += item_stride) {
@@ -416,31 +445,31 @@ decode_split_bf16_kernel(const __grid_constant__ DecodeParams p, const int n_sta
 #pragma unroll
           for (int e = 0; e < 4; ++e) st[e] = (st[e] + st2[e]) * p.scale_log2e;
         } else {
-          // one ldmatrix.x4 = (keys 0-7 | 8-15) x (16-byte chunk 2j | 2j+1) = two 16-channel steps
+          // one ldmatrix.x4 = (tile rows 0-7 | 8-15) x (16-byte chunk 2j | 2j+1) = two 16-channel steps
 #pragma unroll
           for (int j = 0; j < kKSteps / 2; ++j) {
-            uint32_t r[4];
-            ldsm_x4(kb + k_tok * kRowBytes + (((2 * j + k_chk) ^ (k_tok & 7)) << 4), r[0], r[1], r[2], r[3]);
-            const uint32_t a[4] = {e4m3x2_to_f16x2(r[0]), e4m3x2_to_f16x2(r[1]),
-                                   e4m3x2_to_f16x2(r[0] >> 16), e4m3x2_to_f16x2(r[1] >> 16)};
-            const uint32_t b[4] = {e4m3x2_to_f16x2(r[2]), e4m3x2_to_f16x2(r[3]),
-                                   e4m3x2_to_f16x2(r[2] >> 16), e4m3x2_to_f16x2(r[3] >> 16)};
+            uint32_t r[4], a[4], b[4];
+            ldsm_x4(kb + k8_tok * kRowBytes + (((2 * j + k_chk) ^ fp8_k_swizzle(k8_tok)) << 4), r[0], r[1], r[2], r[3]);
+            e4m3x4_to_f16x2x2(r[0], a[0], a[2]);
+            e4m3x4_to_f16x2x2(r[1], a[1], a[3]);
+            e4m3x4_to_f16x2x2(r[2], b[0], b[2]);
+            e4m3x4_to_f16x2x2(r[3], b[1], b[3]);
             mma_f16(st, a, qb[2 * j][0], qb[2 * j][1]);
             mma_f16(st2, b, qb[2 * j + 1][0], qb[2 * j + 1][1]);
           }
-          // the shared exponents of the page's rows sit behind its K and V rows
+          // the shared exponents of the page's rows sit behind its K and V elements
           const unsigned char* xs = stages + (size_t)s * kStageBytes + wig * kBlkBytes + 2 * kPage * kRowBytes;
-          const float ks0 = exp_byte_to_float(xs[frow]) * p.scale_log2e;
-          const float ks1 = exp_byte_to_float(xs[frow + 8]) * p.scale_log2e;
-          vscale0 = exp_byte_to_float(xs[kPage + frow]);
-          vscale1 = exp_byte_to_float(xs[kPage + frow + 8]);
+          const float ks0 = exp_byte_to_float(xs[key0]) * p.scale_log2e;
+          const float ks1 = exp_byte_to_float(xs[key0 + 2]) * p.scale_log2e;
+          vscale0 = exp_byte_to_float(xs[kPage + key0]);
+          vscale1 = exp_byte_to_float(xs[kPage + key0 + 2]);
           st[0] = (st[0] + st2[0]) * ks0; st[1] = (st[1] + st2[1]) * ks0;
           st[2] = (st[2] + st2[2]) * ks1; st[3] = (st[3] + st2[3]) * ks1;
         }
-        if (tok_base + kPage > x.t1) {  // ragged end of the split: keys are rows frow, frow + 8
+        if (tok_base + kPage > x.t1) {  // ragged end of the split: this thread's two keys (tile rows frow, frow + 8)
           const int lim = x.t1 - tok_base;
-          if (frow >= lim) st[0] = st[1] = -INFINITY;
-          if (frow + 8 >= lim) st[2] = st[3] = -INFINITY;
+          if ((KV8 ? key0 : frow) >= lim) st[0] = st[1] = -INFINITY;
+          if ((KV8 ? key0 + 2 : frow + 8) >= lim) st[2] = st[3] = -INFINITY;
         }
         // column (head) max over the 16 keys: two rows here, eight row groups across lanes
         float mx0 = fmaxf(st[0], st[2]), mx1 = fmaxf(st[1], st[3]);
@@ -450,11 +479,18 @@ decode_split_bf16_kernel(const __grid_constant__ DecodeParams p, const int n_sta
           mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, sh));
         }
         const float mn0 = fmaxf(m[0], mx0), mn1 = fmaxf(m[1], mx1);
-        const float a0 = exp2f(m[0] - mn0), a1 = exp2f(m[1] - mn1);
+        float a0, a1;
+        if constexpr (!KV8) {
+          a0 = exp2f(m[0] - mn0); a1 = exp2f(m[1] - mn1);
+          st[0] = exp2f(st[0] - mn0); st[1] = exp2f(st[1] - mn1);
+          st[2] = exp2f(st[2] - mn0); st[3] = exp2f(st[3] - mn1);
+        } else {   // (arguments are <= 0: a single MUFU op each, tiny results flushed to zero)
+          a0 = ex2_ftz(m[0] - mn0); a1 = ex2_ftz(m[1] - mn1);
+          st[0] = ex2_ftz(st[0] - mn0); st[1] = ex2_ftz(st[1] - mn1);
+          st[2] = ex2_ftz(st[2] - mn0); st[3] = ex2_ftz(st[3] - mn1);
+        }
         m[0] = mn0;
         m[1] = mn1;
-        st[0] = exp2f(st[0] - mn0); st[1] = exp2f(st[1] - mn1);
-        st[2] = exp2f(st[2] - mn0); st[3] = exp2f(st[3] - mn1);
         l[0] = l[0] * a0 + (st[0] + st[2]);
         l[1] = l[1] * a1 + (st[1] + st[3]);
         // P^T as two bf16 terms (value + rounding residual): the stream leaves tensor
@@ -481,27 +517,29 @@ decode_split_bf16_kernel(const __grid_constant__ DecodeParams p, const int n_sta
         } else {
           // P^T as one fp16 term (11 significant bits against the 4 of the stored V), each
           // weight already multiplied by its V row's 2^X
-          const uint32_t ph0 = movmatrix_t(pack_f16(st[0] * vscale0, st[1] * vscale0));   // keys 0-7
-          const uint32_t ph1 = movmatrix_t(pack_f16(st[2] * vscale1, st[3] * vscale1));   // keys 8-15
+          const uint32_t ph0 = movmatrix_t(pack_f16(st[0] * vscale0, st[1] * vscale0));   // tile rows 0-7
+          const uint32_t ph1 = movmatrix_t(pack_f16(st[2] * vscale1, st[3] * vscale1));   // tile rows 8-15
+          // once the running maxima have settled, most pages leave them alone (a0 = a1 = 1)
+          if (__any_sync(0xffffffffu, a0 != 1.f || a1 != 1.f)) {
 #pragma unroll
-          for (int jt = 0; jt < D / 16; ++jt) {
-            o[jt][0] *= a0; o[jt][1] *= a1;
-            o[jt][2] *= a0; o[jt][3] *= a1;
+            for (int jt = 0; jt < D / 16; ++jt) {
+              o[jt][0] *= a0; o[jt][1] *= a1;
+              o[jt][2] *= a0; o[jt][3] *= a1;
+            }
           }
-          // A transposed 8x8 tile of byte pairs gives this thread keys 2t, 2t+1 of the channel
-          // pair 2 frow, 2 frow + 1: the even channel becomes accumulator row frow, the odd one
-          // row frow + 8 (see the merge below)
+          // V^T rows are channels, 16 key bytes each: one ldmatrix.x4 = 32 channels; a register
+          // holds keys 4t .. 4t+3 of a channel, which are the contraction indices 2t, 2t+1 and
+          // 2t+8, 2t+9 in the key order of the tile rows above
 #pragma unroll
           for (int j = 0; j < D / 32; ++j) {
-            uint32_t r[4];
-            ldsm_x4_t(vb + k_tok * kRowBytes + (((2 * j + k_chk) ^ (k_tok & 7)) << 4), r[0], r[1], r[2], r[3]);
-#pragma unroll
-            for (int c = 0; c < 2; ++c) {
-              const uint32_t lo = __byte_perm(r[2 * c], 0u, 0x3120), hi = __byte_perm(r[2 * c + 1], 0u, 0x3120);
-              const uint32_t a[4] = {e4m3x2_to_f16x2(lo), e4m3x2_to_f16x2(lo >> 16),
-                                     e4m3x2_to_f16x2(hi), e4m3x2_to_f16x2(hi >> 16)};
-              mma_f16(o[2 * j + c], a, ph0, ph1);
-            }
+            uint32_t r[4], a[4], b[4];
+            ldsm_x4(vb + (32 * j + lane) * kPage, r[0], r[1], r[2], r[3]);
+            e4m3x4_to_f16x2x2(r[0], a[0], a[2]);
+            e4m3x4_to_f16x2x2(r[1], a[1], a[3]);
+            e4m3x4_to_f16x2x2(r[2], b[0], b[2]);
+            e4m3x4_to_f16x2x2(r[3], b[1], b[3]);
+            mma_f16(o[2 * j], a, ph0, ph1);
+            mma_f16(o[2 * j + 1], b, ph0, ph1);
           }
         }
       }
@@ -524,13 +562,8 @@ decode_split_bf16_kernel(const __grid_constant__ DecodeParams p, const int n_sta
       if (r < rows) {
 #pragma unroll
         for (int jt = 0; jt < D / 16; ++jt) {
-          if constexpr (!KV8) {
-            mo[r * D + jt * 16 + frow] = o[jt][e];
-            mo[r * D + jt * 16 + frow + 8] = o[jt][2 + e];
-          } else {   // accumulator rows frow / frow + 8 are channels 2 frow / 2 frow + 1 of the block
-            mo[r * D + jt * 16 + 2 * frow] = o[jt][e];
-            mo[r * D + jt * 16 + 2 * frow + 1] = o[jt][2 + e];
-          }
+          mo[r * D + jt * 16 + frow] = o[jt][e];
+          mo[r * D + jt * 16 + frow + 8] = o[jt][2 + e];
         }
         if (frow == 0) { mml[r * 2] = m[e]; mml[r * 2 + 1] = l[e]; }
       }
@@ -639,16 +672,20 @@ cudaError_t launch_decode_split_bf16(const DecodeParams& p, int sm_count, cudaSt
   // At most one item per two SMs, and items of several stages: a cluster of two CTAs per item.
   const bool paired = 2 * p.total_items <= sm_count && max_keys >= 4 * kTileKeys;
   const int cl = paired ? 2 : 1;
+  const int kv8 = p.geom.fp8;
   const int ncw = small ? 4 : 8;
   const size_t budget = small ? 110 * 1024 : 220 * 1024;
-  const int kv8 = p.geom.fp8;
   if (kv8 && D != 128) return cudaErrorInvalidValue;
-  int n_stages = kMaxStages;
+  int n_stages = kv8 ? kMaxStages : 8;
   while (n_stages > 2 && smem_bytes(D, p.group, n_stages, ncw, cl, kv8) > budget) --n_stages;
-  // Two consumer groups take alternate tiles: with an even ring every stage always belongs to the
-  // same group, which then waits for its phases one after the other (a parity wait is only valid
-  // for the phase right after the last one known complete).
-  if (ncw == 8 && (n_stages & 1)) --n_stages;
+  // The consumer groups take tiles in turn: with a ring that is a multiple of the number of groups
+  // every stage always belongs to the same group, which then waits for its phases one after the
+  // other (a parity wait is only valid for the phase right after the last one known complete).
+  // With several producer warps a stage must also always belong to the same producer.
+  const int groups = ncw / kGroupWarps, producers = producer_warps(ncw, kv8);
+  const int unit = groups > producers ? groups : producers;   // (1, 2 or 4: the larger is a multiple of the smaller)
+  n_stages -= n_stages % unit;
+  if (n_stages < unit) return cudaErrorInvalidConfiguration;
   const size_t smem = smem_bytes(D, p.group, n_stages, ncw, cl, kv8);
   const int slots = small ? 2 * sm_count : sm_count;
   const int grid = paired ? 2 * p.total_items : (p.total_items < slots ? p.total_items : slots);
@@ -657,7 +694,7 @@ cudaError_t launch_decode_split_bf16(const DecodeParams& p, int sm_count, cudaSt
   // first global access
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(grid);
-  cfg.blockDim = dim3((ncw + 1) * 32);
+  cfg.blockDim = dim3((ncw + producer_warps(ncw, kv8)) * 32);
   cfg.dynamicSmemBytes = smem;
   cfg.stream = st;
   cudaLaunchAttribute attr[2];

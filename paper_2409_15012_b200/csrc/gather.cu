@@ -89,9 +89,16 @@ __global__ void __launch_bounds__(kThreads) gather_fp8_kernel(const __grid_const
         page = p.table[(int64_t)e.seq * p.table_stride + pos / kPage];
         slot = pos % kPage;
       }
-      // 8 codes = half of a stored 16-byte chunk
-      const uint2 codes = *reinterpret_cast<const uint2*>(p.pool + kv_chunk_offset(ge, page, g, which, slot, chunk >> 1) +
-                                                          (chunk & 1) * 8);
+      uint2 codes;
+      if (which == 0) {   // 8 codes = half of a stored 16-byte chunk
+        codes = *reinterpret_cast<const uint2*>(p.pool + kv_chunk_offset(ge, page, g, 0, slot, chunk >> 1) + (chunk & 1) * 8);
+      } else {            // V is stored transposed: one byte per channel row
+        const unsigned char* src = reinterpret_cast<const unsigned char*>(p.pool) + kv_fp8_v_offset(ge, page, g, chunk * 8, slot);
+        uint32_t w[2] = {0u, 0u};
+#pragma unroll
+        for (int i = 0; i < 8; ++i) w[i >> 2] |= (uint32_t)src[i * kPage] << (8 * (i & 3));
+        codes = make_uint2(w[0], w[1]);
+      }
       const int X = (int)*reinterpret_cast<const unsigned char*>(p.pool + kv_exp_offset(ge, page, g, which, slot)) - 127;
       const float scale = X > -127 ? __int_as_float((X + 127) << 23) : __int_as_float(0x00400000);   // 2^X (2^-127 is subnormal)
       const uint32_t cw[2] = {codes.x, codes.y};

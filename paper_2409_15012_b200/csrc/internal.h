@@ -24,9 +24,11 @@ constexpr int kWsChunks = kMaxCallSeqs + kWsExtraChunks + kWsWaveChunks;  // spl
 // chunks of a token row are stored XOR-swizzled by (token & 7): the block in HBM is
 // already the bank-conflict-free shared-memory image that ldmatrix wants, and the
 // copy engine needs no tensor map.  fp32 rows are stored unswizzled.
-// Quantised storage (FP8 E4M3 elements, one shared exponent byte per stored row): the rows
-// are D bytes, swizzled the same way, and the block ends with the 16 exponent bytes of its K
-// rows and the 16 of its V rows:  [K: 16 x D B][V: 16 x D B][X_K: 16 B][X_V: 16 B].
+// Quantised storage (FP8 E4M3 elements, one shared exponent byte per head vector):
+//   [K: 16 tokens x D bytes][V^T: D channels x 16 tokens][X_K: 16 B][X_V: 16 B].
+// K rows are swizzled by fp8_k_swizzle(token); V is stored TRANSPOSED (one 16-byte row per
+// channel) because both tensor-core products of the decode kernel want their 8-bit operand
+// with the contraction index contiguous: channels for K, tokens for V.
 // ---------------------------------------------------------------------------
 struct KvGeom {
   int32_t n_kv_heads;
@@ -54,13 +56,24 @@ __host__ __device__ inline KvGeom make_geom(int n_kv_heads, int head_dim, int dt
   return g;
 }
 
+// Chunk permutation of a quantised K row.  The decode kernel reads the 16 tokens of a page in the
+// order 0 1 4 5 8 9 12 13 | 2 3 6 7 10 11 14 15 (see decode_bf16.cu): each half must hit eight
+// different 16-byte columns.
+__host__ __device__ inline int fp8_k_swizzle(int tok) { return (tok & 1) | ((tok >> 2) << 1); }
+
 // Byte offset, inside a pool, of 16-byte chunk `chunk` of the stored row of token slot `tok`
-// (0..15) of page `page`, KV head `g`, which = 0 (K) or 1 (V).
+// (0..15) of page `page`, KV head `g`, which = 0 (K) or 1 (V; native storage only).
 __host__ __device__ inline int64_t kv_chunk_offset(const KvGeom& ge, int64_t page, int g, int which,
                                                    int tok, int chunk) {
-  int c = ge.swizzle ? (chunk ^ (tok & 7)) : chunk;
+  int c = !ge.swizzle ? chunk : ge.fp8 ? (chunk ^ fp8_k_swizzle(tok)) : (chunk ^ (tok & 7));
   return page * ge.page_bytes + (int64_t)g * ge.blk_bytes + (int64_t)which * kPage * ge.st_row_bytes +
          (int64_t)tok * ge.st_row_bytes + (int64_t)c * 16;
+}
+
+// Quantised storage: byte offset of V element (channel, tok) of that page and head.
+__host__ __device__ inline int64_t kv_fp8_v_offset(const KvGeom& ge, int64_t page, int g, int channel, int tok) {
+  return page * ge.page_bytes + (int64_t)g * ge.blk_bytes + (int64_t)kPage * ge.st_row_bytes +
+         (int64_t)channel * kPage + tok;
 }
 
 // Quantised storage: byte offset of the shared-exponent byte of that row.

@@ -80,7 +80,7 @@ def test_fp8_decode_steps_state_bits_and_outputs(hq, hkv, lengths, split):
                 lo = 0 if kind == cf.FULL else max(0, n - W)
                 for pos in sorted({lo, n - 1, (lo + n) // 2}):
                     check_stored(sess.ctx, wl, l, b, pos)
-        print(f"\\nfp8 cache: the quantisation itself moves the outputs by up to {worst_q:.3e} (checker, informative)")
+        print(f"\nfp8 cache: the quantisation itself moves the outputs by up to {worst_q:.3e} (checker, informative)")
     finally:
         sess.close()
 
