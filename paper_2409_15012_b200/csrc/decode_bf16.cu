@@ -306,6 +306,10 @@ decode_split_bf16_kernel(const __grid_constant__ DecodeParams p, const int n_sta
     // K % kProducerWarps == pw
     const int pw = warp - kConsumerWarps;
     int K = 0;  // tiles of this CTA so far (all producers)
+    // stage of this producer's next tile and how often it has been round the ring (kept by
+    // addition: the ring length is a run-time value, and a division per stage sits on the
+    // issue path)
+    int ps = pw, pround = 0;
     bool ok = true;
     const uint64_t l2_policy = l2_policy_of(p.pool, p.l2_keep_bytes, p.l2_pool_bytes);
     for (int it = item0; ok && it < p.total_items; it += item_stride) {
@@ -328,12 +332,14 @@ decode_split_bf16_kernel(const __grid_constant__ DecodeParams p, const int n_sta
           if (tbl && pg + 32 + lane < page_hi) ids_next = tbl[pg + 32 + lane];
         }
         if (kProducerWarps > 1 && K % kProducerWarps != pw) continue;
-        const int s = K % n_stages;
-        if (K >= n_stages) {  // lane 0 waits; the verdict is made warp-uniform
+        const int s = ps;
+        if (pround > 0) {  // lane 0 waits; the verdict is made warp-uniform
           int w = 1;
-          if (lane == 0) w = mbar_wait(empty0 + 8 * s, ((K / n_stages) - 1) & 1, abort_flag);
+          if (lane == 0) w = mbar_wait(empty0 + 8 * s, (pround - 1) & 1, abort_flag);
           if (!__shfl_sync(0xffffffffu, w, 0)) { ok = false; break; }
         }
+        ps += kProducerWarps;
+        if (ps >= n_stages) { ps -= n_stages; ++pround; }
         const int n_pg = min(kGroupWarps, page_hi - pg);
         if (lane == 0) mbar_arrive_expect_tx(full0 + 8 * s, n_pg * kBlkBytes);
         const int my_id = __shfl_sync(0xffffffffu, ids, (rel & 31) + (lane & (kGroupWarps - 1)));
@@ -382,6 +388,7 @@ decode_split_bf16_kernel(const __grid_constant__ DecodeParams p, const int n_sta
   const int key0 = 4 * (frow >> 1) + (frow & 1);                // this thread's score rows: keys key0 and key0 + 2
 
   int K = 0;
+  int cs = grp, cround = 0;   // stage of this group's next tile, passes over the ring (see the producers)
   for (int it = item0; it < p.total_items; it += item_stride) {
     Item x = decode_item(p, it);
     if constexpr (CL > 1) cluster_share(x, crank);
@@ -421,12 +428,13 @@ decode_split_bf16_kernel(const __grid_constant__ DecodeParams p, const int n_sta
     for (int j = 0; j < D / 16; ++j) o[j][0] = o[j][1] = o[j][2] = o[j][3] = 0.f;
 
     const int n_tiles = ((x.t1 + kPage - 1) / kPage - x.t0 / kPage + kGroupWarps - 1) / kGroupWarps;
-    for (int k = 0; k < n_tiles; ++k) {
-      const int Kg = K + k;
-      if ((Kg % kGroups) != grp) continue;
-      const int s = Kg % n_stages;
+    // this group's tiles of the item: every kGroups-th, starting where the count left off
+    for (int k = (grp + kGroups - K % kGroups) % kGroups; k < n_tiles; k += kGroups) {
+      const int s = cs;
       // every lane waits (each needs to observe the copy), the verdict is warp-uniform
-      if (!__all_sync(0xffffffffu, mbar_wait(full0 + 8 * s, (Kg / n_stages) & 1, abort_flag))) break;
+      if (!__all_sync(0xffffffffu, mbar_wait(full0 + 8 * s, cround & 1, abort_flag))) break;
+      cs += kGroups;
+      if (cs >= n_stages) { cs -= n_stages; ++cround; }
       const int tok_base = x.t0 + k * kTileKeys + wig * kPage;
       if (tok_base < x.t1) {
         const uint32_t kb = smem_u32(stages + (size_t)s * kStageBytes + wig * kBlkBytes);
