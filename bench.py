@@ -692,9 +692,15 @@ def run_trace_arm(args):
                "mid-decode layout (1 full cache + 2 shared rings)": cf.layout_mid(1024)}
     for name in ("MA", "MA-EndSlide", "MA-Offset", "MA-Pairs", "MA-Offset-SlideShare", "MA-Pairs-SlideShare"):
         layouts[name] = cf.PAPER_VARIANTS[name]()     # the paper's named variants (layer indices: see synth/configs.py)
+    if args.trace_layouts:
+        keep = [s.strip() for s in args.trace_layouts.split(",")]
+        layouts = {k: v for k, v in layouts.items() if k in keep or k == "standard"}
+    from paper_2409_15012_b200 import binding as mx
+    kvf = mx.KV_FP8_E4M3 if args.kv_format == "fp8" else mx.KV_NATIVE
     res = {}
     for name, lay in layouts.items():
-        res[name] = runner.serve_trace(lay, 12, 3, 128, args.trace_requests, args.trace_prompt, args.trace_gen, 2048)
+        res[name] = runner.serve_trace(lay, 12, 3, 128, args.trace_requests, args.trace_prompt, args.trace_gen, 2048,
+                                       concurrency=args.trace_concurrency, kv_format=kvf)
         res[name]["speedup_over_standard"] = res[name]["tokens_per_s"] / res["standard"]["tokens_per_s"]
         res[name]["cache_bytes_vs_standard"] = res[name]["cache_bytes"] / res["standard"]["cache_bytes"]
     ma = res["MA-Offset"]
@@ -702,6 +708,7 @@ def run_trace_arm(args):
             "unit": "tokens/s", "n_gpus": 1, "higher_is_better": True, "dtype": "bf16", "data": "synthetic",
             "vs_baseline": None,
             "config": {"workload": "serving_trace", "layout": "MA-Offset", "requests": args.trace_requests,
+                       "concurrency": args.trace_concurrency or args.trace_requests, "kv_format": args.kv_format,
                        "prompt_len": args.trace_prompt, "gen_len": args.trace_gen, "chunk": 2048, "heads": "12/3x128",
                        "layers": 24, "window": 1024,
                        "timing": "sum of the library's kernel times (CUDA events around every launch)"},
@@ -757,6 +764,10 @@ def main():
     ap.add_argument("--trace-requests", type=int, default=8)
     ap.add_argument("--trace-prompt", type=int, default=31000)
     ap.add_argument("--trace-gen", type=int, default=100)
+    ap.add_argument("--trace-concurrency", type=int, default=0,
+                    help="requests served at a time (0 = all at once); every layout gets the same number, so the "
+                         "standard layout's cache has to fit")
+    ap.add_argument("--trace-layouts", default="", help="comma-separated subset of the layouts (standard always runs)")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3

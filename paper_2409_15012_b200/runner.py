@@ -212,37 +212,80 @@ def kv_bytes_per_step(wl: cf.Workload, lengths_after: Sequence[int], kv_format: 
 
 
 def serve_trace(layout, n_q_heads: int, n_kv_heads: int, head_dim: int, n_requests: int, prompt_len: int,
-                gen_len: int, chunk: int, device: int = 0, seed: int = 7, dtype: int = cf.BF16) -> Dict:
-    """Attention-only serving of `n_requests` concurrent requests shaped like the paper's
-    benchmark (Section 5.4: long prompts, then generated tokens): the prompts in chunks
-    through attend_chunk + append_kv, then `gen_len` decode steps.  Times are the sums of the
-    library's own kernel times (its profile hooks), so input generation is excluded."""
-    wl = cf.Workload("serving_trace", list(layout), n_q_heads, n_kv_heads, head_dim, dtype, n_requests, 0, seed)
-    sess = Session(wl, [prompt_len] * n_requests, device=device, headroom_tokens=gen_len + 1,
-                   chunk_scratch_tokens=n_requests * (prompt_len + chunk))
+                gen_len: int, chunk: int, device: int = 0, seed: int = 7, dtype: int = cf.BF16,
+                concurrency: int = 0, kv_format: int = mx.KV_NATIVE) -> Dict:
+    """Attention-only serving of `n_requests` requests shaped like the paper's benchmark
+    (Section 5.4: long prompts, then generated tokens), `concurrency` of them at a time (0 = all
+    at once): per wave the prompts in chunks through attend_chunk + append_kv, then `gen_len`
+    decode steps, then the sequence slots are reset for the next wave.  `kernel` times are the
+    sums of the library's own kernel times (its profile hooks), so input generation is excluded;
+    the wall-clock figure beside them includes generating the synthetic inputs on the GPU and
+    issuing every call from Python."""
+    import time
+    conc = n_requests if concurrency <= 0 else min(concurrency, n_requests)
+    wl = cf.Workload("serving_trace", list(layout), n_q_heads, n_kv_heads, head_dim, dtype, conc, 0, seed)
+    sess = Session(wl, [prompt_len] * conc, device=device, headroom_tokens=gen_len + 1,
+                   chunk_scratch_tokens=conc * (prompt_len + chunk), kv_format=kv_format)
     try:
         classes = (mx.K_APPEND, mx.K_DECODE_FULL, mx.K_DECODE_SLIDING, mx.K_COMBINE, mx.K_PREFILL_FULL,
                    mx.K_PREFILL_SLIDING, mx.K_GATHER)
-        sess.ctx.profile_enable(True)
         # prefill_in_chunks hands every reader its owner's K/V tensors, unchanged within a round:
         # the cached keys of a shared cache are copied once per run of layers that read it
         sess.ctx.set_chunk_gather_reuse(True)
-        sess.prefill_in_chunks(chunk)
+        prefill_ms = decode_ms = 0.0
+        done, waves = 0, 0
         torch.cuda.synchronize(sess.dev)
-        prefill_ms = sum(sess.ctx.profile_read(c)[1] for c in classes)
-        outs = sess.alloc_outputs()
-        for _ in range(gen_len):
-            sess.decode_step(sess.step_inputs(), outs)
-        torch.cuda.synchronize(sess.dev)
-        decode_ms = sum(sess.ctx.profile_read(c)[1] for c in classes) - prefill_ms   # the records accumulate
-        sess.ctx.profile_enable(False)
+        t0 = time.perf_counter()
+        while done < n_requests:
+            n_wave = min(conc, n_requests - done)
+            if waves > 0:
+                for b in range(conc):
+                    sess.ctx.seq_reset(b)
+                sess.pos[:] = 0
+            # (a last, smaller wave leaves the other slots empty: their targets are 0)
+            sess.target[:] = 0
+            sess.target[:n_wave] = prompt_len
+            sess.ctx.profile_enable(True)
+            sess.prefill_in_chunks(chunk)
+            torch.cuda.synchronize(sess.dev)
+            prefill_ms += sum(sess.ctx.profile_read(c)[1] for c in classes)
+            sess.ctx.profile_enable(True)        # drops the records read so far
+            if n_wave == conc:
+                outs = sess.alloc_outputs()
+                for _ in range(gen_len):
+                    sess.decode_step(sess.step_inputs(), outs)
+            else:
+                decode_partial(sess, n_wave, gen_len)
+            torch.cuda.synchronize(sess.dev)
+            decode_ms += sum(sess.ctx.profile_read(c)[1] for c in classes)
+            sess.ctx.profile_enable(False)
+            done += n_wave
+            waves += 1
+        wall_s = time.perf_counter() - t0
         status = sess.ctx.get_device_status()
         cache = mx.cache_bytes(sess.ctx.cfg)
     finally:
         sess.close()
     tokens = n_requests * (prompt_len + gen_len)
-    return {"requests": n_requests, "prompt_len": prompt_len, "gen_len": gen_len, "chunk": chunk,
-            "prefill_kernel_ms": prefill_ms, "decode_kernel_ms": decode_ms,
+    return {"requests": n_requests, "concurrency": conc, "waves": waves, "prompt_len": prompt_len, "gen_len": gen_len,
+            "chunk": chunk, "prefill_kernel_ms": prefill_ms, "decode_kernel_ms": decode_ms,
             "tokens_per_s": tokens / ((prefill_ms + decode_ms) * 1e-3),
             "decode_tokens_per_s": n_requests * gen_len / (decode_ms * 1e-3) if decode_ms > 0 else None,
-            "cache_bytes": cache, "device_status": status}
+            "wall_s": wall_s, "wall_tokens_per_s": tokens / wall_s,
+            "cache_bytes": cache, "cache_bytes_per_request": cache / conc, "device_status": status}
+
+
+def decode_partial(sess: Session, n_active: int, steps: int):
+    """Decode steps for the first n_active sequence slots only (a last wave that does not fill
+    the context)."""
+    wl = sess.wl
+    ids = list(range(n_active))
+    outs = sess.alloc_outputs()
+    for _ in range(steps):
+        inputs = sess.step_inputs()
+        for l in range(len(wl.layout)):
+            ent = inputs[l]
+            if "k" in ent:
+                sess._append(l, ids, None, ent["k"][:n_active], ent["v"][:n_active])
+            sess.ctx.decode(l, ids, ent["q"][:n_active], outs[l][:n_active])
+        sess.pos[:n_active] += 1

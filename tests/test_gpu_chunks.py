@@ -163,6 +163,10 @@ def test_serving_trace_small():
                 check_close(g[l, b], ref_decode(wl, l, b, prompts[b] + 5), wl.dtype, f"decode {l}/{b}")
         res = runner.serve_trace(wl.layout, 12, 3, 128, 2, 300, 3, 128)
         assert res["device_status"] == 0 and res["prefill_kernel_ms"] > 0 and res["decode_kernel_ms"] > 0
+        # the same requests two at a time, the last wave only half full: same token count, three waves
+        res = runner.serve_trace(wl.layout, 12, 3, 128, 5, 300, 3, 128, concurrency=2)
+        assert res["device_status"] == 0 and res["waves"] == 3 and res["wall_tokens_per_s"] > 0
+        assert res["tokens_per_s"] >= res["wall_tokens_per_s"]
     finally:
         sess.close()
 

@@ -108,6 +108,46 @@ def test_mixed_serving_full_size():
                     layers=[0, 1, 12, 13, 23], seqs=[short, longest], heads=[2, 17], free_order=perm)
 
 
+def test_mid_decode_full_size_quantised_cache():
+    # the mid-decode configuration on a quantised cache (FP8 E4M3 elements), at the size and in the
+    # launch configuration bench.py times: stored codes and exponents bit for bit at sampled
+    # positions, outputs against the checker's attention over the dequantised history
+    mx, runner = load_lib()
+    wl = cf.mid_decode()
+    sess = runner.Session(wl, [wl.context] * wl.batch, headroom_tokens=2, kv_format=mx.KV_FP8_E4M3)
+    ph = mo.PhysicalCache(wl.layout, wl.n_kv_heads, wl.head_dim, wl.batch, sess.n_pages, store_values=False)
+    sess.mirror = ph
+    G = wl.n_q_heads // wl.n_kv_heads
+    dt = torch_dt(wl.dtype)
+    try:
+        sess.fill(1024)
+        outs = sess.alloc_outputs()
+        sess.decode_step(sess.step_inputs(), outs)
+        torch.cuda.synchronize()
+        assert sess.ctx.get_device_status() == 0
+        compare_state(sess.ctx, ph, wl)
+        n = wl.context + 1
+        for l, b, h in ((0, 0, 3), (12, 31, 17), (1, 5, 30), (23, 17, 8)):
+            kind, W, owner = wl.layout[l]
+            lo = 0 if kind == cf.FULL else n - W
+            K, V = si.kv_tokens_head(wl.seed, owner, b, lo, n - lo, wl.n_kv_heads, wl.head_dim, h // G, dt)
+            # quantise each head vector as the cache does (one KV head at a time: the rule is per head vector)
+            Kq = mo.kv_roundtrip(K.double().numpy()[:, None, :])[:, 0]
+            Vq = mo.kv_roundtrip(V.double().numpy()[:, None, :])[:, 0]
+            q = si.q_tokens(wl.seed, l, b, n - 1, 1, wl.n_q_heads, wl.head_dim, dt)[0, h].double().numpy()
+            ref = mo.softmax_attend(q, Kq, Vq, 1.0 / np.sqrt(wl.head_dim))
+            check_close(outs[l, b, h].float().cpu().double().numpy(), ref, wl.dtype, f"layer {l} seq {b} head {h}")
+        for l, b, pos in ((0, 7, 0), (0, 7, 20001), (12, 30, n - 1), (1, 2, n - 1024), (13, 9, n - 1)):
+            owner = wl.layout[l][2]
+            K, V = si.kv_tokens(wl.seed, owner, b, pos, 1, wl.n_kv_heads, wl.head_dim, dt)
+            kc, kx, vc, vx = sess.ctx.debug_read_kv_fp8(l, b, pos)
+            for got_c, got_x, src in ((kc, kx, K), (vc, vx, V)):
+                codes, X = mo.quantize_kv(src)
+                assert np.array_equal(got_x, X[0]) and np.array_equal(got_c, codes[0]), (l, b, pos)
+    finally:
+        sess.close()
+
+
 def test_prefill_full_size_sampled_rows():
     mx, runner = load_lib()
     wl = cf.prefill_chunk()
