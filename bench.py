@@ -42,11 +42,11 @@ NOMINAL_BF16_TFLOPS = 2250.0     # dense bf16 datasheet figure of a B200 (contex
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 # (dram__bytes_read.sum + dram__bytes_write.sum) / algorithmic KV bytes of the dominant kernel, from an
-# ncu capture of one standard-layer launch at batch 4 (541.30 MB moved for 536.95 MB of keys and values;
+# ncu capture of one standard-layer launch at batch 4 (540.62 MB moved for 536.94 MB of keys and values;
 # the full-size launch holds too much device memory for a multi-pass capture).  DRAM traffic grows in
 # proportion to the keys read, so the full-size figure is this ratio times the launch's algorithmic
 # bytes.  Set to None when the kernel changes until the counters are taken again.
-DECODE_FULL_TRAFFIC_RATIO = 541.304832 / 536.952832
+DECODE_FULL_TRAFFIC_RATIO = 540.617984 / 536.936448
 
 
 def load_peaks():
@@ -380,9 +380,10 @@ def device_pass(sess, runner, wl, ring, outs, stream, K, Wm, barrier, sampler=No
     def bytes_next_step():
         return runner.kv_bytes_per_step(wl, [int(p) + 1 for p in sess.pos], sess.kv_format)
 
+    tables = [sess.step_tables(inp, outs) for inp in ring]    # pointer tables, built once per ring entry
     step = 0
     for _ in range(Wm):
-        sess.decode_step(ring[step % len(ring)], outs, stream)
+        sess.decode_step(ring[step % len(ring)], outs, stream, tables=tables[step % len(ring)])
         step += 1
     launches0 = sess.ctx.get_launch_count()
     barrier()
@@ -397,7 +398,7 @@ def device_pass(sess, runner, wl, ring, outs, stream, K, Wm, barrier, sampler=No
         e0.record(stream)
         for _ in range(K):
             b += bytes_next_step()
-            sess.decode_step(ring[step % len(ring)], outs, stream)
+            sess.decode_step(ring[step % len(ring)], outs, stream, tables=tables[step % len(ring)])
             step += 1
         e1.record(stream)
         events.append((e0, e1))
@@ -529,6 +530,10 @@ def run_gpu_arm(args, wl):
     d2h_cuts = sorted({n_layers // 2, (5 * n_layers) // 6, n_layers - 1} - {0, n_layers})   # outputs leave in pieces
     ev_out = [torch.cuda.Event() for _ in d2h_cuts]
     ids_all = list(range(wl.batch))
+    # the step is issued in a few mixattn_decode_layers calls, cut where a copy has to be awaited
+    # (second piece of the inputs) or started (a piece of the outputs)
+    dev_tables = sess.step_tables(dev_buf, outs)
+    bounds = sorted({0, cut_layer, n_layers} | set(d2h_cuts))
 
     def e2e_step(s):
         src = host_flat[s % kRing]
@@ -537,20 +542,17 @@ def run_gpu_arm(args, wl):
             ev_in[0].record(h2d_stream)
             dev_flat[cut:].copy_(src[cut:], non_blocking=True)
             ev_in[1].record(h2d_stream)
-        for l in range(n_layers):
-            if l == 0 or l == cut_layer:
-                stream.wait_event(ev_in[0 if l == 0 else 1])
-            ent = dev_buf[l]
-            if "k" in ent:
-                sess.ctx.append_kv(l, ids_all, None, ent["k"], ent["v"], stream)
-            sess.ctx.decode(l, ids_all, ent["q"], outs[l], stream)
-            if l + 1 in d2h_cuts:
-                i = d2h_cuts.index(l + 1)
+        for lo_l, hi_l in zip(bounds[:-1], bounds[1:]):
+            if lo_l == 0 or lo_l == cut_layer:
+                stream.wait_event(ev_in[0 if lo_l == 0 else 1])
+            sess.ctx.decode_layers(lo_l, hi_l, ids_all, *dev_tables, stream)
+            if hi_l in d2h_cuts:
+                i = d2h_cuts.index(hi_l)
                 lo = d2h_cuts[i - 1] if i > 0 else 0
                 ev_out[i].record(stream)
                 d2h_stream.wait_event(ev_out[i])
                 with torch.cuda.stream(d2h_stream):
-                    host_out[lo:l + 1].copy_(outs[lo:l + 1], non_blocking=True)
+                    host_out[lo:hi_l].copy_(outs[lo:hi_l], non_blocking=True)
         sess.pos += 1
         with torch.cuda.stream(stream):
             host_out[d2h_cuts[-1]:].copy_(outs[d2h_cuts[-1]:], non_blocking=True)
@@ -589,9 +591,10 @@ def run_gpu_arm(args, wl):
     sess.ctx.profile_enable(True)
     full_bytes = 0
     Kp = min(K, 20)
+    prof_tables = [sess.step_tables(inp, outs) for inp in step_inputs]
     for s in range(Kp):
         full_bytes += sum(int(p) + 1 for p in sess.pos) * per_tok
-        sess.decode_step(step_inputs[s % kRing], outs, stream)
+        sess.decode_step(step_inputs[s % kRing], outs, stream, tables=prof_tables[s % kRing])
     n_full, ms_full = sess.ctx.profile_read(mx.K_DECODE_FULL)
     n_slide, ms_slide = sess.ctx.profile_read(mx.K_DECODE_SLIDING)
     n_comb, ms_comb = sess.ctx.profile_read(mx.K_COMBINE)

@@ -51,7 +51,7 @@ enum {
   MIXATTN_ERR_OUT_OF_PAGES = -4,   /* the paged pool has too few free pages for the call            */
   MIXATTN_ERR_EMPTY_CONTEXT = -5,  /* decode on a sequence whose cache holds no token               */
   MIXATTN_ERR_BAD_SEQ = -6,        /* sequence id outside 0 .. max_seqs-1                           */
-  MIXATTN_ERR_UNSUPPORTED = -7,    /* valid request this build does not implement                   */
+  MIXATTN_ERR_UNSUPPORTED = -7,    /* valid request this library does not implement                 */
   MIXATTN_ERR_CUDA = -8,           /* a CUDA call failed, or the context is host-only               */
   MIXATTN_ERR_TOO_LARGE = -9       /* mixattn_decode_static_scratch: request exceeds the static array */
 };
@@ -185,6 +185,23 @@ int mixattn_append_kv_rope(mixattn_ctx* ctx, int32_t layer, int32_t n_seqs, cons
  * (nothing is written), BAD_SEQ, INVALID_ARG, CUDA. */
 int mixattn_decode(mixattn_ctx* ctx, int32_t layer, int32_t n_seqs, const int32_t* seq_ids,
                    const void* q, void* out, void* stream);
+
+/* One decode step over the layers layer_begin .. layer_end - 1, in order (Section 3, layer by
+ * layer as a forward pass visits them; the generation loop of Section 5.4's workload): for each
+ * layer, mixattn_append_kv of one new token per sequence if the layer owns its cache, then
+ * mixattn_decode.  One call instead of one or two per layer: at small batches issuing the calls
+ * is what a step costs.
+ *   q, out   host arrays indexed by layer (n_layers entries; only the range is read) of device
+ *            pointers, [n_seqs, n_q_heads, head_dim] each
+ *   k, v     the same for the new token's K/V, [n_seqs, n_kv_heads, head_dim]; entries of
+ *            layers that reuse a cache are ignored and may be NULL
+ * The effect is that of the individual calls made one after the other, and the call stops at
+ * the first of them that fails, returning its status: layers before it stand (their caches
+ * have moved).  *layers_done, if not NULL, receives the number of layers completed.
+ * Errors: INVALID_ARG for a bad range or null arrays, else those of the two calls. */
+int mixattn_decode_layers(mixattn_ctx* ctx, int32_t layer_begin, int32_t layer_end, int32_t n_seqs,
+                          const int32_t* seq_ids, const void* const* q, const void* const* k,
+                          const void* const* v, void* const* out, void* stream, int32_t* layers_done);
 
 /* Prompt attention of `layer` for n_seqs sequences that start at position 0
  * (Section 3; causal as in Section 1).  Query i attends to keys j <= i

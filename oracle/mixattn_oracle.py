@@ -24,7 +24,7 @@ and of ring buffers (slot = position mod s); attention computed from what the
 physical half still stores must equal the logical half.
 
 Quantised KV storage (FP8 E4M3 elements with a shared power-of-two scale per
-head vector) is a reading of this build, not the paper's: see the section on
+head vector) is a reading of this library, not the paper's: see the section on
 it below and its pins in tests/test_oracle_fp8.py.
 
 Pins (tests/test_oracle_pins.py): dense brute-force masked softmax on tiny

@@ -77,6 +77,7 @@ def _load() -> C.CDLL:
         "mixattn_append_kv_rope": [vp, i32, i32, p32, p32, vp, vp, C.c_float, vp],
         "mixattn_decode": [vp, i32, i32, p32, vp, vp, vp],
         "mixattn_decode_static_scratch": [vp, i32, i32, p32, vp, vp, vp],
+        "mixattn_decode_layers": [vp, i32, i32, i32, p32, C.POINTER(vp), C.POINTER(vp), C.POINTER(vp), C.POINTER(vp), vp, p32],
         "mixattn_attend_chunk": [vp, i32, i32, p32, p32, vp, vp, vp, vp, vp],
         "mixattn_prefill": [vp, i32, i32, p32, p32, vp, vp, vp, vp, vp],
         "mixattn_get_len": [vp, i32, i32, p32],
@@ -105,7 +106,7 @@ def _load() -> C.CDLL:
 lib = _load()
 EXPORTS = [
     "mixattn_arena_bytes", "mixattn_cache_bytes", "mixattn_create", "mixattn_destroy",
-    "mixattn_seq_reset", "mixattn_append_kv", "mixattn_append_kv_rope", "mixattn_decode", "mixattn_decode_static_scratch", "mixattn_prefill",
+    "mixattn_seq_reset", "mixattn_append_kv", "mixattn_append_kv_rope", "mixattn_decode", "mixattn_decode_static_scratch", "mixattn_decode_layers", "mixattn_prefill",
     "mixattn_attend_chunk",
     "mixattn_get_len", "mixattn_get_block_table", "mixattn_get_n_free_pages",
     "mixattn_get_ring_state", "mixattn_locate", "mixattn_debug_read_kv", "mixattn_debug_read_kv_fp8",
@@ -250,6 +251,29 @@ class Context:
         s = _i32(seq_ids)
         return lib.mixattn_decode_static_scratch(self.h, layer, len(s), _p32(s), _dev(q), _dev(out),
                                                  _stream(stream))
+
+    def pointer_table(self, tensors):
+        """Host array of device pointers, one per layer (None -> NULL), for mixattn_decode_layers.
+        `tensors` maps a layer index to a tensor, or is a sequence indexed by layer."""
+        n = self.cfg.n_layers
+        arr = (C.c_void_p * n)()
+        for l in range(n):
+            t = tensors.get(l) if isinstance(tensors, dict) else tensors[l]
+            arr[l] = None if t is None else int(t.data_ptr())
+        return arr
+
+    def rc_decode_layers(self, layer_begin, layer_end, seq_ids, q_tab, k_tab, v_tab, out_tab, stream=None):
+        """mixattn_decode_layers with pointer tables from pointer_table(); returns (status, layers_done)."""
+        s = _i32(seq_ids)
+        done = C.c_int32(0)
+        rc = lib.mixattn_decode_layers(self.h, layer_begin, layer_end, len(s), _p32(s), q_tab, k_tab, v_tab, out_tab,
+                                       _stream(stream), C.byref(done))
+        return rc, done.value
+
+    def decode_layers(self, layer_begin, layer_end, seq_ids, q_tab, k_tab, v_tab, out_tab, stream=None):
+        rc, _ = self.rc_decode_layers(layer_begin, layer_end, seq_ids, q_tab, k_tab, v_tab, out_tab, stream)
+        if rc:
+            raise MixAttnError(rc, "mixattn_decode_layers")
 
     def rc_prefill(self, layer, seq_ids, seq_lens, q, k, v, out, stream=None) -> int:
         s, n = _i32(seq_ids), _i32(seq_lens)

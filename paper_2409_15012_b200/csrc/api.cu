@@ -491,6 +491,26 @@ int mixattn_decode(mixattn_ctx* c, int32_t layer, int32_t n_seqs, const int32_t*
   return MIXATTN_OK;
 }
 
+int mixattn_decode_layers(mixattn_ctx* c, int32_t layer_begin, int32_t layer_end, int32_t n_seqs,
+                          const int32_t* seq_ids, const void* const* q, const void* const* k,
+                          const void* const* v, void* const* out, void* stream, int32_t* layers_done) {
+  if (layers_done != nullptr) *layers_done = 0;
+  if (c == nullptr || layer_begin < 0 || layer_end < layer_begin || layer_end > c->cm.n_layers())
+    return MIXATTN_ERR_INVALID_ARG;
+  if (layer_end > layer_begin && (q == nullptr || out == nullptr || k == nullptr || v == nullptr))
+    return MIXATTN_ERR_INVALID_ARG;
+  for (int l = layer_begin; l < layer_end; ++l) {
+    if (c->cm.layer(l).owner == l) {
+      int rc = append_impl(c, l, n_seqs, seq_ids, nullptr, k[l], v[l], stream, 0.0);
+      if (rc != MIXATTN_OK) return rc;
+    }
+    int rc = mixattn_decode(c, l, n_seqs, seq_ids, q[l], out[l], stream);
+    if (rc != MIXATTN_OK) return rc;
+    if (layers_done != nullptr) *layers_done = l - layer_begin + 1;
+  }
+  return MIXATTN_OK;
+}
+
 int mixattn_prefill(mixattn_ctx* c, int32_t layer, int32_t n_seqs, const int32_t* seq_ids,
                     const int32_t* seq_lens, const void* q, const void* k, const void* v,
                     void* out, void* stream) {

@@ -115,15 +115,28 @@ class Session:
         wl = self.wl
         return torch.empty(len(wl.layout), wl.batch, wl.n_q_heads, wl.head_dim, dtype=self.dt, device=self.dev)
 
-    def decode_step(self, inputs, outs: torch.Tensor, stream=None, advance: bool = True):
-        """One decode step of the whole model: per layer, append (owners) then attend."""
+    def step_tables(self, inputs, outs: torch.Tensor):
+        """Pointer tables of one step's inputs and outputs for mixattn_decode_layers."""
+        L = len(self.wl.layout)
+        return (self.ctx.pointer_table([inputs[l]["q"] for l in range(L)]),
+                self.ctx.pointer_table([inputs[l].get("k") for l in range(L)]),
+                self.ctx.pointer_table([inputs[l].get("v") for l in range(L)]),
+                self.ctx.pointer_table([outs[l] for l in range(L)]))
+
+    def decode_step(self, inputs, outs: torch.Tensor, stream=None, advance: bool = True, tables=None,
+                    layer_range=None):
+        """One decode step of the whole model (or of the layers in layer_range): per layer, append
+        (owners) then attend, issued as one mixattn_decode_layers call.  `tables` = step_tables(inputs,
+        outs) when the caller has built them ahead of time."""
         wl = self.wl
         ids = list(range(wl.batch))
-        for l in range(len(wl.layout)):
-            ent = inputs[l]
-            if "k" in ent:
-                self._append(l, ids, None, ent["k"], ent["v"], stream)
-            self.ctx.decode(l, ids, ent["q"], outs[l], stream)
+        lo, hi = (0, len(wl.layout)) if layer_range is None else layer_range
+        q_tab, k_tab, v_tab, o_tab = self.step_tables(inputs, outs) if tables is None else tables
+        self.ctx.decode_layers(lo, hi, ids, q_tab, k_tab, v_tab, o_tab, stream)
+        if self.mirror is not None:
+            for l in range(lo, hi):
+                if wl.layout[l][2] == l:
+                    self.mirror.append(l, ids, None)
         if advance:
             self.pos += 1
 

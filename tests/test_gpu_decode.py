@@ -166,3 +166,43 @@ def test_bf16_few_items_short_and_long_sequences_together():
     # stage or less leaves the second CTA without keys, 65 keys give it a single one
     wl = cf.mid_decode().scaled(layout=cf.layout_tiny(512), batch=4, context=1000, n_q_heads=16, n_kv_heads=4)
     run_decode_case(wl, [1000, 4, 63, 64], steps=2, chunk=250)
+
+
+def test_decode_layers_is_the_per_layer_calls():
+    # one mixattn_decode_layers call over all layers, and over two ranges, against the individual
+    # append_kv / decode calls: same cache state, same bits
+    mx, runner = load_lib()
+    wl = cf.mid_decode().scaled(layout=cf.layout_mid(256, 6), batch=3, context=0)
+    lengths = [700, 40, 2100]
+    outs_by_mode = []
+    for mode in ("calls", "one", "ranges"):
+        sess = runner.Session(wl, lengths, headroom_tokens=3)
+        try:
+            sess.fill(512)
+            ids = list(range(wl.batch))
+            for step in range(2):
+                inputs = sess.step_inputs()
+                outs = sess.alloc_outputs()
+                outs.fill_(float("nan"))
+                if mode == "calls":
+                    for l in range(len(wl.layout)):
+                        ent = inputs[l]
+                        if "k" in ent:
+                            sess.ctx.append_kv(l, ids, None, ent["k"], ent["v"])
+                        sess.ctx.decode(l, ids, ent["q"], outs[l])
+                    sess.pos += 1
+                elif mode == "one":
+                    sess.decode_step(inputs, outs)
+                else:
+                    sess.decode_step(inputs, outs, advance=False, layer_range=(0, 2))
+                    sess.decode_step(inputs, outs, layer_range=(2, len(wl.layout)))
+            torch.cuda.synchronize()
+            assert sess.ctx.get_device_status() == 0
+            state = [[sess.ctx.get_len(l, b) for b in ids] for l in range(len(wl.layout))]
+            outs_by_mode.append((outs.clone(), state, [sess.ctx.get_block_table(b) for b in ids]))
+        finally:
+            sess.close()
+    ref = outs_by_mode[0]
+    for got in outs_by_mode[1:]:
+        assert torch.equal(got[0].view(torch.int16), ref[0].view(torch.int16))
+        assert got[1] == ref[1] and got[2] == ref[2]

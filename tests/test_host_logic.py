@@ -207,3 +207,23 @@ def test_quantised_storage_config_rules_and_cache_bytes():
     ctx.append_kv(0, [0, 1], [20, 3])
     assert ctx.get_len(12, 0) == 20 and ctx.get_block_table(0) == [0, 1] and ctx.get_block_table(1) == [2]
     ctx.close()
+
+
+def test_decode_layers_stops_at_the_first_failing_call_and_says_where():
+    import ctypes as C
+    lay = cf.layout_tiny(64)
+    ctx = mx.Context(lay, 4, 2, 64, mx.F32, 2, 8, device=-1)
+    tab = (C.c_void_p * 4)(*([256] * 4))     # (never dereferenced: a host-only context launches nothing)
+    # a host-only context keeps the books but cannot attend: layer 0's append stands, its decode fails
+    rc, done = ctx.rc_decode_layers(0, 4, [0, 1], tab, tab, tab, tab)
+    assert rc == mx.ERR_CUDA and done == 0
+    assert ctx.get_len(0, 0) == 1 and ctx.get_len(1, 0) == 0
+    # an empty range does nothing; bad ranges are refused
+    assert ctx.rc_decode_layers(2, 2, [0], tab, tab, tab, tab) == (0, 0)
+    assert ctx.rc_decode_layers(3, 2, [0], tab, tab, tab, tab)[0] == mx.ERR_INVALID_ARG
+    assert ctx.rc_decode_layers(0, 5, [0], tab, tab, tab, tab)[0] == mx.ERR_INVALID_ARG
+    assert ctx.rc_decode_layers(0, 1, [0], None, tab, tab, tab)[0] == mx.ERR_INVALID_ARG
+    # a bad sequence id is refused by the first call, nothing moves
+    rc, done = ctx.rc_decode_layers(1, 3, [7], tab, tab, tab, tab)
+    assert rc == mx.ERR_BAD_SEQ and done == 0 and ctx.get_len(1, 0) == 0
+    ctx.close()
