@@ -8,7 +8,7 @@ import torch
 from synth import configs as cf
 from synth import inputs as si
 
-from gpu_common import run_decode_case
+from gpu_common import load_lib, run_decode_case
 
 pytestmark = pytest.mark.gpu
 
