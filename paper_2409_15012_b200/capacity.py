@@ -16,27 +16,29 @@ from . import binding as mx
 
 
 def cache_bytes(layout: Sequence, n_q_heads: int, n_kv_heads: int, head_dim: int, dtype: int,
-                n_seqs: int, tokens_per_seq: int) -> int:
-    """Bytes of K/V storage for n_seqs sequences of tokens_per_seq tokens each."""
+                n_seqs: int, tokens_per_seq: int, kv_format: int = mx.KV_NATIVE) -> int:
+    """Bytes of K/V storage for n_seqs sequences of tokens_per_seq tokens each (kv_format:
+    native, or the quantised storage of Section 2's "KV Quantization")."""
     n_pages = n_seqs * (-(-tokens_per_seq // 16))
-    cfg, keep = mx.make_config(layout, n_q_heads, n_kv_heads, head_dim, dtype, n_seqs, max(n_pages, 1))
+    cfg, keep = mx.make_config(layout, n_q_heads, n_kv_heads, head_dim, dtype, n_seqs, max(n_pages, 1),
+                               kv_format=kv_format)
     return mx.cache_bytes(cfg)
 
 
 def max_sequences(layout: Sequence, n_q_heads: int, n_kv_heads: int, head_dim: int, dtype: int,
-                  tokens_per_seq: int, budget_bytes: int) -> int:
+                  tokens_per_seq: int, budget_bytes: int, kv_format: int = mx.KV_NATIVE) -> int:
     """Largest batch of sequences of tokens_per_seq tokens whose caches fit in budget_bytes.
     Storage is linear in the number of sequences (pages and rings are per sequence)."""
-    per_seq = cache_bytes(layout, n_q_heads, n_kv_heads, head_dim, dtype, 1, tokens_per_seq)
+    per_seq = cache_bytes(layout, n_q_heads, n_kv_heads, head_dim, dtype, 1, tokens_per_seq, kv_format)
     return budget_bytes // per_seq
 
 
 def capacity_table(layouts: Dict[str, Sequence], n_q_heads: int, n_kv_heads: int, head_dim: int, dtype: int,
-                   tokens_per_seq: int, budget_bytes: int):
+                   tokens_per_seq: int, budget_bytes: int, kv_format: int = mx.KV_NATIVE):
     """{name: (bytes per sequence, max sequences, max total tokens)} for each layout."""
     out = {}
     for name, lay in layouts.items():
-        per_seq = cache_bytes(lay, n_q_heads, n_kv_heads, head_dim, dtype, 1, tokens_per_seq)
-        n = max_sequences(lay, n_q_heads, n_kv_heads, head_dim, dtype, tokens_per_seq, budget_bytes)
+        per_seq = cache_bytes(lay, n_q_heads, n_kv_heads, head_dim, dtype, 1, tokens_per_seq, kv_format)
+        n = max_sequences(lay, n_q_heads, n_kv_heads, head_dim, dtype, tokens_per_seq, budget_bytes, kv_format)
         out[name] = (per_seq, n, n * tokens_per_seq)
     return out

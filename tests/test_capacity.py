@@ -82,3 +82,12 @@ def test_named_variants_have_the_properties_the_paper_states():
     for name in V:
         if name.startswith("MA"):
             assert tab[name][0] * 5 < tab["standard"][0]
+
+
+def test_quantised_storage_scales_every_layout_by_129_over_256():
+    V = {k: f() for k, f in cf.PAPER_VARIANTS.items()}
+    a = capacity.capacity_table(V, 12, 3, 128, mx.BF16, 32000, 150 * 10**9)
+    b = capacity.capacity_table(V, 12, 3, 128, mx.BF16, 32000, 150 * 10**9, kv_format=mx.KV_FP8_E4M3)
+    for name in V:
+        assert b[name][0] * 256 == a[name][0] * 129
+        assert b[name][1] >= a[name][1] * 256 // 129 - 1
