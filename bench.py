@@ -377,9 +377,6 @@ def device_pass(sess, runner, wl, ring, outs, stream, K, Wm, barrier, sampler=No
     launching stream, inputs resident in HBM.  The first region decides how many more follow
     (n_regions_for).  Returns (mean ms per region, mean KV bytes per region, regions, launches
     per region)."""
-    def bytes_next_step():
-        return runner.kv_bytes_per_step(wl, [int(p) + 1 for p in sess.pos], sess.kv_format)
-
     tables = [sess.step_tables(inp, outs) for inp in ring]    # pointer tables, built once per ring entry
     step = 0
     for _ in range(Wm):
@@ -394,10 +391,10 @@ def device_pass(sess, runner, wl, ring, outs, stream, K, Wm, barrier, sampler=No
     def region():
         nonlocal step
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        b = 0
+        # bytes of the region's K steps, counted ahead of the timed calls (every step adds one token per sequence)
+        b = sum(runner.kv_bytes_per_step(wl, sess.pos + 1 + k, sess.kv_format) for k in range(K))
         e0.record(stream)
         for _ in range(K):
-            b += bytes_next_step()
             sess.decode_step(ring[step % len(ring)], outs, stream, tables=tables[step % len(ring)])
             step += 1
         e1.record(stream)
@@ -480,9 +477,6 @@ def run_gpu_arm(args, wl):
         if dist is not None:
             dist.barrier()
         torch.cuda.synchronize()
-
-    def bytes_next_step():
-        return runner.kv_bytes_per_step(wl, [int(p) + 1 for p in sess.pos], kvf)
 
     # ---- device-resident pass: `value` ----
     kRing = min(8, Wm + K)
@@ -569,11 +563,10 @@ def run_gpu_arm(args, wl):
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     step = Wm
     for _ in range(regions):
-        b = 0
+        b = sum(runner.kv_bytes_per_step(wl, sess.pos + 1 + k, kvf) for k in range(K))   # counted ahead of the timed steps
         t0 = time.perf_counter()
         ev0.record(stream)
         for _ in range(K):
-            b += bytes_next_step()
             e2e_step(step)
             step += 1
         ev1.record(stream)

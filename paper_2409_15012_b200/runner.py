@@ -217,10 +217,10 @@ def kv_bytes_per_step(wl: cf.Workload, lengths_after: Sequence[int], kv_format: 
     per_tok = 2 * wl.n_kv_heads * wl.head_dim * e
     if kv_format == mx.KV_FP8_E4M3:
         per_tok = 2 * wl.n_kv_heads * (wl.head_dim + 1)
+    n = np.asarray(lengths_after, dtype=np.int64)
     total = 0
     for kind, window, _ in wl.layout:
-        for n in lengths_after:
-            total += (min(int(n), window) if kind == cf.SLIDING else int(n)) * per_tok
+        total += int((np.minimum(n, window) if kind == cf.SLIDING else n).sum()) * per_tok
     return total
 
 
