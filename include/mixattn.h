@@ -214,7 +214,11 @@ int mixattn_decode_layers(mixattn_ctx* ctx, int32_t layer_begin, int32_t layer_e
  * If `layer` owns its cache the call also stores K/V as mixattn_append_kv
  * would (a ring ends up holding the last min(S_b, window) tokens); the
  * owner's cache for these sequences must be empty, else UNSUPPORTED.  A
- * reader stores nothing.  Errors: as append_kv and decode. */
+ * reader stores nothing.  Errors: as append_kv and decode.
+ * Performance note: bf16 with head_dim 128 and 16-byte aligned tensors runs
+ * on the tensor cores; fp32 contexts, head_dim 64 and unaligned tensors take
+ * an exact CUDA-core kernel that is about two orders of magnitude slower
+ * (the same holds for mixattn_attend_chunk). */
 int mixattn_prefill(mixattn_ctx* ctx, int32_t layer, int32_t n_seqs, const int32_t* seq_ids,
                     const int32_t* seq_lens, const void* q, const void* k, const void* v,
                     void* out, void* stream);
