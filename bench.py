@@ -268,8 +268,12 @@ def chunk_figures(mx, runner, peaks, device, prefix=6144, chunk=2048):
         ids, lens = list(range(B)), [chunk] * B
         pairs_full = sum(prefix + r + 1 for r in range(chunk))
         pairs_slide = sum(min(prefix + r + 1, W) for r in range(chunk))
-        for name, layer, pairs, cls in (("full", 12, pairs_full, mx.K_PREFILL_FULL),
-                                        ("sliding", 2, pairs_slide, mx.K_PREFILL_SLIDING)):
+        # "sliding": the ring read in place by the attention kernel (the default); "sliding_copied":
+        # the same call with the cached keys copied out of the ring first
+        for name, layer, pairs, cls, in_place in (("full", 12, pairs_full, mx.K_PREFILL_FULL, True),
+                                                  ("sliding", 2, pairs_slide, mx.K_PREFILL_SLIDING, True),
+                                                  ("sliding_copied", 2, pairs_slide, mx.K_PREFILL_SLIDING, False)):
+            sess.ctx.set_chunk_ring_direct(in_place)
             owner = wl.layout[layer][2]
             q = si.q_tokens_multi(wl.seed, layer, ids, [prefix] * B, chunk, Hq, D, sess.dt,
                                   sess.dev).reshape(-1, Hq, D)
@@ -287,12 +291,14 @@ def chunk_figures(mx, runner, peaks, device, prefix=6144, chunk=2048):
             ng, msg = sess.ctx.profile_read(mx.K_GATHER)
             sess.ctx.profile_enable(False)
             flops = 4.0 * D * pairs * Hq * B
-            t = (ms / n + msg / ng) * 1e-3
-            res[name] = {"ms_attention": ms / n, "ms_gather": msg / ng, "tflops": flops / t / 1e12,
+            ms_gather = msg / ng if ng else 0.0
+            t = (ms / n + ms_gather) * 1e-3
+            res[name] = {"ms_attention": ms / n, "ms_gather": ms_gather, "tflops": flops / t / 1e12,
                          "frac_of_bf16_peak": flops / t / 1e12 / peaks["bf16_tflops"],
                          "frac_of_nominal_2250": flops / t / 1e12 / NOMINAL_BF16_TFLOPS, "useful_flop": flops}
-        # the same chunk through all 24 layers, each reader handed its owner's K/V, with the copy of
-        # the cached keys shared by the layers that read one cache (4 copies: F, S1, F, S2)
+        # the same chunk through all 24 layers, each reader handed its owner's K/V; the rings are
+        # read in place, and the copy of the standard cache's keys serves both layers that read it
+        sess.ctx.set_chunk_ring_direct(True)
         sess.ctx.set_chunk_gather_reuse(True)
         kv = {}
         for o in sess.owners:
@@ -302,6 +308,7 @@ def chunk_figures(mx, runner, peaks, device, prefix=6144, chunk=2048):
         out = torch.empty_like(q)
         flops_pass = 0.0
         for timed in (False, True):
+            sess.ctx.set_chunk_gather_reuse(True)   # forgets the previous pass: a chunk's first reader copies
             sess.ctx.profile_enable(timed)
             for layer, (kind, _, owner) in enumerate(wl.layout):
                 sess.ctx.attend_chunk(layer, ids, lens, q, kv[owner][0], kv[owner][1], out)

@@ -240,7 +240,10 @@ int mixattn_prefill(mixattn_ctx* ctx, int32_t layer, int32_t n_seqs, const int32
  * window of the chunk's first token when the last of them runs).
  * The cached keys the chunk needs (all of a paged cache, the last window-1
  * tokens of a ring) and the chunk's are first copied into plain tensors in the
- * context's chunk scratch, sequences in groups that fit it.
+ * context's chunk scratch, sequences in groups that fit it.  Exception: a ring
+ * whose window is a multiple of 128 tokens (bf16, head_dim 128, native storage)
+ * is read in place, see mixattn_set_chunk_ring_direct; the size rules below
+ * are the same either way.
  * Errors: UNSUPPORTED if the context was created with chunk_scratch_tokens = 0,
  * TOO_LARGE if one sequence's keys alone exceed the scratch, BAD_SEQ,
  * INVALID_ARG (null, duplicates, S_b < 1, n + S_b beyond max_seq_len), CUDA. */
@@ -261,6 +264,20 @@ int mixattn_attend_chunk(mixattn_ctx* ctx, int32_t layer, int32_t n_seqs, const 
  * and forgets what the scratch holds.  Results are identical either way.
  * Errors: INVALID_ARG for a null context. */
 int mixattn_set_chunk_gather_reuse(mixattn_ctx* ctx, int32_t enable);
+
+/* Chunk calls on sliding-window layers without the copy (Section 3: such a
+ * layer keeps the last `window` tokens; the chunk's queries need at most the
+ * last window-1 of them).  Token p of a ring lives in slot p mod window, so
+ * when window is a multiple of the 128-key tile of the tensor-core kernel, a
+ * tile of cached keys is eight whole pages of the sequence's ring, stored in
+ * the layout the tensor cores read; the kernel then fetches those tiles from
+ * the ring itself and the chunk's own K/V from the caller's tensors.  Applies
+ * to bf16 contexts with head_dim 128 and native KV storage; every other chunk
+ * call copies as described above.  On by default; enable = 0 makes every chunk
+ * call copy.  Both ways attend to the same keys; the results differ by
+ * rounding only (the keys are cut into tiles at different places).
+ * Errors: INVALID_ARG for a null context. */
+int mixattn_set_chunk_ring_direct(mixattn_ctx* ctx, int32_t enable);
 
 /* Size of the static device array behind mixattn_decode_static_scratch. */
 #define MIXATTN_STATIC_SCRATCH_BYTES (8u << 20)

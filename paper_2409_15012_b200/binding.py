@@ -90,6 +90,7 @@ def _load() -> C.CDLL:
         "mixattn_get_device_status": [vp, p32],
         "mixattn_set_split_tokens": [vp, i32],
         "mixattn_set_chunk_gather_reuse": [vp, i32],
+        "mixattn_set_chunk_ring_direct": [vp, i32],
         "mixattn_profile_enable": [vp, i32],
         "mixattn_profile_read": [vp, i32, p32, C.POINTER(C.c_float)],
         "mixattn_get_launch_count": [vp, C.POINTER(C.c_int64)],
@@ -111,6 +112,7 @@ EXPORTS = [
     "mixattn_get_len", "mixattn_get_block_table", "mixattn_get_n_free_pages",
     "mixattn_get_ring_state", "mixattn_locate", "mixattn_debug_read_kv", "mixattn_debug_read_kv_fp8",
     "mixattn_get_device_status", "mixattn_set_split_tokens", "mixattn_set_chunk_gather_reuse",
+    "mixattn_set_chunk_ring_direct",
     "mixattn_profile_enable",
     "mixattn_profile_read", "mixattn_get_launch_count", "mixattn_strerror",
 ]
@@ -381,6 +383,13 @@ class Context:
         rc = lib.mixattn_set_chunk_gather_reuse(self.h, 1 if enable else 0)
         if rc:
             raise MixAttnError(rc, "mixattn_set_chunk_gather_reuse")
+
+    def set_chunk_ring_direct(self, enable: bool):
+        """Sliding-window chunk calls read the ring in place where its window is a whole number of
+        128-key tiles (on by default); off = they copy the cached keys like every other chunk call."""
+        rc = lib.mixattn_set_chunk_ring_direct(self.h, 1 if enable else 0)
+        if rc:
+            raise MixAttnError(rc, "mixattn_set_chunk_ring_direct")
 
     def profile_enable(self, enable: bool):
         rc = lib.mixattn_profile_enable(self.h, 1 if enable else 0)

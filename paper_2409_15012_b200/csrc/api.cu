@@ -95,6 +95,9 @@ struct mixattn_ctx {
   // Chunk calls of layers that share a cache gather the same rows: what the scratch holds is
   // remembered so that, when the caller has enabled it, the copy runs once per run of such calls.
   bool chunk_reuse = false;
+  // Chunk calls of sliding-window layers whose window is a whole number of key tiles read the
+  // cached keys in place from the ring (no copy); off = every chunk call copies.
+  bool chunk_ring_direct = true;
   uint64_t cache_epoch = 0;   // bumped by every call that changes a cache
   struct GatherKey {
     bool valid = false;
@@ -663,8 +666,14 @@ int mixattn_attend_chunk(mixattn_ctx* c, int32_t layer, int32_t n_seqs, const in
     for (int i = 0; i < n_seqs; ++i) rows += (int64_t)n_prefix[i] + seq_lens[i];
     one_piece = one_piece && rows <= scratch;
   }
-  mixattn_ctx::GatherKey& held = c->scratch_holds;
-  const bool reuse = c->chunk_reuse && one_piece && held.valid && held.owner == li.owner &&
+  // A ring whose window is a whole number of key tiles is read where it is: a key tile of the
+  // cached positions is eight consecutive pages of the sequence's ring, in the layout the tensor
+  // cores take.  K / V of the chunk itself then come from the caller's tensors.
+  const bool direct = ring && c->chunk_ring_direct && prefill_tc_ring_direct_supported(c->geom, li.window) &&
+                      prefill_tc_supported(c->cfg.dtype, D, q, k, v) && (((size_t)out) & 15) == 0;
+  mixattn_ctx::GatherKey dummy;
+  mixattn_ctx::GatherKey& held = direct ? dummy : c->scratch_holds;
+  const bool reuse = !direct && c->chunk_reuse && one_piece && held.valid && held.owner == li.owner &&
                      held.epoch == c->cache_epoch && held.k == k && held.v == v && held.st == st &&
                      held.ids.size() == (size_t)n_seqs &&
                      std::equal(held.ids.begin(), held.ids.end(), seq_ids) &&
@@ -698,8 +707,10 @@ int mixattn_attend_chunk(mixattn_ctx* c, int32_t layer, int32_t n_seqs, const in
       e.src_row0 = qrow;
       e.dst_row0 = krow;
       p.row0[nb] = qrow;
-      p.krow0[nb] = krow;
-      p.prefix[nb] = n_prefix[i];
+      p.krow0[nb] = direct ? qrow : krow;
+      p.prefix[nb] = direct ? c->cm.len(layer, seq_ids[i]) : n_prefix[i];
+      p.cached[nb] = p.prefix[nb];
+      p.ring_page0[nb] = seq_ids[i] * ring_pages_of(li.window);
       krow += rows;
       qrow += seq_lens[i];
       if (seq_lens[i] > mlen) mlen = seq_lens[i];
@@ -713,14 +724,23 @@ int mixattn_attend_chunk(mixattn_ctx* c, int32_t layer, int32_t n_seqs, const in
     gp.v_chunk = static_cast<const char*>(v) + (size_t)row * Hkv * D * esz;
     p.q = static_cast<const char*>(q) + (size_t)row * Hq * D * esz;
     p.out = static_cast<char*>(out) + (size_t)row * Hq * D * esz;
+    if (direct) {
+      p.k = gp.k_chunk;
+      p.v = gp.v_chunk;
+      p.ring_pool = gp.pool;
+      p.ring_pages = gp.ring_pages;
+      p.ring_total_pages = (int64_t)c->cm.max_seqs() * gp.ring_pages;
+      p.geom = c->geom;
+    }
     cudaError_t e = cudaSuccess;
-    if (!reuse) {
+    if (!reuse && !direct) {
       e = launch_recorded(c, MIXATTN_K_GATHER, st, [&] { return launch_gather(gp, max_rows, st); });
       if (e != cudaSuccess) return MIXATTN_ERR_CUDA;
       held.valid = one_piece;
     }
     const int cls = p.window ? MIXATTN_K_PREFILL_SLIDING : MIXATTN_K_PREFILL_FULL;
     const bool tc = prefill_tc_supported(c->cfg.dtype, D, p.q, p.k, p.v) && (((size_t)p.out) & 15) == 0;
+    if (direct && !tc) return MIXATTN_ERR_INVALID_ARG;   // (not reachable: the pointers were checked above)
     e = launch_recorded(c, cls, st, [&] {
       return tc ? launch_prefill_tc(p, mlen, c->sm_count, st) : launch_prefill_simple(p, c->cfg.dtype, mlen, st);
     });
@@ -912,6 +932,12 @@ int mixattn_set_chunk_gather_reuse(mixattn_ctx* c, int32_t enable) {
   if (c == nullptr) return MIXATTN_ERR_INVALID_ARG;
   c->chunk_reuse = enable != 0;
   c->scratch_holds.valid = false;
+  return MIXATTN_OK;
+}
+
+int mixattn_set_chunk_ring_direct(mixattn_ctx* c, int32_t enable) {
+  if (c == nullptr) return MIXATTN_ERR_INVALID_ARG;
+  c->chunk_ring_direct = enable != 0;
   return MIXATTN_OK;
 }
 

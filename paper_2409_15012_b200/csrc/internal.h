@@ -146,8 +146,17 @@ struct PrefillParams {
   int32_t* status;
   int32_t row0[kMaxCallSeqs + 1];   // first row of each sequence in q / out (packed)
   int32_t krow0[kMaxCallSeqs];      // first row of each sequence in k / v
-  int32_t prefix[kMaxCallSeqs];     // key rows of the sequence that precede its first query:
-                                    // k / v hold prefix + (row0[b + 1] - row0[b]) rows for sequence b
+  int32_t prefix[kMaxCallSeqs];     // keys of the sequence that precede its first query
+  // The first cached[b] of those keys are not in k / v but in a ring cache, read in place by the
+  // tensor-core kernel (k / v then hold prefix[b] - cached[b] + (row0[b + 1] - row0[b]) rows for
+  // sequence b); 0 everywhere = every key comes from k / v.  Keys are then numbered by their
+  // position in the sequence, so that key tiles fall on whole ring pages.
+  int32_t cached[kMaxCallSeqs];
+  int32_t ring_page0[kMaxCallSeqs]; // first page of the sequence's ring in ring_pool
+  const void* ring_pool = nullptr;  // storage of the ring (nullptr = no sequence has cached keys)
+  int32_t ring_pages;               // pages per sequence in the ring (a multiple of 8)
+  int64_t ring_total_pages;         // pages in ring_pool
+  KvGeom geom;
 };
 
 // Copies the cached keys a chunk of queries needs, followed by the chunk's own keys, into
@@ -199,6 +208,7 @@ cudaError_t launch_decode_split_f32(const DecodeParams& p, cudaStream_t st);
 cudaError_t launch_decode_combine(const DecodeParams& p, int dtype, cudaStream_t st);
 cudaError_t launch_prefill_simple(const PrefillParams& p, int dtype, int max_len, cudaStream_t st);
 bool prefill_tc_supported(int dtype, int head_dim, const void* q, const void* k, const void* v);
+bool prefill_tc_ring_direct_supported(const KvGeom& ge, int window);   // cached keys read in place from a ring
 cudaError_t prepare_prefill_tc();
 cudaError_t launch_prefill_tc(const PrefillParams& p, int max_len, int sm_count, cudaStream_t st);
 

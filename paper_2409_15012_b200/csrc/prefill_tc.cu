@@ -84,7 +84,10 @@ struct TcParams {
   __nv_bfloat16* out;
   int32_t row0[kMaxCallSeqs + 1];   // first q / out row of each sequence
   int32_t krow0[kMaxCallSeqs];      // first k / v row of each sequence
-  int32_t prefix[kMaxCallSeqs];     // key rows before the sequence's first query
+  int32_t prefix[kMaxCallSeqs];     // keys before the sequence's first query
+  int32_t cached[kMaxCallSeqs];     // the first so many of them live in a ring cache, not in k / v
+  int32_t ring_page0[kMaxCallSeqs]; // first page of the sequence's ring
+  int32_t ring_pages;               // pages per sequence in the ring (a multiple of 8)
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -130,6 +133,12 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map
   asm volatile(
       "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
       ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(z), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap* map, int c0, int c1, int c2, int c3, int c4,
+                                            uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.5d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5, %6}], [%7];"
+      ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4), "r"(bar) : "memory");
 }
 // Shared-memory matrix descriptor, 128-byte swizzle, sm_100 format (version 1).
 // lbo / sbo in bytes.
@@ -228,11 +237,17 @@ __host__ __device__ constexpr uint32_t idesc_bf16(int b_mn) {
 // tile index, head): the CTAs of the grid work on one sequence at a time, whose K/V stays
 // in L2 (a pass over all sequences at once re-read K/V from HBM 5x), heaviest tiles first,
 // and the heads of a KV group, which read the same K/V tiles, run at the same time.
+constexpr int kNoDup = 1 << 30;
 struct WorkItem {
   int h, g, row_base, krow_base, S, i0, pos0, jt_lo, n_tiles;   // pos0 = position of query row i0 among the keys
+  // Keys cached in a ring are read from the ring, the others from k / v.  When the cached keys
+  // end inside a tile, that tile is visited twice: entry dup - 1 of the item's tile list takes
+  // its cached keys from the ring, entry dup the rest from k / v (each masks the other's keys).
+  int cached, ring_page0, dup;                                  // dup = kNoDup when no tile is visited twice
   bool valid;
   bool lo;   // rows of this tile may see fewer than a tile of keys: P enters P V as two bf16 terms
 };
+template <bool kRing>
 __device__ __forceinline__ WorkItem get_item(const TcParams& p, int id) {
   WorkItem w;
   const int per_seq = p.max_qt * p.n_q_heads;
@@ -252,6 +267,13 @@ __device__ __forceinline__ WorkItem get_item(const TcParams& p, int id) {
   const int key_lo = p.window > 0 ? max(0, w.pos0 - p.window + 1) : 0;
   w.jt_lo = key_lo / kBN;
   w.n_tiles = key_hi / kBN - w.jt_lo + 1;
+  w.cached = kRing ? p.cached[b] : 0;
+  w.ring_page0 = kRing ? p.ring_page0[b] : 0;
+  w.dup = kNoDup;
+  if (kRing && w.cached % kBN != 0 && w.cached / kBN >= w.jt_lo) {   // (the queries sit behind the cached keys, so that tile is not past the last)
+    w.dup = w.cached / kBN - w.jt_lo + 1;
+    ++w.n_tiles;
+  }
   // A row that sees only a few keys is a mix of a few V rows: its weights' bf16 rounding (2^-9
   // each) does not average out and, on outputs of magnitude 2..4, would add to the output's own
   // bf16 rounding.  Such rows (the first query tile of a sequence, or a window shorter than a
@@ -261,9 +283,19 @@ __device__ __forceinline__ WorkItem get_item(const TcParams& p, int id) {
   return w;
 }
 
+// key tile (index along the sequence's keys) of entry j of an item's tile list
+template <bool kRing>
+__device__ __forceinline__ int tile_of(const WorkItem& w, int j) {
+  return kRing ? w.jt_lo + j - (j >= w.dup ? 1 : 0) : w.jt_lo + j;
+}
+
+// kRing: some sequences have cached keys in a ring (a separate instantiation, so that the
+// ordinary launches carry none of its code)
+template <bool kRing>
 __global__ void __launch_bounds__(kThreads, 1)
 prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
-                  const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ TcParams p) {
+                  const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_ring,
+                  const __grid_constant__ TcParams p) {
   extern __shared__ __align__(1024) unsigned char smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   unsigned char* gbase = smem_raw + (base - smem_u32(smem_raw));
@@ -318,10 +350,11 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_q) : "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_k) : "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_v) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_ring) : "memory");
         bool ok = true;
         int G = 0, it = 0, q_issued = 0, k_issued = 0, v_issued = 0;
         for (int id = blockIdx.x; id < n_ids && ok; id += gridDim.x) {
-          const WorkItem w = get_item(p, id);
+          const WorkItem w = get_item<kRing>(p, id);
           if (!w.valid) continue;
           const int qb = it & 1;
           if (it >= 2) ok = mbar_wait(BAR(B_QE + qb), ((it >> 1) - 1) & 1, abort_flag);
@@ -332,20 +365,37 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
           ++q_issued;
           for (int j = 0; j < w.n_tiles && ok; ++j) {
             const int Gj = G + j;
-            const int row = w.krow_base + (w.jt_lo + j) * kBN;
+            const int jt = tile_of<kRing>(w, j);
+            // A tile of cached keys is eight whole pages of the sequence's ring: the page rows are
+            // stored with the 16-byte chunks already permuted the way the MMA expects a
+            // 128-byte-swizzled tile, so an unswizzled copy of (8 pages x 16 tokens x 128 bytes)
+            // is that tile.  All other tiles come from k / v, whose row 0 is key w.cached.
+            const bool from_ring = kRing && jt * kBN < w.cached && j != w.dup;
+            const int row = w.krow_base + jt * kBN - w.cached;   // (negative rows of the tile shared with the ring read as zeros)
+            const int page = w.ring_page0 + (jt * (kBN / kPage)) % p.ring_pages;
             const int ks = Gj % kKStages, ku = Gj / kKStages;
             if (ku > 0) ok = mbar_wait(BAR(B_KE + ks), (ku - 1) & 1, abort_flag);
             if (!ok) break;
             mbar_expect_tx(BAR(B_KF + ks), kTileBytes);
-            tma_load_3d(base + kSmK + ks * kTileBytes, &tm_k, 0, w.g, row, BAR(B_KF + ks));
-            tma_load_3d(base + kSmK + ks * kTileBytes + kHalfBytes, &tm_k, 64, w.g, row, BAR(B_KF + ks));
+            if (from_ring) {
+              tma_load_5d(base + kSmK + ks * kTileBytes, &tm_ring, 0, 0, 0, w.g, page, BAR(B_KF + ks));
+              tma_load_5d(base + kSmK + ks * kTileBytes + kHalfBytes, &tm_ring, 64, 0, 0, w.g, page, BAR(B_KF + ks));
+            } else {
+              tma_load_3d(base + kSmK + ks * kTileBytes, &tm_k, 0, w.g, row, BAR(B_KF + ks));
+              tma_load_3d(base + kSmK + ks * kTileBytes + kHalfBytes, &tm_k, 64, w.g, row, BAR(B_KF + ks));
+            }
             ++k_issued;
             const int vs = Gj % kVStages, vu = Gj / kVStages;
             if (vu > 0) ok = mbar_wait(BAR(B_VE + vs), (vu - 1) & 1, abort_flag);
             if (!ok) break;
             mbar_expect_tx(BAR(B_VF + vs), kTileBytes);
-            tma_load_3d(base + kSmV + vs * kTileBytes, &tm_v, 0, w.g, row, BAR(B_VF + vs));
-            tma_load_3d(base + kSmV + vs * kTileBytes + kHalfBytes, &tm_v, 64, w.g, row, BAR(B_VF + vs));
+            if (from_ring) {
+              tma_load_5d(base + kSmV + vs * kTileBytes, &tm_ring, 0, 0, 1, w.g, page, BAR(B_VF + vs));
+              tma_load_5d(base + kSmV + vs * kTileBytes + kHalfBytes, &tm_ring, 64, 0, 1, w.g, page, BAR(B_VF + vs));
+            } else {
+              tma_load_3d(base + kSmV + vs * kTileBytes, &tm_v, 0, w.g, row, BAR(B_VF + vs));
+              tma_load_3d(base + kSmV + vs * kTileBytes + kHalfBytes, &tm_v, 64, w.g, row, BAR(B_VF + vs));
+            }
             ++v_issued;
           }
           G += w.n_tiles;
@@ -371,7 +421,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         bool ok = true;
         int G = 0, it = 0;
         for (int id = blockIdx.x; id < n_ids && ok; id += gridDim.x) {
-          const WorkItem w = get_item(p, id);
+          const WorkItem w = get_item<kRing>(p, id);
           if (!w.valid) continue;
           const int qb = it & 1;
           ok = mbar_wait(BAR(B_QF + qb), (it >> 1) & 1, abort_flag);
@@ -409,7 +459,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         bool ok = true;
         int G = 0, it = 0;
         for (int id = blockIdx.x; id < n_ids && ok; id += gridDim.x) {
-          const WorkItem w = get_item(p, id);
+          const WorkItem w = get_item<kRing>(p, id);
           if (!w.valid) continue;
           // the first P V of an item overwrites the O accumulator: the streams must have
           // read the previous item's result
@@ -454,7 +504,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     bool ok = true;
     int it = 0;
     for (int id = blockIdx.x; id < n_ids && ok; id += gridDim.x) {
-      const WorkItem w = get_item(p, id);
+      const WorkItem w = get_item<kRing>(p, id);
       if (!w.valid) continue;
       ok = __all_sync(0xffffffffu, mbar_wait(BAR(B_XC), it & 1, abort_flag));
       if (!ok) break;
@@ -514,7 +564,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     bool ok = true;
     int G = 0, it = 0;
     for (int id = blockIdx.x; id < n_ids && ok; id += gridDim.x) {
-      const WorkItem w = get_item(p, id);
+      const WorkItem w = get_item<kRing>(p, id);
       if (!w.valid) continue;
       const int i = w.pos0 + r;           // query position among the sequence's keys
       float m_ref = -INFINITY, l = 0.f;
@@ -534,13 +584,17 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         constexpr bool kLo = decltype(lo_tag)::value;
         for (int j = 0; j < w.n_tiles; ++j) {
           const int Gj = G + j, sb = Gj & 1;
-          const int j0 = (w.jt_lo + j) * kBN + hs * 64;   // first key of this stream's columns
+          const int j0 = tile_of<kRing>(w, j) * kBN + hs * 64;   // first key of this stream's columns
           const uint32_t s_addr = lane_base + kColS + sb * 128 + hs * 64;
-          // band edges: causal (keys after the query) and window (keys older than i - window)
-          const bool edge = (j0 + 63 > w.pos0) || (p.window > 0 && j0 <= w.pos0 + kBM - 1 - p.window);
+          // band edges: causal (keys after the query) and window (keys older than i - window); and
+          // the two visits of the tile in which the cached keys end
+          const bool edge = (j0 + 63 > w.pos0) || (p.window > 0 && j0 <= w.pos0 + kBM - 1 - p.window) ||
+                            (kRing && (j + 1 == w.dup || j == w.dup));
           auto mask_edges = [&]() {
-            const int k_max = i - j0;                                      // columns <= k_max are causal-visible
-            const int k_min = p.window > 0 ? i - p.window + 1 - j0 : 0;    // columns >= k_min are inside the window
+            int k_max = i - j0;                                      // columns <= k_max are causal-visible
+            int k_min = p.window > 0 ? i - p.window + 1 - j0 : 0;    // columns >= k_min are inside the window
+            if (kRing && j + 1 == w.dup) k_max = min(k_max, w.cached - 1 - j0);   // this visit: the cached keys only
+            if (kRing && j == w.dup) k_min = max(k_min, w.cached - j0);           // this visit: the keys from k / v only
   #pragma unroll
             for (int e = 0; e < 64; ++e)
               if (e > k_max || e < k_min) sv[e] = 0xff800000u;             // -inf
@@ -713,7 +767,28 @@ bool make_map(CUtensorMap* map, const void* ptr, int64_t rows, int heads) {
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Ring storage of one owner layer, native bf16 format with head_dim 128, seen as
+// [pages][heads][K | V][16 tokens][128 channels]; box = 64 channels x 16 tokens x 8 pages of one
+// head's K or V.  The stored rows carry the 128-byte-swizzle permutation already (internal.h),
+// so the copy itself does not swizzle.
+bool make_ring_map(CUtensorMap* map, const void* pool, const KvGeom& ge, int64_t pages) {
+  EncodeTiledFn fn = encode_fn();
+  if (fn == nullptr) return false;
+  cuuint64_t dims[5] = {128, (cuuint64_t)kPage, 2, (cuuint64_t)ge.n_kv_heads, (cuuint64_t)pages};
+  cuuint64_t strides[4] = {(cuuint64_t)ge.row_bytes, (cuuint64_t)kPage * ge.row_bytes, (cuuint64_t)ge.blk_bytes,
+                           (cuuint64_t)ge.page_bytes};
+  cuuint32_t box[5] = {64, (cuuint32_t)kPage, 1, 1, kBN / kPage};
+  cuuint32_t estr[5] = {1, 1, 1, 1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void*>(pool), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 }  // namespace
+
+bool prefill_tc_ring_direct_supported(const KvGeom& ge, int window) {
+  return !ge.fp8 && ge.swizzle && ge.head_dim == 128 && ge.elem_bytes == 2 && window > 0 && window % kBN == 0;
+}
 
 bool prefill_tc_supported(int dtype, int head_dim, const void* q, const void* k, const void* v) {
   auto aligned = [](const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; };
@@ -721,21 +796,32 @@ bool prefill_tc_supported(int dtype, int head_dim, const void* q, const void* k,
 }
 
 cudaError_t prepare_prefill_tc() {
-  return cudaFuncSetAttribute(prefill_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+  cudaError_t e = cudaFuncSetAttribute(prefill_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+  if (e != cudaSuccess) return e;
+  return cudaFuncSetAttribute(prefill_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
 }
 
 cudaError_t launch_prefill_tc(const PrefillParams& pp, int max_len, int sm_count, cudaStream_t st) {
   if (pp.n_seqs <= 0 || max_len <= 0) return cudaSuccess;
   const int64_t rows = pp.row0[pp.n_seqs];
-  int64_t k_rows = 0;   // k / v hold prefix + S rows per sequence
+  int64_t k_rows = 0;   // k / v hold prefix - cached + S rows per sequence
   for (int i = 0; i < pp.n_seqs; ++i) {
-    const int64_t end = (int64_t)pp.krow0[i] + pp.prefix[i] + (pp.row0[i + 1] - pp.row0[i]);
+    const int cached = pp.ring_pool != nullptr ? pp.cached[i] : 0;
+    if (cached < 0 || cached > pp.prefix[i]) return cudaErrorInvalidValue;
+    const int64_t end = (int64_t)pp.krow0[i] + pp.prefix[i] - cached + (pp.row0[i + 1] - pp.row0[i]);
     if (end > k_rows) k_rows = end;
   }
-  CUtensorMap tq, tk, tv;
+  CUtensorMap tq, tk, tv, tring;
   if (!make_map(&tq, pp.q, rows, pp.n_q_heads) || !make_map(&tk, pp.k, k_rows, pp.n_kv_heads) ||
       !make_map(&tv, pp.v, k_rows, pp.n_kv_heads))
     return cudaErrorInvalidValue;
+  if (pp.ring_pool != nullptr) {
+    if (!prefill_tc_ring_direct_supported(pp.geom, pp.window) || pp.ring_pages * kPage != pp.window ||
+        !make_ring_map(&tring, pp.ring_pool, pp.geom, pp.ring_total_pages))
+      return cudaErrorInvalidValue;
+  } else {
+    tring = tk;   // never read
+  }
   TcParams p;
   p.n_q_heads = pp.n_q_heads;
   p.group = pp.n_q_heads / pp.n_kv_heads;
@@ -748,11 +834,15 @@ cudaError_t launch_prefill_tc(const PrefillParams& pp, int max_len, int sm_count
   for (int i = 0; i < pp.n_seqs; ++i) {
     p.krow0[i] = pp.krow0[i];
     p.prefix[i] = pp.prefix[i];
+    p.cached[i] = pp.ring_pool != nullptr ? pp.cached[i] : 0;
+    p.ring_page0[i] = pp.ring_pool != nullptr ? pp.ring_page0[i] : 0;
   }
+  p.ring_pages = pp.ring_pool != nullptr ? pp.ring_pages : kBN / kPage;
   p.max_qt = (max_len + kBM - 1) / kBM;
   const int64_t n_ids = (int64_t)p.max_qt * pp.n_seqs * pp.n_q_heads;
   const int grid = (int)(n_ids < sm_count ? n_ids : sm_count);   // persistent: one CTA per SM
-  prefill_tc_kernel<<<grid, kThreads, kSmemBytes, st>>>(tq, tk, tv, p);
+  if (pp.ring_pool != nullptr) prefill_tc_kernel<true><<<grid, kThreads, kSmemBytes, st>>>(tq, tk, tv, tring, p);
+  else prefill_tc_kernel<false><<<grid, kThreads, kSmemBytes, st>>>(tq, tk, tv, tring, p);
   return cudaGetLastError();
 }
 

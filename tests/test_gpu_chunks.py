@@ -14,7 +14,7 @@ from gpu_common import check_close, check_stored_bits, compare_state, load_lib, 
 pytestmark = pytest.mark.gpu
 
 
-def run_chunked(wl: cf.Workload, schedule, scratch: int, rows_per_chunk=None):
+def run_chunked(wl: cf.Workload, schedule, scratch: int, rows_per_chunk=None, ring_direct=True):
     """schedule[b] = chunk lengths of sequence b (0 = the sequence sits that round out)."""
     mx, runner = load_lib()
     B = wl.batch
@@ -24,6 +24,7 @@ def run_chunked(wl: cf.Workload, schedule, scratch: int, rows_per_chunk=None):
     dt = torch_dt(wl.dtype)
     pos = [0] * B
     try:
+        sess.ctx.set_chunk_ring_direct(ring_direct)
         for rnd in range(max(len(s) for s in schedule)):
             ids = [b for b in range(B) if rnd < len(schedule[b]) and schedule[b][rnd] > 0]
             lens = [schedule[b][rnd] for b in ids]
@@ -87,19 +88,40 @@ def test_chunks_fp32_tiny_layout():
     run_chunked(wl, schedule, scratch=640)
 
 
-def test_chunks_bf16_tensor_core_path():
+@pytest.mark.parametrize("ring_direct", [True, False])
+def test_chunks_bf16_tensor_core_path(ring_direct):
     # head_dim 128, bf16: the tcgen05 kernel with a key prefix that is not a multiple of the
-    # tile (diagonal inside tiles), window 256 shared by a reader, several query tiles
+    # tile (diagonal inside tiles), window 256 shared by a reader, several query tiles; with the
+    # rings read in place and with every cached key copied first
     wl = cf.prefill_chunk().scaled(layout=cf.layout_tiny(256), batch=2, seq_len=0)
     schedule = [[300, 129, 1, 500, 77], [50, 700, 128, 4, 256]]
-    run_chunked(wl, schedule, scratch=2600)
+    run_chunked(wl, schedule, scratch=2600, ring_direct=ring_direct)
 
 
-def test_chunks_bf16_mid_layout_sampled_rows():
+@pytest.mark.parametrize("ring_direct", [True, False])
+def test_chunks_bf16_mid_layout_sampled_rows(ring_direct):
     # the 24-layer layout (two shared rings of 1024, one shared paged cache), longer prefixes
     wl = cf.prefill_chunk().scaled(batch=2, seq_len=0)
     schedule = [[1500, 1100, 130], [900, 2048, 1]]
-    run_chunked(wl, schedule, scratch=6000, rows_per_chunk=24)
+    run_chunked(wl, schedule, scratch=6000, rows_per_chunk=24, ring_direct=ring_direct)
+
+
+@pytest.mark.parametrize("window", [128, 384])
+def test_chunks_read_the_ring_in_place_at_every_kind_of_prefix(window):
+    # cached lengths that end on a tile edge, one token before and after it, inside the first
+    # tile, exactly at the window, and several turns of the ring later; chunks of one token, of
+    # less than a tile, of a tile and of several; three sequences at different offsets in one call
+    wl = cf.prefill_chunk().scaled(layout=cf.layout_tiny(window), batch=3, seq_len=0)
+    schedule = [[1, 126, 1, 1, 127, window - 1, 1, 2 * window + 77, 130, 5],
+                [128, 128, 1, window, 3, 0, 700, 1, 255, 256],
+                [0, 127, 2, 0, 129, 64, 64, 64, 1000, 1]]
+    run_chunked(wl, schedule, scratch=4096)
+
+
+def test_chunk_window_not_a_multiple_of_the_tile_still_copies():
+    # window 200: not a whole number of key tiles, so the call copies whatever the switch says
+    wl = cf.prefill_chunk().scaled(layout=cf.layout_tiny(200), batch=2, seq_len=0)
+    run_chunked(wl, [[300, 129, 1, 200], [50, 500, 128, 4]], scratch=2600, ring_direct=True)
 
 
 def test_chunk_errors():
@@ -171,13 +193,14 @@ def test_serving_trace_small():
         sess.close()
 
 
-@pytest.mark.parametrize("scratch_seqs", [2, 1])
-def test_gather_reuse_same_outputs_fewer_copies(scratch_seqs):
+@pytest.mark.parametrize("scratch_seqs,ring_direct", [(2, False), (1, False), (2, True)])
+def test_gather_reuse_same_outputs_fewer_copies(scratch_seqs, ring_direct):
     # Layers that share a cache gather the same rows: with reuse enabled the copy runs once per run
     # of such layers (6-layer layout: standard owner, ring owner, two ring readers, a reader of the
     # standard cache, a second ring owner = 4 copies per round instead of 6) and every output is
     # bit-identical.  With a scratch that holds one sequence at a time the call works in two
-    # pieces and must copy every time.
+    # pieces and must copy every time.  With the rings read in place only the two layers on the
+    # standard cache copy, and the second of them finds the first one's rows still in the scratch.
     mx, runner = load_lib()
     layout = [(cf.FULL, 0, 0), (cf.SLIDING, 256, 1), (cf.SLIDING, 256, 1), (cf.SLIDING, 256, 1),
               (cf.FULL, 0, 0), (cf.SLIDING, 256, 5)]
@@ -189,6 +212,7 @@ def test_gather_reuse_same_outputs_fewer_copies(scratch_seqs):
                               chunk_scratch_tokens=scratch_seqs * total if scratch_seqs == 2 else total + 8)
         try:
             sess.ctx.set_chunk_gather_reuse(reuse)
+            sess.ctx.set_chunk_ring_direct(ring_direct)
             sess.ctx.profile_enable(True)
             outs = sess.prefill_in_chunks(chunk)
             torch.cuda.synchronize()
@@ -202,7 +226,9 @@ def test_gather_reuse_same_outputs_fewer_copies(scratch_seqs):
     for a, b in zip(off, on):
         assert torch.equal(a.view(torch.int16), b.view(torch.int16))
     rounds = total // chunk
-    if scratch_seqs == 2:
+    if ring_direct:
+        assert n_off == 2 * rounds and n_on == 1 * rounds
+    elif scratch_seqs == 2:
         assert n_off == 6 * rounds and n_on == 4 * rounds
     else:
         # the first round (empty caches, 2 x 300 rows) still fits in one piece; the later rounds

@@ -181,6 +181,9 @@ def test_chunk_and_rope_calls_on_a_host_only_context():
     # the switch for sharing one copy among the layers of a cache is host state: settable without a
     # device, and it changes no check above
     assert mx.lib.mixattn_set_chunk_gather_reuse(None, 1) == mx.ERR_INVALID_ARG
+    assert mx.lib.mixattn_set_chunk_ring_direct(None, 1) == mx.ERR_INVALID_ARG
+    ctx.set_chunk_ring_direct(False)
+    ctx.set_chunk_ring_direct(True)
     ctx.set_chunk_gather_reuse(True)
     assert ctx.rc_attend_chunk(0, [0], [13], None, None, None, None) == mx.ERR_TOO_LARGE
     assert ctx.rc_attend_chunk(1, [0], [25], None, None, None, None) == mx.ERR_CUDA
