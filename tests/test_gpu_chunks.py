@@ -98,12 +98,12 @@ def test_chunks_bf16_tensor_core_path(ring_direct):
     run_chunked(wl, schedule, scratch=2600, ring_direct=ring_direct)
 
 
-@pytest.mark.parametrize("ring_direct", [True, False])
-def test_chunks_bf16_mid_layout_sampled_rows(ring_direct):
-    # the 24-layer layout (two shared rings of 1024, one shared paged cache), longer prefixes
+def test_chunks_bf16_mid_layout_sampled_rows():
+    # the 24-layer layout (two shared rings of 1024 read in place, one shared paged cache whose
+    # keys are copied), longer prefixes
     wl = cf.prefill_chunk().scaled(batch=2, seq_len=0)
     schedule = [[1500, 1100, 130], [900, 2048, 1]]
-    run_chunked(wl, schedule, scratch=6000, rows_per_chunk=24, ring_direct=ring_direct)
+    run_chunked(wl, schedule, scratch=6000, rows_per_chunk=24)
 
 
 @pytest.mark.parametrize("window", [128, 384])
