@@ -473,3 +473,27 @@ def test_logical_cache_prefill_records_for_owners_only():
         lc.prefill(0, 0, rnd(rng, S, Hq, D), K[0], V[0])
     assert ei.value.code == mo.ERR_UNSUPPORTED
     assert lc.history(0, 0)[0].shape[0] == S
+
+
+@pytest.mark.parametrize("window,whole_tiles", [(128, True), (384, True), (1024, True), (200, False), (64, False)])
+def test_a_tile_of_cached_positions_is_whole_ring_pages_iff_window_is_whole_tiles(window, whole_tiles):
+    # Section 3's sliding-window cache as the ring of `window` slots (token t in slot t mod window).
+    # What a kernel reading cached keys in place relies on: with 16-slot pages and a window that is
+    # a multiple of 128, the stored tokens of every aligned run of 128 positions sit in
+    # consecutive slots that start on a multiple of 128 (eight whole pages), for any length;
+    # for other windows some run wraps inside the ring or starts off a page boundary.
+    layout = [(cf.SLIDING, window, 0)]
+    always = True
+    for n in (1, 127, 128, 129, window - 1, window, window + 1, 3 * window + 77, 5 * window):
+        if n < 1:
+            continue
+        ph = mo.PhysicalCache(layout, 1, 8, 1, 1, max_seq_len=8192, store_values=False)
+        ph.append(0, [0], [n])
+        lo = max(0, n - window)
+        for t in range(lo // 128, (n - 1) // 128 + 1):
+            stored = [p for p in range(128 * t, 128 * t + 128) if lo <= p < n]
+            slots = [ph.locate(0, 0, p)[1] for p in stored]
+            first = slots[0] - (stored[0] - 128 * t)       # slot the tile's first position would have
+            ok = first % 128 == 0 and first + 128 <= window and slots == [first + (p - 128 * t) for p in stored]
+            always = always and ok
+    assert always == whole_tiles
