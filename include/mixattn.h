@@ -215,10 +215,10 @@ int mixattn_decode_layers(mixattn_ctx* ctx, int32_t layer_begin, int32_t layer_e
  * would (a ring ends up holding the last min(S_b, window) tokens); the
  * owner's cache for these sequences must be empty, else UNSUPPORTED.  A
  * reader stores nothing.  Errors: as append_kv and decode.
- * Performance note: bf16 with head_dim 128 and 16-byte aligned tensors runs
- * on the tensor cores; fp32 contexts, head_dim 64 and unaligned tensors take
- * an exact CUDA-core kernel that is about two orders of magnitude slower
- * (the same holds for mixattn_attend_chunk). */
+ * Performance note: bf16 (head_dim 128 or 64) with 16-byte aligned tensors
+ * runs on the tensor cores; fp32 contexts and unaligned tensors take an exact
+ * CUDA-core kernel that is about two orders of magnitude slower (the same
+ * holds for mixattn_attend_chunk). */
 int mixattn_prefill(mixattn_ctx* ctx, int32_t layer, int32_t n_seqs, const int32_t* seq_ids,
                     const int32_t* seq_lens, const void* q, const void* k, const void* v,
                     void* out, void* stream);
@@ -241,7 +241,7 @@ int mixattn_prefill(mixattn_ctx* ctx, int32_t layer, int32_t n_seqs, const int32
  * The cached keys the chunk needs (all of a paged cache, the last window-1
  * tokens of a ring) and the chunk's are first copied into plain tensors in the
  * context's chunk scratch, sequences in groups that fit it.  Exception: a ring
- * whose window is a multiple of 128 tokens (bf16, head_dim 128, native storage)
+ * whose window is a multiple of 128 tokens (bf16, native storage)
  * is read in place, see mixattn_set_chunk_ring_direct; the size rules below
  * are the same either way.
  * Errors: UNSUPPORTED if the context was created with chunk_scratch_tokens = 0,
@@ -272,7 +272,7 @@ int mixattn_set_chunk_gather_reuse(mixattn_ctx* ctx, int32_t enable);
  * tile of cached keys is eight whole pages of the sequence's ring, stored in
  * the layout the tensor cores read; the kernel then fetches those tiles from
  * the ring itself and the chunk's own K/V from the caller's tensors.  Applies
- * to bf16 contexts with head_dim 128 and native KV storage; every other chunk
+ * to bf16 contexts with native KV storage; every other chunk
  * call copies as described above.  On by default; enable = 0 makes every chunk
  * call copy.  Both ways attend to the same keys; the results differ by
  * rounding only (the keys are cut into tiles at different places).

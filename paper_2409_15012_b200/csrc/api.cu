@@ -575,8 +575,7 @@ int mixattn_prefill(mixattn_ctx* c, int32_t layer, int32_t n_seqs, const int32_t
     p.v = static_cast<const char*>(v) + (size_t)row * Hkv * D * esz;
     row += r;
     const int cls = p.window ? MIXATTN_K_PREFILL_SLIDING : MIXATTN_K_PREFILL_FULL;
-    // bf16 with head_dim 128 runs on the tensor-core kernel; everything else (fp32 mode,
-    // head_dim 64) on the exact CUDA-core kernel
+    // bf16 runs on the tensor-core kernel, fp32 mode on the exact CUDA-core kernel
     const bool tc = prefill_tc_supported(c->cfg.dtype, D, p.q, p.k, p.v) && (((size_t)p.out) & 15) == 0;
     cudaError_t e = launch_recorded(c, cls, st, [&] {
       return tc ? launch_prefill_tc(p, mlen, c->sm_count, st) : launch_prefill_simple(p, c->cfg.dtype, mlen, st);

@@ -1,4 +1,5 @@
-// Prompt attention on the 5th-generation tensor cores (tcgen05 + TMEM), bf16, head_dim 128.
+// Prompt attention on the 5th-generation tensor cores (tcgen05 + TMEM), bf16, head_dim 128 or 64
+// (described for 128; the 64-channel form is noted at the kernel).
 //
 // Paper, Section 3 with the causal order of Section 1: query i attends to keys j <= i
 // (standard layer) or i - window < j <= i (sliding window).  Flash-attention forward:
@@ -228,9 +229,9 @@ __device__ __forceinline__ void split_bf16(float x, float y, uint32_t& hi, uint3
   lo = pack_bf16(x - __uint_as_float(hi << 16), y - __uint_as_float(hi & 0xffff0000u));
 }
 
-// instruction descriptor: D fp32, A/B bf16, M = 128, N = 128; b_mn = 1 for an MN-major B
-__host__ __device__ constexpr uint32_t idesc_bf16(int b_mn) {
-  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)b_mn << 16) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
+// instruction descriptor: D fp32, A/B bf16, M = 128, N = n; b_mn = 1 for an MN-major B
+__host__ __device__ constexpr uint32_t idesc_bf16(int b_mn, uint32_t n = 128) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)b_mn << 16) | ((n >> 3) << 17) | ((128u >> 4) << 24);
 }
 
 // One work item: query tile qt of head h of sequence b.  Ids enumerate (sequence, reverse
@@ -291,11 +292,17 @@ __device__ __forceinline__ int tile_of(const WorkItem& w, int j) {
 
 // kRing: some sequences have cached keys in a ring (a separate instantiation, so that the
 // ordinary launches carry none of its code)
-template <bool kRing>
+// kD: head_dim, 128 or 64.  With 64 channels an operand tile is one [128 x 64] block instead of
+// two (the buffers keep their size), the score product takes four steps of 16 channels, the
+// P V products write 64 accumulator columns, and the softmax warps do exactly the same work.
+template <bool kRing, int kD>
 __global__ void __launch_bounds__(kThreads, 1)
 prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                   const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_ring,
                   const __grid_constant__ TcParams p) {
+  static_assert(kD == 128 || kD == 64, "head_dim");
+  constexpr uint32_t kOpBytes = kD == 128 ? kTileBytes : kHalfBytes;   // bytes of one Q / K / V tile
+  constexpr int kSteps = kD / 16;                                        // 16-channel steps of the score product
   extern __shared__ __align__(1024) unsigned char smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   unsigned char* gbase = smem_raw + (base - smem_u32(smem_raw));
@@ -359,9 +366,9 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
           const int qb = it & 1;
           if (it >= 2) ok = mbar_wait(BAR(B_QE + qb), ((it >> 1) - 1) & 1, abort_flag);
           if (!ok) break;
-          mbar_expect_tx(BAR(B_QF + qb), kTileBytes);
+          mbar_expect_tx(BAR(B_QF + qb), kOpBytes);
           tma_load_3d(base + kSmQ + qb * kTileBytes, &tm_q, 0, w.h, w.row_base + w.i0, BAR(B_QF + qb));
-          tma_load_3d(base + kSmQ + qb * kTileBytes + kHalfBytes, &tm_q, 64, w.h, w.row_base + w.i0, BAR(B_QF + qb));
+          if (kD == 128) tma_load_3d(base + kSmQ + qb * kTileBytes + kHalfBytes, &tm_q, 64, w.h, w.row_base + w.i0, BAR(B_QF + qb));
           ++q_issued;
           for (int j = 0; j < w.n_tiles && ok; ++j) {
             const int Gj = G + j;
@@ -376,25 +383,25 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
             const int ks = Gj % kKStages, ku = Gj / kKStages;
             if (ku > 0) ok = mbar_wait(BAR(B_KE + ks), (ku - 1) & 1, abort_flag);
             if (!ok) break;
-            mbar_expect_tx(BAR(B_KF + ks), kTileBytes);
+            mbar_expect_tx(BAR(B_KF + ks), kOpBytes);
             if (from_ring) {
               tma_load_5d(base + kSmK + ks * kTileBytes, &tm_ring, 0, 0, 0, w.g, page, BAR(B_KF + ks));
-              tma_load_5d(base + kSmK + ks * kTileBytes + kHalfBytes, &tm_ring, 64, 0, 0, w.g, page, BAR(B_KF + ks));
+              if (kD == 128) tma_load_5d(base + kSmK + ks * kTileBytes + kHalfBytes, &tm_ring, 64, 0, 0, w.g, page, BAR(B_KF + ks));
             } else {
               tma_load_3d(base + kSmK + ks * kTileBytes, &tm_k, 0, w.g, row, BAR(B_KF + ks));
-              tma_load_3d(base + kSmK + ks * kTileBytes + kHalfBytes, &tm_k, 64, w.g, row, BAR(B_KF + ks));
+              if (kD == 128) tma_load_3d(base + kSmK + ks * kTileBytes + kHalfBytes, &tm_k, 64, w.g, row, BAR(B_KF + ks));
             }
             ++k_issued;
             const int vs = Gj % kVStages, vu = Gj / kVStages;
             if (vu > 0) ok = mbar_wait(BAR(B_VE + vs), (vu - 1) & 1, abort_flag);
             if (!ok) break;
-            mbar_expect_tx(BAR(B_VF + vs), kTileBytes);
+            mbar_expect_tx(BAR(B_VF + vs), kOpBytes);
             if (from_ring) {
               tma_load_5d(base + kSmV + vs * kTileBytes, &tm_ring, 0, 0, 1, w.g, page, BAR(B_VF + vs));
-              tma_load_5d(base + kSmV + vs * kTileBytes + kHalfBytes, &tm_ring, 64, 0, 1, w.g, page, BAR(B_VF + vs));
+              if (kD == 128) tma_load_5d(base + kSmV + vs * kTileBytes + kHalfBytes, &tm_ring, 64, 0, 1, w.g, page, BAR(B_VF + vs));
             } else {
               tma_load_3d(base + kSmV + vs * kTileBytes, &tm_v, 0, w.g, row, BAR(B_VF + vs));
-              tma_load_3d(base + kSmV + vs * kTileBytes + kHalfBytes, &tm_v, 64, w.g, row, BAR(B_VF + vs));
+              if (kD == 128) tma_load_3d(base + kSmV + vs * kTileBytes + kHalfBytes, &tm_v, 64, w.g, row, BAR(B_VF + vs));
             }
             ++v_issued;
           }
@@ -425,9 +432,9 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
           if (!w.valid) continue;
           const int qb = it & 1;
           ok = mbar_wait(BAR(B_QF + qb), (it >> 1) & 1, abort_flag);
-          uint64_t qdesc[8];
+          uint64_t qdesc[kSteps];
   #pragma unroll
-          for (int ks = 0; ks < 8; ++ks)   // head_dim 128 = 8 steps of 16 channels
+          for (int ks = 0; ks < kSteps; ++ks)   // head_dim = kSteps steps of 16 channels
             qdesc[ks] = smem_desc(base + kSmQ + qb * kTileBytes + (ks >> 2) * kHalfBytes + (ks & 3) * 32, 16, 1024);
           for (int j = 0; j < w.n_tiles && ok; ++j) {
             // S(G) = Q K^T into S buffer G & 1, which held S(G-2) / P(G-2): wait until both
@@ -439,7 +446,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
             tc_fence_after();
             const uint64_t kdesc = smem_desc(base + kSmK + ks_ * kTileBytes, 16, 1024);
   #pragma unroll
-            for (int ks = 0; ks < 8; ++ks)
+            for (int ks = 0; ks < kSteps; ++ks)
               umma_bf16(tmem + kColS + sb * 128, qdesc[ks],
                         kdesc + (uint64_t)((ks >> 2) * (kHalfBytes >> 4) + (ks & 3) * 2), kIdescS, ks > 0);
             umma_commit(BAR(B_SF + sb));    // scores ready
@@ -454,7 +461,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     } else {
       // ------------------------------ MMA issuers, P V (one per stream) ------------------------------
       if (lane == 0) {
-        constexpr uint32_t kIdescPV = idesc_bf16(1);
+        constexpr uint32_t kIdescPV = idesc_bf16(1, kD);
         const int hs = warp - 2;
         bool ok = true;
         int G = 0, it = 0;
@@ -519,14 +526,14 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
       const float inv = 1.f / (lo.y * e_lo + hi.y * e_hi);
       const float w_lo = e_lo * inv, w_hi = e_hi * inv;
       const int i = w.i0 + r;
-      __nv_bfloat16* orow = p.out + ((int64_t)(w.row_base + i) * p.n_q_heads + w.h) * 128;
+      __nv_bfloat16* orow = p.out + ((int64_t)(w.row_base + i) * p.n_q_heads + w.h) * kD;
 #pragma unroll
-      for (int c = 0; c < 4; ++c) {
+      for (int c = 0; c < kD / 32; ++c) {
         uint32_t olo[32], ohi[32];
         tmem_ld32(lane_base + kColO + c * 32, olo);
         tmem_ld32(lane_base + kColO + 128 + c * 32, ohi);
         tmem_wait_ld();
-        if (c == 3) {   // the accumulators may be overwritten by the next item
+        if (c == kD / 32 - 1) {   // the accumulators may be overwritten by the next item
           tc_fence_before();
           __syncwarp();
           if (lane == 0) mbar_arrive(BAR(B_OR));
@@ -667,7 +674,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
               if (!__all_sync(0xffffffffu, mbar_wait(BAR(B_SR + (sb ^ 1)), ((Gj - 1) >> 1) & 1, abort_flag))) { ok = false; break; }
               tc_fence_after();
   #pragma unroll 1
-              for (int c = 0; c < 4; ++c) {
+              for (int c = 0; c < kD / 32; ++c) {
                 uint32_t ov[32];
                 tmem_ld32(o_addr + c * 32, ov);
                 tmem_wait_ld();
@@ -754,12 +761,12 @@ EncodeTiledFn encode_fn() {
   return fn;
 }
 
-// [rows, heads, 128] bf16 tensor; box = 64 channels x 1 head x 128 rows, 128-byte swizzle
-bool make_map(CUtensorMap* map, const void* ptr, int64_t rows, int heads) {
+// [rows, heads, D] bf16 tensor; box = 64 channels x 1 head x 128 rows, 128-byte swizzle
+bool make_map(CUtensorMap* map, const void* ptr, int64_t rows, int heads, int D) {
   EncodeTiledFn fn = encode_fn();
   if (fn == nullptr) return false;
-  cuuint64_t dims[3] = {128, (cuuint64_t)heads, (cuuint64_t)rows};
-  cuuint64_t strides[2] = {128 * 2, (cuuint64_t)heads * 128 * 2};
+  cuuint64_t dims[3] = {(cuuint64_t)D, (cuuint64_t)heads, (cuuint64_t)rows};
+  cuuint64_t strides[2] = {(cuuint64_t)D * 2, (cuuint64_t)heads * D * 2};
   cuuint32_t box[3] = {64, 1, 128};
   cuuint32_t estr[3] = {1, 1, 1};
   return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, estr,
@@ -767,14 +774,14 @@ bool make_map(CUtensorMap* map, const void* ptr, int64_t rows, int heads) {
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-// Ring storage of one owner layer, native bf16 format with head_dim 128, seen as
-// [pages][heads][K | V][16 tokens][128 channels]; box = 64 channels x 16 tokens x 8 pages of one
+// Ring storage of one owner layer, native bf16 format, seen as
+// [pages][heads][K | V][16 tokens][head_dim channels]; box = 64 channels x 16 tokens x 8 pages of one
 // head's K or V.  The stored rows carry the 128-byte-swizzle permutation already (internal.h),
 // so the copy itself does not swizzle.
 bool make_ring_map(CUtensorMap* map, const void* pool, const KvGeom& ge, int64_t pages) {
   EncodeTiledFn fn = encode_fn();
   if (fn == nullptr) return false;
-  cuuint64_t dims[5] = {128, (cuuint64_t)kPage, 2, (cuuint64_t)ge.n_kv_heads, (cuuint64_t)pages};
+  cuuint64_t dims[5] = {(cuuint64_t)ge.head_dim, (cuuint64_t)kPage, 2, (cuuint64_t)ge.n_kv_heads, (cuuint64_t)pages};
   cuuint64_t strides[4] = {(cuuint64_t)ge.row_bytes, (cuuint64_t)kPage * ge.row_bytes, (cuuint64_t)ge.blk_bytes,
                            (cuuint64_t)ge.page_bytes};
   cuuint32_t box[5] = {64, (cuuint32_t)kPage, 1, 1, kBN / kPage};
@@ -787,18 +794,20 @@ bool make_ring_map(CUtensorMap* map, const void* pool, const KvGeom& ge, int64_t
 }  // namespace
 
 bool prefill_tc_ring_direct_supported(const KvGeom& ge, int window) {
-  return !ge.fp8 && ge.swizzle && ge.head_dim == 128 && ge.elem_bytes == 2 && window > 0 && window % kBN == 0;
+  return !ge.fp8 && ge.swizzle && (ge.head_dim == 128 || ge.head_dim == 64) && ge.elem_bytes == 2 && window > 0 && window % kBN == 0;
 }
 
 bool prefill_tc_supported(int dtype, int head_dim, const void* q, const void* k, const void* v) {
   auto aligned = [](const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; };
-  return dtype == MIXATTN_BF16 && head_dim == 128 && aligned(q) && aligned(k) && aligned(v) && encode_fn() != nullptr;
+  return dtype == MIXATTN_BF16 && (head_dim == 128 || head_dim == 64) && aligned(q) && aligned(k) && aligned(v) && encode_fn() != nullptr;
 }
 
 cudaError_t prepare_prefill_tc() {
-  cudaError_t e = cudaFuncSetAttribute(prefill_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
-  if (e != cudaSuccess) return e;
-  return cudaFuncSetAttribute(prefill_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+  cudaError_t e = cudaFuncSetAttribute(prefill_tc_kernel<false, 128>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(prefill_tc_kernel<true, 128>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(prefill_tc_kernel<false, 64>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(prefill_tc_kernel<true, 64>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+  return e;
 }
 
 cudaError_t launch_prefill_tc(const PrefillParams& pp, int max_len, int sm_count, cudaStream_t st) {
@@ -812,8 +821,10 @@ cudaError_t launch_prefill_tc(const PrefillParams& pp, int max_len, int sm_count
     if (end > k_rows) k_rows = end;
   }
   CUtensorMap tq, tk, tv, tring;
-  if (!make_map(&tq, pp.q, rows, pp.n_q_heads) || !make_map(&tk, pp.k, k_rows, pp.n_kv_heads) ||
-      !make_map(&tv, pp.v, k_rows, pp.n_kv_heads))
+  const int D = pp.head_dim;
+  if (D != 128 && D != 64) return cudaErrorInvalidValue;
+  if (!make_map(&tq, pp.q, rows, pp.n_q_heads, D) || !make_map(&tk, pp.k, k_rows, pp.n_kv_heads, D) ||
+      !make_map(&tv, pp.v, k_rows, pp.n_kv_heads, D))
     return cudaErrorInvalidValue;
   if (pp.ring_pool != nullptr) {
     if (!prefill_tc_ring_direct_supported(pp.geom, pp.window) || pp.ring_pages * kPage != pp.window ||
@@ -841,8 +852,14 @@ cudaError_t launch_prefill_tc(const PrefillParams& pp, int max_len, int sm_count
   p.max_qt = (max_len + kBM - 1) / kBM;
   const int64_t n_ids = (int64_t)p.max_qt * pp.n_seqs * pp.n_q_heads;
   const int grid = (int)(n_ids < sm_count ? n_ids : sm_count);   // persistent: one CTA per SM
-  if (pp.ring_pool != nullptr) prefill_tc_kernel<true><<<grid, kThreads, kSmemBytes, st>>>(tq, tk, tv, tring, p);
-  else prefill_tc_kernel<false><<<grid, kThreads, kSmemBytes, st>>>(tq, tk, tv, tring, p);
+  const bool ring = pp.ring_pool != nullptr;
+  if (D == 128) {
+    if (ring) prefill_tc_kernel<true, 128><<<grid, kThreads, kSmemBytes, st>>>(tq, tk, tv, tring, p);
+    else prefill_tc_kernel<false, 128><<<grid, kThreads, kSmemBytes, st>>>(tq, tk, tv, tring, p);
+  } else {
+    if (ring) prefill_tc_kernel<true, 64><<<grid, kThreads, kSmemBytes, st>>>(tq, tk, tv, tring, p);
+    else prefill_tc_kernel<false, 64><<<grid, kThreads, kSmemBytes, st>>>(tq, tk, tv, tring, p);
+  }
   return cudaGetLastError();
 }
 

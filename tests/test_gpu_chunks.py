@@ -118,6 +118,12 @@ def test_chunks_read_the_ring_in_place_at_every_kind_of_prefix(window):
     run_chunked(wl, schedule, scratch=4096)
 
 
+def test_chunks_bf16_head_dim_64():
+    # 64-channel heads: rings read in place (pages of 16 x 128-byte rows), paged caches copied
+    wl = cf.prefill_chunk().scaled(layout=cf.layout_tiny(256), batch=2, seq_len=0, n_q_heads=8, n_kv_heads=2, head_dim=64)
+    run_chunked(wl, [[300, 129, 1, 500, 77], [50, 700, 128, 4, 256]], scratch=2600)
+
+
 def test_chunk_window_not_a_multiple_of_the_tile_still_copies():
     # window 200: not a whole number of key tiles, so the call copies whatever the switch says
     wl = cf.prefill_chunk().scaled(layout=cf.layout_tiny(200), batch=2, seq_len=0)

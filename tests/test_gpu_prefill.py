@@ -66,6 +66,13 @@ def test_prefill_bf16_small(S, W):
     run_prefill_case(wl)
 
 
+@pytest.mark.parametrize("S,W", [(700, 256), (333, 1024), (129, 128)])
+def test_prefill_bf16_head_dim_64(S, W):
+    # the tensor-core kernel's 64-channel form: one operand block per tile, 64 accumulator columns
+    wl = cf.prefill_chunk().scaled(layout=cf.layout_tiny(W), batch=2, seq_len=S, n_q_heads=12, n_kv_heads=3, head_dim=64)
+    run_prefill_case(wl)
+
+
 def test_prefill_bf16_mid_layout_small():
     wl = cf.prefill_chunk().scaled(layout=cf.layout_mid(256, 6), batch=2, seq_len=600)
     rows = [0, 1, 127, 128, 255, 256, 257, 599] + list(range(300, 340))
@@ -104,9 +111,9 @@ def _prefill_direct(mx, wl, seq_lens, layer):
 
 
 @pytest.mark.parametrize("hq,hkv,d,dtype", [(8, 8, 128, cf.BF16), (12, 3, 128, cf.BF16), (2, 1, 128, cf.BF16),
-                                            (8, 2, 64, cf.BF16), (6, 3, 128, cf.F32)])
+                                            (8, 2, 64, cf.BF16), (16, 1, 64, cf.BF16), (6, 3, 128, cf.F32), (6, 3, 64, cf.F32)])
 def test_prefill_head_shapes_and_ragged_lengths(hq, hkv, d, dtype):
-    # MHA, the paper's 12/3, a single pair, head_dim 64 (CUDA-core path), fp32; sequences of
+    # MHA, the paper's 12/3, a single pair, head_dim 64, fp32 (CUDA-core path); sequences of
     # different lengths packed in one call, one of them a single token
     mx, runner = load_lib()
     seq_lens = [333, 129, 1, 128]
