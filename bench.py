@@ -39,6 +39,7 @@ from synth import inputs as si
 
 METRIC = "decode attention HBM GB/s (% of peak) & tokens/s; prefill TFLOP/s (% bf16 peak)"
 NOMINAL_BF16_TFLOPS = 2250.0     # dense bf16 datasheet figure of a B200 (context; fractions of it are reported too)
+BURST_IDLE_S = 0.5   # idle time before each short tensor-core measurement (see prefill_figures)
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 # (dram__bytes_read.sum + dram__bytes_write.sum) / algorithmic KV bytes of the dominant kernel, from an
@@ -55,6 +56,7 @@ def load_peaks():
         with open(path) as f:
             d = json.load(f)
         d["_source"] = "measured"
+        d.setdefault("bf16_tflops_sustained", FALLBACK_PEAKS["bf16_tflops_sustained"])
         return d
     d = dict(FALLBACK_PEAKS)
     d["_source"] = "fallback"
@@ -231,6 +233,10 @@ def prefill_figures(mx, runner, peaks, device):
             q, k, v = sess.prefill_inputs(layer)      # readers: no cache writes, repeatable
             out = torch.empty_like(q)
             reps = 20
+            # a burst figure, read against a burst peak that was measured on an otherwise idle GPU:
+            # let the board's power average fall back before each one
+            torch.cuda.synchronize()
+            time.sleep(BURST_IDLE_S)
             for _ in range(3):
                 sess.prefill_layer(layer, q, k, v, out)
             torch.cuda.synchronize()
@@ -253,6 +259,35 @@ def prefill_figures(mx, runner, peaks, device):
     finally:
         sess.close()
     return res
+
+
+def prefill_sustained(mx, runner, peaks, device, res):
+    """The launches of prefill_figures last 12-40 ms each way: bursts, read against the burst
+    peak.  Here the same launch is repeated for about 1.5 s, which settles at the clock the power
+    limit allows; the last two thirds of the loop are read against the sustained peak.  Runs after
+    every burst measurement, so that none of them starts on a GPU a long loop has just driven to
+    its power limit."""
+    wl = cf.prefill_chunk()
+    sess = runner.Session(wl, [0] * wl.batch, device=device)
+    try:
+        for name, layer, cls in (("full", 12, mx.K_PREFILL_FULL), ("sliding", 2, mx.K_PREFILL_SLIDING)):
+            q, k, v = sess.prefill_inputs(layer)
+            out = torch.empty_like(q)
+            n_loop = max(30, int(1500.0 / res[name]["ms_per_layer"]))
+            for _ in range(n_loop // 3):
+                sess.prefill_layer(layer, q, k, v, out)
+            sess.ctx.profile_enable(True)
+            for _ in range(n_loop - n_loop // 3):
+                sess.prefill_layer(layer, q, k, v, out)
+            n_s, ms_s = sess.ctx.profile_read(cls)
+            sess.ctx.profile_enable(False)
+            tf_s = res[name]["useful_flop"] / (ms_s / n_s * 1e-3) / 1e12
+            res[name]["sustained"] = {"tflops": tf_s, "ms_per_layer": ms_s / n_s, "launches_timed": n_s,
+                                      "frac_of_bf16_peak_sustained": tf_s / peaks["bf16_tflops_sustained"]}
+        res["target_half_of_measured_sustained_met"] = res["sliding"]["sustained"]["frac_of_bf16_peak_sustained"] >= 0.5
+        res["peak_tflops_sustained"] = peaks["bf16_tflops_sustained"]
+    finally:
+        sess.close()
 
 
 def chunk_figures(mx, runner, peaks, device, prefix=6144, chunk=2048):
@@ -281,6 +316,8 @@ def chunk_figures(mx, runner, peaks, device, prefix=6144, chunk=2048):
             K, V = K.reshape(-1, wl.n_kv_heads, D), V.reshape(-1, wl.n_kv_heads, D)
             out = torch.empty_like(q)
             reps = 10
+            torch.cuda.synchronize()
+            time.sleep(BURST_IDLE_S)
             for _ in range(2):
                 sess.ctx.attend_chunk(layer, ids, lens, q, K, V, out)
             torch.cuda.synchronize()
@@ -651,6 +688,8 @@ def run_gpu_arm(args, wl):
             sess.close()
             closed = True
         others = other_workload_figures(runner, peaks, local, min(K, 20), Wm)
+    if prefill is not None:
+        prefill_sustained(mx, runner, peaks, local, prefill)   # last: it leaves the GPU at its power limit
 
     line = {
         "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": K, "warmup": Wm,
